@@ -1,0 +1,199 @@
+/*
+ * libcstr - regular-language constraints for batched LM decoding on one GPU.
+ *
+ * The library holds the data-parallel part of the automata-based constraint
+ * method of "Automata-based constraints for language model decoding":
+ *
+ *   1. the token-level automaton: the composition of a character (byte) DFA
+ *      with the vocabulary's detokenizer, emitted densely as
+ *          next[q][v] = delta*(q, bytes(v))      (-1 = no edge)
+ *          mask[q] bit v = (next[q][v] != -1)
+ *      for every DFA state q and vocabulary token v;
+ *   2. the per-step recipe: mask from the current state, penalise the logits
+ *      with -infinity, select a token, advance the state - for a whole batch.
+ *
+ * Conventions
+ *   - Every function returns 0 (CSTR_OK) or a negative CSTR_ERR_* code and
+ *     never throws, aborts or traps; cstr_last_error() gives a message for the
+ *     calling thread's last failure.
+ *   - "HOST" / "DEVICE" says where a pointer must point.  The caller owns all
+ *     such arrays; the library owns what is behind its opaque handles and frees
+ *     it in the matching cstr_free_*.  Handles are bound to the CUDA device
+ *     that was current when they were created; that device must be current in
+ *     later calls.
+ *   - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
+ *   - S = DFA states, V = vocabulary size, W = ceil(V / 32) mask words.
+ */
+#ifndef CSTR_H
+#define CSTR_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CSTR_OK 0
+#define CSTR_ERR_NULL (-1)      /* a required pointer was NULL                        */
+#define CSTR_ERR_ARG (-2)       /* a size / index argument is out of range            */
+#define CSTR_ERR_DFA (-3)       /* transition target outside [-1, S)                  */
+#define CSTR_ERR_VOCAB (-4)     /* offsets decreasing, negative or too large          */
+#define CSTR_ERR_DTYPE (-5)     /* unknown logits dtype                               */
+#define CSTR_ERR_SHAPE (-6)     /* ld < V, tables with different V, capacity exceeded */
+#define CSTR_ERR_CUDA (-7)      /* a CUDA runtime call failed                         */
+#define CSTR_ERR_NOMEM (-8)     /* host or device allocation failed                   */
+#define CSTR_ERR_DEVICE (-9)    /* handle belongs to another CUDA device              */
+
+#define CSTR_F32 0              /* logits are IEEE fp32                               */
+#define CSTR_BF16 1             /* logits are bfloat16                                */
+
+#define CSTR_MAX_TABLES 16      /* tables one cstr_step call can mix                  */
+
+typedef struct cstr_dfa cstr_dfa_t;             /* device copy of a byte-level DFA            */
+typedef struct cstr_vocab cstr_vocab_t;         /* device copy of a vocabulary                */
+typedef struct cstr_table cstr_table_t;         /* device mask[S][W] + next[S][V]             */
+typedef struct cstr_workspace cstr_workspace_t; /* per-stream scratch of cstr_step            */
+
+/* ------------------------------------------------------------------ DFA */
+
+/*
+ * Load a deterministic byte-level FSA (Section 2.1: an FSA (Sigma, Q, I, F, E)
+ * that is deterministic has no epsilon edge and at most one edge per state and
+ * symbol, so it is a table).  Sigma is the 256 byte values.
+ *   trans        HOST  int32 [n_states][256], target state or -1 (no edge)
+ *   accept       HOST  uint8 [n_states], non-zero = final state
+ *   n_states     >= 1;  start_state in [0, n_states)
+ * Validates every target, copies to the device (int16 entries when
+ * n_states <= 32767, else int32) and returns the handle in *out.
+ * Synchronous; allocates device memory.
+ */
+int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
+                  int32_t start_state, cstr_dfa_t **out);
+void cstr_free_dfa(cstr_dfa_t *dfa);
+
+/* ---------------------------------------------------------------- vocab */
+
+/*
+ * Load a vocabulary: token v detokenizes to vocab_bytes[offsets[v] ..
+ * offsets[v+1]) (App. B.1: each token has one character sequence d(v); the
+ * detokenization of a token sequence is the concatenation).  This is the
+ * vocabulary-specific half of the method, prepared once per LM like the
+ * detokenizing transducer T_V of Algorithm 1 (Section 2.4, "can easily be
+ * pre-computed for each LM").
+ *   vocab_bytes  HOST  uint8 [offsets[vocab_size]]
+ *   offsets      HOST  int64 [vocab_size + 1], offsets[0] == 0, non-decreasing,
+ *                total below 2^31
+ * Duplicate strings are allowed (each id gets its own column).  A token of
+ * length 0 never has an edge.  Synchronous; allocates device memory.
+ */
+int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offsets, int32_t vocab_size,
+                    cstr_vocab_t **out);
+void cstr_free_vocab(cstr_vocab_t *vocab);
+
+/* ---------------------------------------------------------------- table */
+
+/*
+ * Allocate an empty token table able to hold up to max_states states over
+ * `vocab`.  `vocab` must outlive every cstr_table_build on this table.
+ */
+int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states, cstr_table_t **out);
+
+/*
+ * Build the token-level automaton A_{R o V} = Determinize(A_R o T_V) of
+ * Algorithm 2 in its dense form (Theorem 2 fixes its meaning: a token sequence
+ * is accepted iff its detokenization is accepted by the DFA):
+ *     next[q][v] = state reached from q by reading bytes(v), -1 as soon as a
+ *                  byte has no edge or if the token is empty
+ *     mask[q] word v/32 bit v%32 (LSB first) = next[q][v] != -1; unused high
+ *                  bits of the last word are 0
+ * If eos_id >= 0, that token's bytes are ignored: it is allowed exactly in
+ * accepting states and leads to -1 ("finished").
+ * Only enqueues kernels on cuda_stream: no allocation, no host synchronisation.
+ * The table may be rebuilt any number of times (dfa->n_states <= max_states);
+ * it must not be in use by a cstr_step that has not completed.
+ */
+int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                     void *cuda_stream);
+
+/*
+ * One-call form: load the vocabulary from HOST arrays (as cstr_load_vocab),
+ * create a table sized for `dfa` and build it.  The table owns its private
+ * vocabulary copy.  Allocates; the build itself is enqueued on cuda_stream.
+ */
+int cstr_build_token_table(const cstr_dfa_t *dfa, const uint8_t *vocab_bytes,
+                           const int64_t *offsets, int32_t vocab_size, int32_t eos_id,
+                           void *cuda_stream, cstr_table_t **out);
+
+/* Shape of the automaton the table currently holds (any pointer may be NULL). */
+int cstr_table_info(const cstr_table_t *table, int32_t *n_states, int32_t *vocab_size,
+                    int32_t *mask_words, int32_t *start_state);
+
+/*
+ * Copy states [state_lo, state_hi) of a built table to the host in logical
+ * form, whatever the device layout is:
+ *   mask_host  HOST uint32 [(state_hi-state_lo)][W]      or NULL
+ *   next_host  HOST int32  [(state_hi-state_lo)][V]      or NULL   (-1 = no edge)
+ * Synchronises cuda_stream first.
+ */
+int cstr_table_download(const cstr_table_t *table, int32_t state_lo, int32_t state_hi,
+                        uint32_t *mask_host, int32_t *next_host, void *cuda_stream);
+void cstr_free_table(cstr_table_t *table);
+
+/* ----------------------------------------------------------------- step */
+
+/*
+ * Scratch for cstr_step: 16 bytes per row plus status counters, zeroed.  Use
+ * one workspace per stream; two steps that may overlap on the GPU must not
+ * share one.
+ */
+int cstr_workspace_create(int32_t max_batch, cstr_workspace_t **out);
+void cstr_free_workspace(cstr_workspace_t *ws);
+
+/*
+ * One constrained decoding step for `batch` independent rows (Algorithm 2,
+ * loop body; the three-step recipe of Section 1), in one kernel:
+ *   A      = tokens v with mask bit set for the row's state q
+ *   masked = logits where v in A, -infinity elsewhere (allowed entries are bit
+ *            copies, NaN payloads and -0 included)
+ *   token  = argmax over v in A of fp32(logits[v]) (+ noise[v], one rounded
+ *            fp32 addition); equal values: lowest id; NaN never wins; an allowed
+ *            -infinity still beats "none"
+ *   q      = next[q][token]
+ *
+ *   tables, n_tables  HOST array of 1..CSTR_MAX_TABLES built tables with equal V
+ *   row_table   DEVICE int32 [batch] table index per row, or NULL (all rows: tables[0])
+ *   logits      DEVICE [batch][ld] of `dtype`; ld >= V is the row stride in elements
+ *   noise       DEVICE float [batch][ld] or NULL (greedy); e.g. Gumbel noise for sampling
+ *   states      DEVICE int32 [batch], in/out; all rows of a fresh sequence start
+ *               at the table's start state
+ *   tokens_out  DEVICE int32 [batch]
+ *   masked_out  DEVICE [batch][ld] of `dtype`; columns >= V are not written; may be
+ *               the same buffer as logits (exactly equal pointers, in-place)
+ *   accept_out  DEVICE uint8 [batch] or NULL: 1 iff the new state is accepting
+ * A row whose state is -1 (finished / inactive), out of range, or whose table
+ * index is out of range, and a row with no selectable token, get token -1,
+ * state -1 and all -infinity; nothing out of bounds is ever touched.
+ * Only enqueues work on cuda_stream (no allocation, no host synchronisation).
+ * The fast path needs logits / masked_out / noise 16-byte aligned with
+ * ld * sizeof(element) a multiple of 16; other layouts take a slower kernel.
+ */
+int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t *row_table,
+              const void *logits, int32_t dtype, int64_t ld, const float *noise,
+              int32_t *states, int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
+              int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
+
+/*
+ * Rows since the last call whose input state or table index was out of range
+ * (not counting -1), and active rows that had no selectable token.
+ * Synchronises cuda_stream, then resets both counters.  Either pointer may be NULL.
+ */
+int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t *bad_state_rows,
+                     int64_t *empty_mask_rows);
+
+/* Message for the calling thread's most recent error ("" if none). */
+const char *cstr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSTR_H */

@@ -1,0 +1,509 @@
+// libcstr host side: handles, validation, uploads, table download, errors.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "cstr_internal.cuh"
+
+static thread_local char g_err[512] = "";
+
+int cstr_fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+extern "C" const char *cstr_last_error(void) { return g_err; }
+
+static int check_device(int handle_device, const char *what)
+{
+    int cur = -1;
+    CSTR_CUDA_TRY(cudaGetDevice(&cur));
+    if (cur != handle_device)
+        return cstr_fail(CSTR_ERR_DEVICE, "%s was created on device %d but device %d is current",
+                         what, handle_device, cur);
+    return CSTR_OK;
+}
+
+// ------------------------------------------------------------------ DFA
+
+extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
+{
+    if (!dfa)
+        return;
+    cudaFree(dfa->trans);
+    cudaFree(dfa->accept);
+    delete dfa;
+}
+
+extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
+                             int32_t start_state, cstr_dfa_t **out)
+{
+    if (!trans || !accept || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_dfa: null pointer");
+    *out = nullptr;
+    if (n_states < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: n_states = %d, need >= 1", n_states);
+    if (start_state < 0 || start_state >= n_states)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: start_state %d outside [0, %d)",
+                         start_state, n_states);
+    const int64_t n = (int64_t)n_states * 256;
+    for (int64_t i = 0; i < n; ++i) {
+        if (trans[i] < -1 || trans[i] >= n_states)
+            return cstr_fail(CSTR_ERR_DFA,
+                             "cstr_load_dfa: state %lld byte %lld has target %d outside [-1, %d)",
+                             (long long)(i / 256), (long long)(i % 256), trans[i], n_states);
+    }
+    cstr_dfa *d = new (std::nothrow) cstr_dfa();
+    if (!d)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+    memset(d, 0, sizeof *d);
+    int rc = CSTR_OK;
+    cudaError_t e = cudaGetDevice(&d->device);
+    d->n_states = n_states;
+    d->start = start_state;
+    d->wide = n_states > 32767;
+    const size_t esz = d->wide ? 4 : 2;
+    std::vector<uint8_t> flags;
+    std::vector<int16_t> narrow;
+    if (e == cudaSuccess)
+        e = cudaMalloc(&d->trans, (size_t)n * esz);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&d->accept, (size_t)n_states);
+    if (e == cudaSuccess) {
+        try {
+            flags.resize(n_states);
+            for (int32_t q = 0; q < n_states; ++q)
+                flags[q] = accept[q] ? 1 : 0;
+            if (!d->wide) {
+                narrow.resize((size_t)n);
+                for (int64_t i = 0; i < n; ++i)
+                    narrow[(size_t)i] = (int16_t)trans[i];
+            }
+        } catch (const std::bad_alloc &) {
+            cstr_free_dfa(d);
+            return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+        }
+        e = cudaMemcpy(d->trans, d->wide ? (const void *)trans : (const void *)narrow.data(),
+                       (size_t)n * esz, cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpy(d->accept, flags.data(), (size_t)n_states, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                       "cstr_load_dfa: %s", cudaGetErrorString(e));
+        cstr_free_dfa(d);
+        return rc;
+    }
+    *out = d;
+    return CSTR_OK;
+}
+
+// ---------------------------------------------------------------- vocab
+
+extern "C" void cstr_free_vocab(cstr_vocab_t *v)
+{
+    if (!v)
+        return;
+    cudaFree(v->bytes);
+    cudaFree(v->off);
+    cudaFree(v->head);
+    cudaFree(v->len);
+    delete v;
+}
+
+extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offsets,
+                               int32_t vocab_size, cstr_vocab_t **out)
+{
+    if (!offsets || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_vocab: null pointer");
+    *out = nullptr;
+    if (vocab_size < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_vocab: vocab_size = %d, need >= 1", vocab_size);
+    if (offsets[0] != 0)
+        return cstr_fail(CSTR_ERR_VOCAB, "cstr_load_vocab: offsets[0] = %lld, need 0",
+                         (long long)offsets[0]);
+    for (int32_t v = 0; v < vocab_size; ++v) {
+        if (offsets[v + 1] < offsets[v])
+            return cstr_fail(CSTR_ERR_VOCAB, "cstr_load_vocab: offsets decrease at token %d", v);
+    }
+    const int64_t total = offsets[vocab_size];
+    if (total >= ((int64_t)1 << 31))
+        return cstr_fail(CSTR_ERR_VOCAB, "cstr_load_vocab: %lld vocabulary bytes, need < 2^31",
+                         (long long)total);
+    if (total > 0 && !vocab_bytes)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_vocab: null vocab_bytes");
+
+    cstr_vocab *vh = new (std::nothrow) cstr_vocab();
+    if (!vh)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_vocab: out of host memory");
+    memset(vh, 0, sizeof *vh);
+    vh->V = vocab_size;
+    vh->total_bytes = total;
+
+    std::vector<uint32_t> off32, len32;
+    std::vector<uint4> head;
+    try {
+        off32.resize((size_t)vocab_size + 1);
+        len32.resize((size_t)vocab_size);
+        head.resize((size_t)vocab_size);
+    } catch (const std::bad_alloc &) {
+        delete vh;
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_vocab: out of host memory");
+    }
+    uint32_t max_len = 0;
+    for (int32_t v = 0; v <= vocab_size; ++v)
+        off32[v] = (uint32_t)offsets[v];
+    for (int32_t v = 0; v < vocab_size; ++v) {
+        const uint32_t n = off32[v + 1] - off32[v];
+        len32[v] = n;
+        if (n > max_len)
+            max_len = n;
+        uint8_t rec[16] = {0};
+        memcpy(rec, vocab_bytes + off32[v], n < 16 ? n : 16);
+        memcpy(&head[v], rec, 16);
+    }
+    vh->max_len = max_len;
+
+    cudaError_t e = cudaGetDevice(&vh->device);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->bytes, (size_t)total + 16);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->off, ((size_t)vocab_size + 1) * sizeof(uint32_t));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->head, (size_t)vocab_size * sizeof(uint4));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->len, (size_t)vocab_size * sizeof(uint32_t));
+    if (e == cudaSuccess)
+        e = cudaMemset(vh->bytes, 0, (size_t)total + 16);
+    if (e == cudaSuccess && total > 0)
+        e = cudaMemcpy(vh->bytes, vocab_bytes, (size_t)total, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(vh->off, off32.data(), off32.size() * sizeof(uint32_t),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(vh->head, head.data(), head.size() * sizeof(uint4), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(vh->len, len32.data(), len32.size() * sizeof(uint32_t),
+                       cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                           "cstr_load_vocab: %s", cudaGetErrorString(e));
+        cstr_free_vocab(vh);
+        return rc;
+    }
+    *out = vh;
+    return CSTR_OK;
+}
+
+// ---------------------------------------------------------------- table
+
+extern "C" void cstr_free_table(cstr_table_t *t)
+{
+    if (!t)
+        return;
+    cudaFree(t->next);
+    cudaFree(t->mask);
+    cudaFree(t->accept);
+    cstr_free_vocab(t->owned_vocab);
+    delete t;
+}
+
+extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
+                                 cstr_table_t **out)
+{
+    if (!vocab || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_table_create: null pointer");
+    *out = nullptr;
+    if (max_states < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_table_create: max_states = %d, need >= 1", max_states);
+    int rc = check_device(vocab->device, "vocabulary");
+    if (rc)
+        return rc;
+    cstr_table *t = new (std::nothrow) cstr_table();
+    if (!t)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_table_create: out of host memory");
+    memset(t, 0, sizeof *t);
+    t->device = vocab->device;
+    t->vocab = vocab;
+    t->max_states = max_states;
+    t->V = vocab->V;
+    t->W = (vocab->V + 31) / 32;
+    t->ldn = ((int64_t)t->V + 63) / 64 * 64;
+    t->ldw = ((int64_t)t->W + 31) / 32 * 32;
+    t->wide = max_states > 32767;
+    t->eos_id = -1;
+    const size_t next_bytes = (size_t)max_states * (size_t)t->ldn * (t->wide ? 4 : 2);
+    const size_t mask_bytes = (size_t)max_states * (size_t)t->ldw * 4;
+    cudaError_t e = cudaMalloc(&t->next, next_bytes);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->mask, mask_bytes);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->accept, (size_t)max_states);
+    if (e == cudaSuccess)
+        e = cudaMemset(t->mask, 0, mask_bytes);   // padding words stay zero for good
+    if (e == cudaSuccess)
+        e = cudaMemset(t->accept, 0, (size_t)max_states);
+    if (e != cudaSuccess) {
+        rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                       "cstr_table_create (%zu + %zu bytes): %s", next_bytes, mask_bytes,
+                       cudaGetErrorString(e));
+        cstr_free_table(t);
+        return rc;
+    }
+    *out = t;
+    return CSTR_OK;
+}
+
+extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                                void *cuda_stream)
+{
+    if (!table || !dfa)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_table_build: null pointer");
+    int rc = check_device(table->device, "table");
+    if (rc)
+        return rc;
+    if (dfa->device != table->device)
+        return cstr_fail(CSTR_ERR_DEVICE, "cstr_table_build: DFA and table on different devices");
+    if (dfa->n_states > table->max_states)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA has %d states, table holds %d",
+                         dfa->n_states, table->max_states);
+    if (eos_id < -1 || eos_id >= table->V)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_table_build: eos_id %d outside [-1, %d)", eos_id,
+                         table->V);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    table->n_states = dfa->n_states;
+    table->start = dfa->start;
+    table->eos_id = eos_id;
+    CSTR_CUDA_TRY(cudaMemcpyAsync(table->accept, dfa->accept, (size_t)dfa->n_states,
+                                  cudaMemcpyDeviceToDevice, stream));
+    return cstr_launch_build(table, dfa, stream);
+}
+
+extern "C" int cstr_build_token_table(const cstr_dfa_t *dfa, const uint8_t *vocab_bytes,
+                                      const int64_t *offsets, int32_t vocab_size, int32_t eos_id,
+                                      void *cuda_stream, cstr_table_t **out)
+{
+    if (!dfa || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_build_token_table: null pointer");
+    *out = nullptr;
+    cstr_vocab *vocab = nullptr;
+    int rc = cstr_load_vocab(vocab_bytes, offsets, vocab_size, &vocab);
+    if (rc)
+        return rc;
+    cstr_table *t = nullptr;
+    rc = cstr_table_create(vocab, dfa->n_states, &t);
+    if (rc) {
+        cstr_free_vocab(vocab);
+        return rc;
+    }
+    t->owned_vocab = vocab;
+    rc = cstr_table_build(t, dfa, eos_id, cuda_stream);
+    if (rc) {
+        cstr_free_table(t);
+        return rc;
+    }
+    *out = t;
+    return CSTR_OK;
+}
+
+extern "C" int cstr_table_info(const cstr_table_t *t, int32_t *n_states, int32_t *vocab_size,
+                               int32_t *mask_words, int32_t *start_state)
+{
+    if (!t)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_table_info: null table");
+    if (n_states)
+        *n_states = t->n_states;
+    if (vocab_size)
+        *vocab_size = t->V;
+    if (mask_words)
+        *mask_words = t->W;
+    if (start_state)
+        *start_state = t->start;
+    return CSTR_OK;
+}
+
+extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int32_t state_hi,
+                                   uint32_t *mask_host, int32_t *next_host, void *cuda_stream)
+{
+    if (!t)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_table_download: null table");
+    int rc = check_device(t->device, "table");
+    if (rc)
+        return rc;
+    if (state_lo < 0 || state_hi < state_lo || state_hi > t->n_states)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_table_download: states [%d, %d) outside [0, %d)",
+                         state_lo, state_hi, t->n_states);
+    CSTR_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    const int32_t rows = state_hi - state_lo;
+    if (rows == 0)
+        return CSTR_OK;
+    if (mask_host) {
+        CSTR_CUDA_TRY(cudaMemcpy2D(mask_host, (size_t)t->W * 4, t->mask + (int64_t)state_lo * t->ldw,
+                                   (size_t)t->ldw * 4, (size_t)t->W * 4, rows,
+                                   cudaMemcpyDeviceToHost));
+    }
+    if (next_host) {
+        if (t->wide) {
+            CSTR_CUDA_TRY(cudaMemcpy2D(next_host, (size_t)t->V * 4,
+                                       (const int32_t *)t->next + (int64_t)state_lo * t->ldn,
+                                       (size_t)t->ldn * 4, (size_t)t->V * 4, rows,
+                                       cudaMemcpyDeviceToHost));
+        } else {
+            // narrow rows come down in slabs and are widened on the host
+            const int32_t slab = 64;
+            std::vector<int16_t> tmp;
+            try {
+                tmp.resize((size_t)slab * (size_t)t->V);
+            } catch (const std::bad_alloc &) {
+                return cstr_fail(CSTR_ERR_NOMEM, "cstr_table_download: out of host memory");
+            }
+            for (int32_t r0 = 0; r0 < rows; r0 += slab) {
+                const int32_t nr = rows - r0 < slab ? rows - r0 : slab;
+                CSTR_CUDA_TRY(cudaMemcpy2D(tmp.data(), (size_t)t->V * 2,
+                                           (const int16_t *)t->next +
+                                               (int64_t)(state_lo + r0) * t->ldn,
+                                           (size_t)t->ldn * 2, (size_t)t->V * 2, nr,
+                                           cudaMemcpyDeviceToHost));
+                int32_t *dst = next_host + (int64_t)r0 * t->V;
+                const int64_t n = (int64_t)nr * t->V;
+                for (int64_t i = 0; i < n; ++i)
+                    dst[i] = (int32_t)tmp[(size_t)i];
+            }
+        }
+    }
+    return CSTR_OK;
+}
+
+// ------------------------------------------------------------ workspace
+
+extern "C" void cstr_free_workspace(cstr_workspace_t *ws)
+{
+    if (!ws)
+        return;
+    cudaFree(ws->cell);
+    cudaFree(ws->ticket);
+    cudaFree(ws->counters);
+    delete ws;
+}
+
+extern "C" int cstr_workspace_create(int32_t max_batch, cstr_workspace_t **out)
+{
+    if (!out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_workspace_create: null pointer");
+    *out = nullptr;
+    if (max_batch < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_workspace_create: max_batch = %d, need >= 1",
+                         max_batch);
+    cstr_workspace *ws = new (std::nothrow) cstr_workspace();
+    if (!ws)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_workspace_create: out of host memory");
+    memset(ws, 0, sizeof *ws);
+    ws->max_batch = max_batch;
+    cudaError_t e = cudaGetDevice(&ws->device);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->cell, (size_t)max_batch * 8);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->ticket, (size_t)max_batch * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->counters, 16);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->cell, 0, (size_t)max_batch * 8);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->ticket, 0, (size_t)max_batch * 4);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->counters, 0, 16);
+    if (e != cudaSuccess) {
+        int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                           "cstr_workspace_create: %s", cudaGetErrorString(e));
+        cstr_free_workspace(ws);
+        return rc;
+    }
+    *out = ws;
+    return CSTR_OK;
+}
+
+// ----------------------------------------------------------------- step
+
+extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
+                         const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
+                         const float *noise, int32_t *states, int32_t *tokens_out,
+                         void *masked_out, uint8_t *accept_out, int32_t batch,
+                         cstr_workspace_t *ws, void *cuda_stream)
+{
+    if (!tables || !logits || !states || !tokens_out || !masked_out || !ws)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_step: null pointer");
+    if (n_tables < 1 || n_tables > CSTR_MAX_TABLES)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_step: n_tables = %d, need 1..%d", n_tables,
+                         CSTR_MAX_TABLES);
+    if (dtype != CSTR_F32 && dtype != CSTR_BF16)
+        return cstr_fail(CSTR_ERR_DTYPE, "cstr_step: unknown dtype %d", dtype);
+    if (batch < 0)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_step: batch = %d", batch);
+    if (batch > ws->max_batch)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_step: batch %d exceeds workspace capacity %d",
+                         batch, ws->max_batch);
+    int rc = check_device(ws->device, "workspace");
+    if (rc)
+        return rc;
+    cstr_step_args a;
+    memset(&a, 0, sizeof a);
+    for (int32_t i = 0; i < n_tables; ++i) {
+        const cstr_table *t = tables[i];
+        if (!t)
+            return cstr_fail(CSTR_ERR_NULL, "cstr_step: tables[%d] is null", i);
+        if (t->device != ws->device)
+            return cstr_fail(CSTR_ERR_DEVICE, "cstr_step: tables[%d] is on another device", i);
+        if (t->n_states < 1)
+            return cstr_fail(CSTR_ERR_ARG, "cstr_step: tables[%d] has not been built", i);
+        if (t->V != tables[0]->V)
+            return cstr_fail(CSTR_ERR_SHAPE, "cstr_step: tables[%d] has V = %d, tables[0] has %d",
+                             i, t->V, tables[0]->V);
+        a.tables[i] = t;
+    }
+    if (ld < tables[0]->V)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_step: ld = %lld is below V = %d", (long long)ld,
+                         tables[0]->V);
+    if (batch == 0)
+        return CSTR_OK;
+    a.n_tables = n_tables;
+    a.row_table = row_table;
+    a.logits = logits;
+    a.dtype = dtype;
+    a.ld = ld;
+    a.noise = noise;
+    a.states = states;
+    a.tokens_out = tokens_out;
+    a.masked_out = masked_out;
+    a.accept_out = accept_out;
+    a.batch = batch;
+    a.ws = ws;
+    return cstr_launch_step(a, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t *bad_state_rows,
+                                int64_t *empty_mask_rows)
+{
+    if (!ws)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_step_status: null workspace");
+    int rc = check_device(ws->device, "workspace");
+    if (rc)
+        return rc;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long host[2] = {0, 0};
+    CSTR_CUDA_TRY(cudaMemcpyAsync(host, ws->counters, 16, cudaMemcpyDeviceToHost, stream));
+    CSTR_CUDA_TRY(cudaMemsetAsync(ws->counters, 0, 16, stream));
+    CSTR_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (bad_state_rows)
+        *bad_state_rows = (int64_t)host[0];
+    if (empty_mask_rows)
+        *empty_mask_rows = (int64_t)host[1];
+    return CSTR_OK;
+}

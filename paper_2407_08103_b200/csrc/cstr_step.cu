@@ -1,0 +1,437 @@
+// Fused constrained decoding step (Algorithm 2, loop body) for a batch of rows:
+// mask from the row's state, -inf on disallowed logits, arg-max selection with
+// lowest-index tie-break (optionally over logit + supplied noise), next-state
+// update - one streaming pass over the logits, one kernel.
+//
+// A row is split into chunks of whole tiles; one CTA streams one chunk with
+// 128-bit loads/stores, applying the state's bitmask a 32-token word at a time
+// (one coalesced word load per lane per tile, words handed around with
+// shuffles).  Each CTA folds its (value, index) winner into a per-row 64-bit
+// cell with atomicMax on an order-preserving key - a total order, so the
+// result does not depend on arrival order - and the CTA that arrives last at
+// the row's ticket reads the cell, emits token / state / accept flag and
+// resets the scratch.  Nobody waits on anybody.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "cstr_internal.cuh"
+
+namespace {
+
+struct TableDesc {
+    const uint32_t *mask;
+    const void *next;
+    const uint8_t *accept;
+    long long ldn;
+    long long ldw;
+    int n_states;
+    int wide;
+};
+
+struct StepParams {
+    TableDesc tab[CSTR_MAX_TABLES];
+    const int32_t *row_table;
+    const void *logits;
+    const float *noise;
+    void *out;
+    int32_t *states;
+    int32_t *tokens;
+    uint8_t *accept_out;
+    unsigned long long *cell;
+    unsigned int *ticket;
+    unsigned long long *counters;
+    long long ld;
+    int V;
+    int n_tables;
+    int nchunks;         // CTAs per row
+    int tiles_per_cta;
+};
+
+constexpr int kUnroll = 8;          // 16-byte vectors in flight per lane per tile
+constexpr unsigned kFull = 0xffffffffu;
+
+struct Best {
+    float v;
+    int i;   // -1: nothing selected yet
+};
+
+// Scan-order update: indices arrive in increasing order within a thread, so a
+// later candidate wins only if strictly larger (or if nothing is held yet).
+// `cand` is NaN for disallowed positions, so they never win.
+__device__ __forceinline__ void consider(Best &b, float cand, int idx)
+{
+    const bool take = (cand > b.v) || (b.i < 0 && cand == cand);
+    b.v = take ? cand : b.v;
+    b.i = take ? idx : b.i;
+}
+
+// Order-free merge of two partial winners.
+__device__ __forceinline__ void merge(Best &b, float ov, int oi)
+{
+    const bool take = oi >= 0 && (b.i < 0 || ov > b.v || (ov == b.v && oi < b.i));
+    b.v = take ? ov : b.v;
+    b.i = take ? oi : b.i;
+}
+
+// Monotone map float -> uint32 (after folding -0 into +0), then (key, ~index).
+__device__ __forceinline__ unsigned long long pack_key(float v, int idx)
+{
+    v = v + 0.0f;                                   // -0.0 + 0.0 = +0.0 (round to nearest)
+    const unsigned u = __float_as_uint(v);
+    const unsigned hi = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)hi << 32) | (unsigned long long)(0xffffffffu - (unsigned)idx);
+}
+
+struct RowCtx {
+    int r, chunk, t, q;
+    bool active;
+    const uint32_t *mrow;
+};
+
+__device__ __forceinline__ RowCtx row_context(const StepParams &p)
+{
+    RowCtx c;
+    c.r = blockIdx.x / p.nchunks;
+    c.chunk = blockIdx.x - c.r * p.nchunks;
+    c.t = p.row_table ? p.row_table[c.r] : 0;
+    c.q = p.states[c.r];
+    const bool table_ok = c.t >= 0 && c.t < p.n_tables;
+    const int tt = table_ok ? c.t : 0;
+    c.active = table_ok && c.q >= 0 && c.q < p.tab[tt].n_states;
+    c.t = tt;
+    c.mrow = c.active ? p.tab[tt].mask + (long long)c.q * p.tab[tt].ldw : nullptr;
+    return c;
+}
+
+// CTA-level reduction, cross-CTA fold, and the last arriver's finalisation.
+__device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c, Best b)
+{
+    __shared__ float s_v[32];
+    __shared__ int s_i[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_down_sync(kFull, b.v, off);
+        const int oi = __shfl_down_sync(kFull, b.i, off);
+        merge(b, ov, oi);
+    }
+    if (lane == 0) {
+        s_v[warp] = b.v;
+        s_i[warp] = b.i;
+    }
+    __syncthreads();
+    if (threadIdx.x != 0)
+        return;
+    const int nwarps = (blockDim.x + 31) >> 5;
+    for (int w = 1; w < nwarps; ++w)
+        merge(b, s_v[w], s_i[w]);
+    if (b.i >= 0)
+        atomicMax(p.cell + c.r, pack_key(b.v, b.i));
+    __threadfence();
+    const unsigned prev = atomicAdd(p.ticket + c.r, 1u);
+    if (prev != (unsigned)p.nchunks - 1u)
+        return;
+    __threadfence();
+    const unsigned long long key = atomicExch(p.cell + c.r, 0ull);
+    p.ticket[c.r] = 0u;
+    int tok = -1, q2 = CSTR_DEAD;
+    const TableDesc &tb = p.tab[c.t];
+    if (c.active && key != 0ull) {
+        tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
+        const long long at = (long long)c.q * tb.ldn + tok;
+        q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const int16_t *)tb.next)[at];
+    } else if (c.active) {
+        atomicAdd(p.counters + 1, 1ull);
+    } else if (c.q != -1) {
+        atomicAdd(p.counters + 0, 1ull);
+    }
+    p.tokens[c.r] = tok;
+    p.states[c.r] = q2;
+    if (p.accept_out)
+        p.accept_out[c.r] = (q2 >= 0) ? (uint8_t)(tb.accept[q2] != 0) : (uint8_t)0;
+}
+
+// ---- per-vector processing ------------------------------------------------
+
+// fp32: 4 logits per 16-byte vector, 4 mask bits.
+__device__ __forceinline__ float4 apply_f32(float4 x, const float4 *nz, unsigned bits, int idx,
+                                            Best &b)
+{
+    const float ninf = -CUDART_INF_F, qnan = CUDART_NAN_F;
+    float in[4] = {x.x, x.y, x.z, x.w};
+    float out[4];
+    float add[4] = {0.f, 0.f, 0.f, 0.f};
+    if (nz) {
+        add[0] = nz->x; add[1] = nz->y; add[2] = nz->z; add[3] = nz->w;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const bool ok = (bits >> e) & 1u;
+        out[e] = ok ? in[e] : ninf;
+        const float s = nz ? in[e] + add[e] : in[e];
+        consider(b, ok ? s : qnan, idx + e);
+    }
+    return make_float4(out[0], out[1], out[2], out[3]);
+}
+
+// bf16: 8 logits per 16-byte vector, 8 mask bits; noise comes as two float4.
+__device__ __forceinline__ uint4 apply_bf16(uint4 x, const float4 *nz, unsigned bits, int idx,
+                                            Best &b)
+{
+    const float qnan = CUDART_NAN_F;
+    unsigned in[4] = {x.x, x.y, x.z, x.w};
+    unsigned out[4];
+    float add[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (nz) {
+        add[0] = nz[0].x; add[1] = nz[0].y; add[2] = nz[0].z; add[3] = nz[0].w;
+        add[4] = nz[1].x; add[5] = nz[1].y; add[6] = nz[1].z; add[7] = nz[1].w;
+    }
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const bool ok0 = (bits >> (2 * h)) & 1u, ok1 = (bits >> (2 * h + 1)) & 1u;
+        const unsigned lo = in[h] & 0xffffu, hi = in[h] & 0xffff0000u;
+        out[h] = (ok0 ? lo : 0xff80u) | (ok1 ? hi : 0xff800000u);
+        float f0 = __uint_as_float(lo << 16), f1 = __uint_as_float(hi);   // exact widening
+        if (nz) {
+            f0 = f0 + add[2 * h];
+            f1 = f1 + add[2 * h + 1];
+        }
+        consider(b, ok0 ? f0 : qnan, idx + 2 * h);
+        consider(b, ok1 ? f1 : qnan, idx + 2 * h + 1);
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+// Scalar element, shared by the vector kernel's ragged tail and the scalar kernel.
+template <bool BF16>
+__device__ __forceinline__ void apply_one(const StepParams &p, const RowCtx &c, long long row_off,
+                                          int i, Best &b)
+{
+    bool ok = false;
+    if (c.active)
+        ok = (c.mrow[i >> 5] >> (i & 31)) & 1u;
+    if (BF16) {
+        const unsigned short *in = (const unsigned short *)p.logits + row_off;
+        unsigned short *out = (unsigned short *)p.out + row_off;
+        const unsigned short raw = in[i];
+        float f = __uint_as_float((unsigned)raw << 16);
+        if (p.noise && ok)
+            f = f + p.noise[row_off + i];
+        out[i] = ok ? raw : (unsigned short)0xff80u;
+        consider(b, ok ? f : CUDART_NAN_F, i);
+    } else {
+        const float *in = (const float *)p.logits + row_off;
+        float *out = (float *)p.out + row_off;
+        const float raw = in[i];
+        float f = raw;
+        if (p.noise && ok)
+            f = f + p.noise[row_off + i];
+        out[i] = ok ? raw : -CUDART_INF_F;
+        consider(b, ok ? f : CUDART_NAN_F, i);
+    }
+}
+
+// ---- vector kernel ----------------------------------------------------------
+
+template <bool BF16, bool NOISE>
+__global__ void __launch_bounds__(256)
+step_vec_kernel(const __grid_constant__ StepParams p)
+{
+    constexpr int VEC = BF16 ? 8 : 4;               // logits per 16-byte vector
+    constexpr int TILE = 32 * VEC * kUnroll;        // tokens per warp tile
+    constexpr int WORDS = TILE / 32;                // mask words per tile (32 or 64)
+    constexpr int WPL = WORDS / 32;                 // mask words per lane per tile
+    constexpr int LANES_PER_WORD = 32 / VEC;
+
+    const RowCtx c = row_context(p);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const long long row_off = (long long)c.r * p.ld;
+    const uint4 *in = (const uint4 *)((const char *)p.logits + row_off * (BF16 ? 2 : 4));
+    uint4 *out = (uint4 *)((char *)p.out + row_off * (BF16 ? 2 : 4));
+    const float4 *nzrow = NOISE ? (const float4 *)(p.noise + row_off) : nullptr;
+    const int total_tiles = (p.V + TILE - 1) / TILE;
+    const int tile_end = min(total_tiles, (c.chunk + 1) * p.tiles_per_cta);
+    const int Vv = p.V - p.V % VEC;                 // tokens covered by whole vectors
+
+    Best b = {-CUDART_INF_F, -1};
+
+    for (int tile = c.chunk * p.tiles_per_cta + warp; tile < tile_end; tile += nwarps) {
+        const int tok0 = tile * TILE;
+        if (!c.active) {                            // finished / invalid row: all -inf
+            const uint4 fill = BF16 ? make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u)
+                                    : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                const int tok = tok0 + (j * 32 + lane) * VEC;
+                if (tok < Vv)
+                    __stcs(out + tok / VEC, fill);
+            }
+            continue;
+        }
+        uint32_t mw[WPL];
+#pragma unroll
+        for (int i = 0; i < WPL; ++i) {
+            const long long widx = (long long)tile * WORDS + i * 32 + lane;
+            mw[i] = (widx < p.tab[c.t].ldw) ? __ldg(c.mrow + widx) : 0u;
+        }
+        uint4 x[kUnroll];
+        float4 nz[NOISE ? kUnroll * (BF16 ? 2 : 1) : 1];
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            const int tok = tok0 + (j * 32 + lane) * VEC;
+            x[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (tok < Vv)
+                x[j] = __ldcs(in + tok / VEC);
+        }
+        if (NOISE) {
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                const int tok = tok0 + (j * 32 + lane) * VEC;
+                if (BF16) {
+                    nz[2 * j] = nz[2 * j + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (tok < Vv) {
+                        nz[2 * j] = __ldcs(nzrow + tok / 4);
+                        nz[2 * j + 1] = __ldcs(nzrow + tok / 4 + 1);
+                    }
+                } else {
+                    nz[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (tok < Vv)
+                        nz[j] = __ldcs(nzrow + tok / 4);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            const int tok = tok0 + (j * 32 + lane) * VEC;
+            const int word_in_tile = j * VEC + lane / LANES_PER_WORD;
+            const uint32_t word = __shfl_sync(kFull, mw[word_in_tile / 32], word_in_tile % 32);
+            const unsigned bits = (word >> ((lane % LANES_PER_WORD) * VEC)) & ((1u << VEC) - 1u);
+            if (tok < Vv) {
+                if (BF16) {
+                    const uint4 o = apply_bf16(x[j], NOISE ? &nz[2 * j] : nullptr, bits, tok, b);
+                    __stcs(out + tok / VEC, o);
+                } else {
+                    const float4 xf = make_float4(__uint_as_float(x[j].x), __uint_as_float(x[j].y),
+                                                  __uint_as_float(x[j].z), __uint_as_float(x[j].w));
+                    const float4 o = apply_f32(xf, NOISE ? &nz[j] : nullptr, bits, tok, b);
+                    __stcs(out + tok / VEC,
+                           make_uint4(__float_as_uint(o.x), __float_as_uint(o.y),
+                                      __float_as_uint(o.z), __float_as_uint(o.w)));
+                }
+            }
+        }
+    }
+    // ragged tail (V not a multiple of the vector width): highest indices of the row
+    if (c.chunk == p.nchunks - 1 && warp == 0 && Vv + lane < p.V)
+        apply_one<BF16>(p, c, row_off, Vv + lane, b);
+
+    finish_row(p, c, b);
+}
+
+// ---- scalar kernel: any alignment / stride ----------------------------------
+
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+step_scalar_kernel(const __grid_constant__ StepParams p)
+{
+    constexpr int VEC = BF16 ? 8 : 4;
+    constexpr int TILE = 32 * VEC * kUnroll;
+    const RowCtx c = row_context(p);
+    const long long row_off = (long long)c.r * p.ld;
+    const long long begin = (long long)c.chunk * p.tiles_per_cta * TILE;
+    const int end = (int)min((long long)p.V, begin + (long long)p.tiles_per_cta * TILE);
+    Best b = {-CUDART_INF_F, -1};
+    for (int i = (int)begin + threadIdx.x; i < end; i += blockDim.x)
+        apply_one<BF16>(p, c, row_off, i, b);
+    finish_row(p, c, b);
+}
+
+int g_sm_count[64] = {0};
+
+int sm_count(int device)
+{
+    if (device < 0 || device >= 64)
+        return 148;
+    if (g_sm_count[device] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n < 1)
+            n = 148;
+        g_sm_count[device] = n;
+    }
+    return g_sm_count[device];
+}
+
+}  // namespace
+
+int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
+{
+    StepParams p;
+    for (int i = 0; i < CSTR_MAX_TABLES; ++i) {
+        const cstr_table *t = a.tables[i < a.n_tables ? i : 0];
+        p.tab[i].mask = t->mask;
+        p.tab[i].next = t->next;
+        p.tab[i].accept = t->accept;
+        p.tab[i].ldn = t->ldn;
+        p.tab[i].ldw = t->ldw;
+        p.tab[i].n_states = t->n_states;
+        p.tab[i].wide = t->wide;
+    }
+    const cstr_table *t0 = a.tables[0];
+    p.row_table = a.row_table;
+    p.logits = a.logits;
+    p.noise = a.noise;
+    p.out = a.masked_out;
+    p.states = a.states;
+    p.tokens = a.tokens_out;
+    p.accept_out = a.accept_out;
+    p.cell = a.ws->cell;
+    p.ticket = a.ws->ticket;
+    p.counters = a.ws->counters;
+    p.ld = a.ld;
+    p.V = t0->V;
+    p.n_tables = a.n_tables;
+
+    const bool bf16 = a.dtype == CSTR_BF16;
+    const int esz = bf16 ? 2 : 4;
+    const int tile = 32 * (bf16 ? 8 : 4) * kUnroll;
+    const int total_tiles = (p.V + tile - 1) / tile;
+    // 8 tiles (one per warp) per CTA when there is enough work to fill the
+    // machine a few times over, fewer for small batches.
+    const long long want_ctas = 4LL * sm_count(a.ws->device);
+    int tiles_per_cta = 8;
+    while (tiles_per_cta > 1 &&
+           (long long)a.batch * ((total_tiles + tiles_per_cta - 1) / tiles_per_cta) < want_ctas)
+        tiles_per_cta >>= 1;
+    p.tiles_per_cta = tiles_per_cta;
+    p.nchunks = (total_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    const long long ctas = (long long)a.batch * p.nchunks;
+    if (ctas > 0x7fffffffLL)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_step: batch x vocabulary too large for one launch");
+    const int threads = 32 * (tiles_per_cta < 8 ? tiles_per_cta : 8);
+
+    auto aligned16 = [](const void *ptr) { return ((uintptr_t)ptr & 15u) == 0; };
+    const bool vec_ok = aligned16(a.logits) && aligned16(a.masked_out) &&
+                        (a.ld * esz) % 16 == 0 &&
+                        (!a.noise || (aligned16(a.noise) && (a.ld * 4) % 16 == 0));
+    const unsigned grid = (unsigned)ctas;
+    if (vec_ok) {
+        if (bf16) {
+            if (a.noise)
+                step_vec_kernel<true, true><<<grid, threads, 0, stream>>>(p);
+            else
+                step_vec_kernel<true, false><<<grid, threads, 0, stream>>>(p);
+        } else {
+            if (a.noise)
+                step_vec_kernel<false, true><<<grid, threads, 0, stream>>>(p);
+            else
+                step_vec_kernel<false, false><<<grid, threads, 0, stream>>>(p);
+        }
+    } else {
+        if (bf16)
+            step_scalar_kernel<true><<<grid, threads, 0, stream>>>(p);
+        else
+            step_scalar_kernel<false><<<grid, threads, 0, stream>>>(p);
+    }
+    CSTR_CUDA_TRY(cudaGetLastError());
+    return CSTR_OK;
+}

@@ -1,0 +1,225 @@
+"""Thin ctypes binding of libcstr (argument marshalling only).
+
+Functions carry the names of the C entry points in ``include/cstr.h``; device
+arrays are ``torch`` CUDA tensors (used here only as owners of device memory)
+and streams are ``torch.cuda`` streams.  There is no CPU path: importing works
+anywhere, but any call raises if ``libcstr.so`` cannot be loaded.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from .build import LIB_PATH
+
+CSTR_F32 = 0
+CSTR_BF16 = 1
+CSTR_MAX_TABLES = 16
+
+EXPORTS = [
+    "cstr_load_dfa", "cstr_free_dfa", "cstr_load_vocab", "cstr_free_vocab",
+    "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
+    "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
+    "cstr_step", "cstr_step_status", "cstr_last_error",
+]
+
+_lib = None
+
+
+class CstrError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__("libcstr error %d: %s" % (code, message))
+        self.code = code
+
+
+def lib():
+    """Load libcstr.so (built in-tree by ``build.build_library``); fail loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libcstr.so is missing at %s: build it with "
+                "`python -m paper_2407_08103_b200.build` (needs nvcc); there is no fallback path"
+                % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            fn.restype = ctypes.c_int
+        L.cstr_last_error.restype = ctypes.c_char_p
+        for name in ("cstr_free_dfa", "cstr_free_vocab", "cstr_free_table", "cstr_free_workspace"):
+            getattr(L, name).restype = None
+        _lib = L
+    return _lib
+
+
+def _check(rc):
+    if rc != 0:
+        raise CstrError(rc, lib().cstr_last_error().decode("utf-8", "replace"))
+
+
+def _np_ptr(a):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+def _dev_ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class _Handle:
+    _free = None
+
+    def __init__(self, ptr):
+        self.ptr = ptr
+
+    def close(self):
+        if self.ptr:
+            getattr(lib(), self._free)(self.ptr)
+            self.ptr = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Dfa(_Handle):
+    _free = "cstr_free_dfa"
+
+
+class Vocab(_Handle):
+    _free = "cstr_free_vocab"
+
+
+class Table(_Handle):
+    _free = "cstr_free_table"
+    vocab = None  # keeps the vocabulary handle alive
+
+
+class Workspace(_Handle):
+    _free = "cstr_free_workspace"
+
+
+def cstr_load_dfa(trans, accept, start_state=0) -> Dfa:
+    trans = np.ascontiguousarray(trans, dtype=np.int32)
+    accept = np.ascontiguousarray(accept, dtype=np.uint8)
+    if trans.ndim != 2 or trans.shape[1] != 256 or accept.shape != (trans.shape[0],):
+        raise ValueError("trans must be [S][256] and accept [S]")
+    out = ctypes.c_void_p()
+    _check(lib().cstr_load_dfa(_np_ptr(trans), _np_ptr(accept), ctypes.c_int32(trans.shape[0]),
+                               ctypes.c_int32(start_state), ctypes.byref(out)))
+    return Dfa(out)
+
+
+def cstr_load_vocab(vocab_bytes, offsets) -> Vocab:
+    vocab_bytes = np.ascontiguousarray(vocab_bytes, dtype=np.uint8)
+    offsets = np.ascontiguousarray(offsets, dtype=np.int64)
+    out = ctypes.c_void_p()
+    _check(lib().cstr_load_vocab(_np_ptr(vocab_bytes), _np_ptr(offsets),
+                                 ctypes.c_int32(offsets.size - 1), ctypes.byref(out)))
+    return Vocab(out)
+
+
+def cstr_table_create(vocab: Vocab, max_states: int) -> Table:
+    out = ctypes.c_void_p()
+    _check(lib().cstr_table_create(vocab.ptr, ctypes.c_int32(max_states), ctypes.byref(out)))
+    t = Table(out)
+    t.vocab = vocab
+    return t
+
+
+def cstr_table_build(table: Table, dfa: Dfa, eos_id: int = -1, stream=None) -> None:
+    _check(lib().cstr_table_build(table.ptr, dfa.ptr, ctypes.c_int32(eos_id), _stream_ptr(stream)))
+
+
+def cstr_build_token_table(dfa: Dfa, vocab_bytes, offsets, eos_id: int = -1, stream=None) -> Table:
+    vocab_bytes = np.ascontiguousarray(vocab_bytes, dtype=np.uint8)
+    offsets = np.ascontiguousarray(offsets, dtype=np.int64)
+    out = ctypes.c_void_p()
+    _check(lib().cstr_build_token_table(dfa.ptr, _np_ptr(vocab_bytes), _np_ptr(offsets),
+                                        ctypes.c_int32(offsets.size - 1), ctypes.c_int32(eos_id),
+                                        _stream_ptr(stream), ctypes.byref(out)))
+    return Table(out)
+
+
+def cstr_table_info(table: Table):
+    vals = [ctypes.c_int32() for _ in range(4)]
+    _check(lib().cstr_table_info(table.ptr, *[ctypes.byref(v) for v in vals]))
+    n_states, vocab_size, words, start = (int(v.value) for v in vals)
+    return dict(n_states=n_states, vocab_size=vocab_size, mask_words=words, start_state=start)
+
+
+def cstr_table_download(table: Table, state_lo: int = 0, state_hi: int | None = None,
+                        want_mask: bool = True, want_next: bool = True, stream=None):
+    info = cstr_table_info(table)
+    state_hi = info["n_states"] if state_hi is None else state_hi
+    rows = max(state_hi - state_lo, 0)
+    mask = np.empty((rows, info["mask_words"]), dtype=np.uint32) if want_mask else None
+    nxt = np.empty((rows, info["vocab_size"]), dtype=np.int32) if want_next else None
+    _check(lib().cstr_table_download(table.ptr, ctypes.c_int32(state_lo), ctypes.c_int32(state_hi),
+                                     _np_ptr(mask), _np_ptr(nxt), _stream_ptr(stream)))
+    return nxt, mask
+
+
+def cstr_workspace_create(max_batch: int) -> Workspace:
+    out = ctypes.c_void_p()
+    _check(lib().cstr_workspace_create(ctypes.c_int32(max_batch), ctypes.byref(out)))
+    return Workspace(out)
+
+
+def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noise=None,
+              row_table=None, accept_out=None, vocab_ld: int | None = None, stream=None) -> None:
+    """Enqueue one constrained decoding step.  All tensors are CUDA tensors:
+    ``logits``/``masked_out`` ``[B][ld]`` float32 or bfloat16, ``noise`` float32
+    ``[B][ld]`` or None, ``states``/``tokens_out``/``row_table`` int32 ``[B]``,
+    ``accept_out`` uint8 ``[B]`` or None."""
+    import torch
+    if isinstance(tables, Table):
+        tables = [tables]
+    if logits.dtype == torch.float32:
+        dtype = CSTR_F32
+    elif logits.dtype == torch.bfloat16:
+        dtype = CSTR_BF16
+    else:
+        raise TypeError("logits must be float32 or bfloat16")
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [B][ld] with unit inner stride")
+    ld = logits.stride(0) if vocab_ld is None else vocab_ld
+    batch = logits.shape[0]
+    for name, t in (("masked_out", masked_out), ("noise", noise)):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != ld or t.shape[0] != batch):
+            raise ValueError("%s must have the layout of logits" % name)
+    if masked_out.dtype != logits.dtype:
+        raise TypeError("masked_out must have the dtype of logits")
+    if noise is not None and noise.dtype != torch.float32:
+        raise TypeError("noise must be float32")
+    for name, t, dt in (("states", states, torch.int32), ("tokens_out", tokens_out, torch.int32),
+                        ("row_table", row_table, torch.int32), ("accept_out", accept_out, torch.uint8)):
+        if t is not None and (t.dtype != dt or t.numel() < batch or not t.is_contiguous()):
+            raise ValueError("%s must be a contiguous %s tensor with one entry per row" % (name, dt))
+    arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
+    _check(lib().cstr_step(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table), _dev_ptr(logits),
+                           ctypes.c_int32(dtype), ctypes.c_int64(ld), _dev_ptr(noise),
+                           _dev_ptr(states), _dev_ptr(tokens_out), _dev_ptr(masked_out),
+                           _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
+                           _stream_ptr(stream)))
+
+
+def cstr_step_status(ws: Workspace, stream=None):
+    bad, empty = ctypes.c_int64(), ctypes.c_int64()
+    _check(lib().cstr_step_status(ws.ptr, _stream_ptr(stream), ctypes.byref(bad), ctypes.byref(empty)))
+    return int(bad.value), int(empty.value)
+
+
+def cstr_last_error() -> str:
+    return lib().cstr_last_error().decode("utf-8", "replace")

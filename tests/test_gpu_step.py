@@ -1,0 +1,220 @@
+"""GPU parity: the fused constrained step vs the CPU oracle, bit exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2407_08103_b200 import cstr
+from paper_2407_08103_b200.decode import ConstrainedDecoder
+from synth import (f32_to_bf16_bits, gumbel_noise, normal_logits, random_range_dfa,
+                   vocab_from_strings)
+from synth.configs import CONFIGS, config_dfas, config_vocab, row_table_for
+from synth.regex_frontend import regex_to_dfa
+
+from gpu_common import DEV, bits_equal, from_dev_logits, gpu_tables, run_step_both, to_dev_logits
+from test_gpu_table import dense_random_dfa, random_vocab
+
+pytestmark = pytest.mark.gpu
+
+
+def rand_logits(rng, B, V, ld, dtype):
+    x = np.zeros((B, ld), dtype=np.float32)
+    x[:, :V] = rng.standard_normal((B, V)).astype(np.float32)
+    x[:, V:] = 50.0                         # padding larger than any logit: must be ignored
+    return x if dtype == "f32" else f32_to_bf16_bits(x)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_small(seed):
+    rng = np.random.default_rng(100 + seed)
+    S = int(rng.choice([1, 3, 40, 300]))
+    V = int(rng.choice([1, 7, 32, 33, 1000, 1024, 1027, 4096, 9001, 20000]))
+    B = int(rng.choice([1, 2, 5, 33]))
+    dtype = "bf16" if seed % 2 else "f32"
+    align = 8 if dtype == "bf16" else 4
+    ld = V if seed % 4 < 2 else (V + align - 1) // align * align + align   # unaligned and padded strides
+    dfa = dense_random_dfa(rng, S, live=float(rng.choice([0.05, 0.6, 1.0])))
+    vb, vo = random_vocab(rng, V, max_len=6)
+    tables = gpu_tables([dfa], vb, vo)
+    logits = rand_logits(rng, B, V, ld, dtype)
+    states = rng.integers(-1, S, size=B).astype(np.int32)
+    noise = None
+    if seed % 3 == 0:
+        noise = np.zeros((B, ld), dtype=np.float32)
+        noise[:, :V] = -np.log(-np.log(rng.random((B, V)))).astype(np.float32)
+    run_step_both([dfa], tables, vb, vo, logits, states, noise=noise, in_place=(seed % 5 == 0))
+
+
+def test_ties_signed_zero_nan_inf_across_chunks():
+    # Several chunks per row (V spans many tiles); the tie / NaN / inf rules
+    # must hold across CTA boundaries, not only inside one thread.
+    V, B = 70000, 8
+    dfa = (np.zeros((1, 256), dtype=np.int32), np.ones(1, dtype=np.uint8), 0)   # everything allowed
+    toks = [bytes([65 + i % 26]) for i in range(V)]
+    vb, vo = vocab_from_strings(toks)
+    tables = gpu_tables([dfa], vb, vo)
+    x = np.full((B, V), -3.0, dtype=np.float32)
+    x[0, [100, 40000, 69999]] = 2.5                  # equal maxima in three chunks: lowest id
+    x[1, 50000] = -0.0; x[1, 60000] = 0.0; x[1, :] = np.where(x[1] == -3.0, -1.0, x[1])   # -0 == +0: lowest id
+    x[2, 60000] = -0.0; x[2, 50000] = 0.0; x[2, :] = np.where(x[2] == -3.0, -1.0, x[2])
+    x[3, :] = np.nan; x[3, 65000] = -np.inf          # a -inf beats NaNs
+    x[4, :] = np.nan                                 # nothing selectable
+    x[5, 123] = np.inf; x[5, 69000] = np.inf
+    x[6, :] = -np.inf                                # all -inf: token 0
+    x[7, 33333] = np.float32(1e-45)                  # denormal vs negatives
+    ref = run_step_both([dfa], tables, vb, vo, x, np.zeros(B, dtype=np.int32))
+    assert ref["tokens"].tolist() == [100, 50000, 50000, 65000, -1, 123, 0, 33333]
+    # the same with noise whose sum creates ties and NaN (inf + -inf)
+    noise = np.zeros((B, V), dtype=np.float32)
+    noise[0, 100] = -1.0
+    noise[5, 123] = -np.inf
+    ref = run_step_both([dfa], tables, vb, vo, x, np.zeros(B, dtype=np.int32), noise=noise)
+    assert ref["tokens"][0] == 40000 and ref["tokens"][5] == 69000
+
+
+def test_inactive_bad_and_empty_rows():
+    dfa = regex_to_dfa("(a|b)*c")
+    toks = [b"a", b"b", b"c", b"ab", b"zz", b"bc", b"ca"] + [b"q%d" % i for i in range(3000)]
+    vb, vo = vocab_from_strings(toks)
+    tables = gpu_tables([dfa], vb, vo)
+    V = len(toks)
+    S = dfa[0].shape[0]
+    acc_state = int(np.nonzero(dfa[1])[0][0])
+    states = np.array([-1, S, -7, 2 ** 30, dfa[2], acc_state], dtype=np.int32)
+    rng = np.random.default_rng(0)
+    for dtype in ("f32", "bf16"):
+        logits = rand_logits(rng, 6, V, (V + 7) // 8 * 8, dtype)
+        ref = run_step_both([dfa], tables, vb, vo, logits, states)
+        assert ref["bad_state_rows"] == 3 and ref["empty_mask_rows"] == 1
+
+
+def test_eos_token():
+    dfa = regex_to_dfa("ab?")
+    toks = [b"a", b"b", b"<eos>", b"ab"]
+    vb, vo = vocab_from_strings(toks)
+    tables = gpu_tables([dfa], vb, vo, eos_id=2)
+    logits = np.array([[0.0, 0.0, 5.0, 1.0]] * 3, dtype=np.float32)
+    states = np.arange(3, dtype=np.int32) % dfa[0].shape[0]
+    run_step_both([dfa], tables, vb, vo, logits, states, eos_id=2)
+
+
+def test_mixed_tables_and_bad_table_index():
+    rng = np.random.default_rng(4)
+    V = 5000
+    vb, vo = random_vocab(rng, V, max_len=5)
+    dfas = [dense_random_dfa(rng, S) for S in (5, 70, 300)]
+    tables = gpu_tables(dfas, vb, vo)
+    B = 24
+    row_table = rng.integers(0, 3, size=B).astype(np.int32)
+    row_table[3] = 3        # out of range
+    row_table[9] = -1
+    states = np.array([rng.integers(0, dfas[min(max(t, 0), 2)][0].shape[0]) for t in row_table],
+                      dtype=np.int32)
+    logits = rand_logits(rng, B, V, V, "f32")
+    ref = run_step_both(dfas, tables, vb, vo, logits, states, row_table=row_table)
+    assert ref["tokens"][3] == -1 and ref["tokens"][9] == -1 and ref["bad_state_rows"] == 2
+
+
+def test_error_codes_on_device_arguments():
+    dfa = regex_to_dfa("a*")
+    vb, vo = vocab_from_strings([b"a", b"b", b"aa"])
+    vb2, vo2 = vocab_from_strings([b"a", b"b"])
+    (t3,) = gpu_tables([dfa], vb, vo)
+    (t2,) = gpu_tables([dfa], vb2, vo2)
+    ws = cstr.cstr_workspace_create(2)
+    logits = torch.zeros(2, 3, device=DEV)
+    st = torch.zeros(2, dtype=torch.int32, device=DEV)
+    tok = torch.zeros(2, dtype=torch.int32, device=DEV)
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_step([t3, t2], logits, st, tok, torch.empty_like(logits), ws)
+    assert e.value.code == -6
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_step([t3], logits, st, tok, torch.empty_like(logits), ws, vocab_ld=2)
+    assert e.value.code == -6
+    big = torch.zeros(3, 3, device=DEV)
+    st3 = torch.zeros(3, dtype=torch.int32, device=DEV)
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_step([t3], big, st3, st3.clone(), torch.empty_like(big), ws)
+    assert e.value.code == -6
+    unbuilt = cstr.cstr_table_create(t3.vocab, 4)
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_step([unbuilt], logits, st, tok, torch.empty_like(logits), ws)
+    assert e.value.code == -2
+    with pytest.raises(cstr.CstrError):
+        cstr.cstr_table_download(t3, 0, 99)
+
+
+def decode_and_check(name, steps, pool, sample_rows, batch=None, check_all_rows_steps=2):
+    """Run `steps` decoding steps of a workload on the GPU (logits cycling through a
+    pool of `pool` seeded tensors); the oracle replays every step for `sample_rows`
+    (whole trajectory: its own states feed its next step) and all rows for the first steps."""
+    w = CONFIGS[name]
+    B = w.batch if batch is None else batch
+    dfas = config_dfas(name)
+    vb, vo = config_vocab(name)
+    V = vo.size - 1
+    tables = gpu_tables(dfas, vb, vo)
+    row_table = row_table_for(w, B)
+    dec = ConstrainedDecoder(tables, B, row_table=row_table)
+    pools, noises = [], []
+    for k in range(pool):
+        pools.append(normal_logits(w.logits_seed, k, range(B), V, sigma=w.sigma, dtype=w.dtype))
+        noises.append(gumbel_noise(w.noise_seed, k, range(B), V) if w.gumbel else None)
+    d_pool = [to_dev_logits(p) for p in pools]
+    d_noise = [None if n is None else torch.from_numpy(n).to(DEV) for n in noises]
+    rows = sorted(set(sample_rows))
+    starts = np.array([dfas[0 if row_table is None else row_table[r]][2] for r in range(B)], dtype=np.int32)
+    o_states_all = starts.copy()
+    o_states = starts[rows].copy()
+    threads = min(oracle.max_threads(), 32)
+    emitted = 0
+    for t in range(steps):
+        k = t % pool
+        tokens, masked = dec.step(d_pool[k], noise=d_noise[k])
+        g_tok = tokens.cpu().numpy()
+        g_st = dec.states.cpu().numpy()
+        g_masked = from_dev_logits(masked[rows])
+        if t < check_all_rows_steps:
+            ref = oracle.step(dfas, vb, vo, pools[k], o_states_all, noise=noises[k],
+                              row_table=row_table, threads=threads)
+            assert np.array_equal(g_tok, ref["tokens"]) and np.array_equal(g_st, ref["states"])
+            assert bits_equal(from_dev_logits(masked), ref["masked"])
+            o_states_all = ref["states"]
+        ref = oracle.step(dfas, vb, vo, pools[k][rows], o_states,
+                          noise=None if noises[k] is None else noises[k][rows],
+                          row_table=None if row_table is None else row_table[rows], threads=threads)
+        assert np.array_equal(g_tok[rows], ref["tokens"]), "step %d tokens" % t
+        assert np.array_equal(g_st[rows], ref["states"]), "step %d states" % t
+        assert bits_equal(g_masked, ref["masked"]), "step %d masked logits" % t
+        o_states = ref["states"]
+        emitted += int((ref["tokens"] >= 0).sum())
+    assert emitted > 0
+    return dec
+
+
+def test_config_api_1k_full_decode():
+    decode_and_check("api_1k", steps=32, pool=32, sample_rows=range(4), check_all_rows_steps=32)
+
+
+def test_config_json_32k_full_decode():
+    decode_and_check("json_32k", steps=256, pool=4, sample_rows=range(64), check_all_rows_steps=4)
+
+
+def test_config_schema40_128k_gumbel():
+    decode_and_check("schema40_128k", steps=48, pool=2, sample_rows=[0, 1, 100, 255])
+
+
+def test_config_string_256k():
+    decode_and_check("string_256k", steps=12, pool=2, sample_rows=[0, 7, 300, 511],
+                     check_all_rows_steps=1)
+
+
+def test_config_random10k_mixed_batch():
+    decode_and_check("random10k_256k", steps=6, pool=1, sample_rows=[0, 127, 128, 500, 1023],
+                     check_all_rows_steps=1)
+
+
+def test_two_calls_share_a_workspace_in_stream_order():
+    # scratch is reset by the kernel itself: back-to-back steps on one stream need no host work
+    dec = decode_and_check("api_1k", steps=4, pool=4, sample_rows=range(4), batch=64)
+    assert dec.status()[0] == 0

@@ -1,0 +1,132 @@
+"""GPU parity: token table built by libcstr vs the CPU oracle, bit exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2407_08103_b200 import cstr
+from synth import random_range_dfa, vocab_from_strings
+from synth.configs import config_dfas, config_vocab
+from synth.regex_frontend import regex_to_dfa
+
+from gpu_common import check_table, gpu_tables
+
+pytestmark = pytest.mark.gpu
+
+
+def random_vocab(rng, V, max_len=20, alphabet=None, empty_prob=0.02):
+    alphabet = np.arange(256, dtype=np.uint8) if alphabet is None else np.frombuffer(alphabet, dtype=np.uint8)
+    toks = []
+    for _ in range(V):
+        n = 0 if rng.random() < empty_prob else int(min(rng.geometric(0.3), max_len))
+        toks.append(bytes(alphabet[rng.integers(0, alphabet.size, size=n)]))
+    return vocab_from_strings(toks)
+
+
+def dense_random_dfa(rng, S, live=0.7):
+    trans = rng.integers(0, S, size=(S, 256)).astype(np.int32)
+    trans[rng.random((S, 256)) > live] = -1
+    return trans, (rng.random(S) < 0.3).astype(np.uint8), int(rng.integers(S))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small(seed):
+    rng = np.random.default_rng(seed)
+    S = int(rng.choice([1, 2, 3, 17, 64, 100, 257]))
+    V = int(rng.choice([1, 5, 31, 32, 33, 255, 256, 257, 1000, 2049]))
+    dfa = dense_random_dfa(rng, S, live=float(rng.choice([0.2, 0.7, 1.0])))
+    vb, vo = random_vocab(rng, V)
+    eos = int(rng.integers(-1, V)) if seed % 3 == 0 else -1
+    (table,) = gpu_tables([dfa], vb, vo, eos_id=eos)
+    check_table(table, dfa, vb, vo, eos_id=eos)
+
+
+def test_degenerate_cases():
+    # a single state with no edges; all-dead and all-live DFAs; only empty tokens; 16/17-byte tokens
+    dead = (np.full((1, 256), -1, dtype=np.int32), np.zeros(1, dtype=np.uint8), 0)
+    loop = (np.zeros((1, 256), dtype=np.int32), np.ones(1, dtype=np.uint8), 0)
+    toks = [b"", b"a", b"x" * 15, b"y" * 16, b"z" * 17, b"w" * 40, b"", bytes(range(256))]
+    vb, vo = vocab_from_strings(toks)
+    for dfa in (dead, loop):
+        (table,) = gpu_tables([dfa], vb, vo)
+        check_table(table, dfa, vb, vo)
+    vb, vo = vocab_from_strings([b"", b"", b""])
+    (table,) = gpu_tables([loop], vb, vo)
+    check_table(table, loop, vb, vo)
+    # long tokens walking a chain DFA: dies exactly at position 20
+    S = 21
+    trans = np.full((S, 256), -1, dtype=np.int32)
+    for q in range(S - 1):
+        trans[q, 0x61] = q + 1
+    chain = (trans, np.eye(1, S, S - 1, dtype=np.uint8)[0], 0)
+    vb, vo = vocab_from_strings([b"a" * n for n in range(0, 30)])
+    (table,) = gpu_tables([chain], vb, vo)
+    check_table(table, chain, vb, vo)
+
+
+def test_rebuild_reuses_the_table_and_wide_capacity():
+    rng = np.random.default_rng(5)
+    vb, vo = random_vocab(rng, 700)
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    table = cstr.cstr_table_create(vocab, 300)
+    for S in (300, 7, 120):
+        dfa = dense_random_dfa(rng, S)
+        h = cstr.cstr_load_dfa(*dfa)
+        cstr.cstr_table_build(table, h, -1)
+        check_table(table, dfa, vb, vo)
+    too_big = cstr.cstr_load_dfa(*dense_random_dfa(rng, 301))
+    with pytest.raises(cstr.CstrError):
+        cstr.cstr_table_build(table, too_big, -1)
+    # capacity above 32767 states stores 32-bit entries; a small DFA still fits
+    vb2, vo2 = random_vocab(rng, 40)
+    vocab2 = cstr.cstr_load_vocab(vb2, vo2)
+    wide = cstr.cstr_table_create(vocab2, 40000)
+    dfa = dense_random_dfa(rng, 50)
+    h_small = cstr.cstr_load_dfa(*dfa)
+    cstr.cstr_table_build(wide, h_small, -1)
+    check_table(wide, dfa, vb2, vo2)
+    big = random_range_dfa(33000, seed=9)
+    h_big = cstr.cstr_load_dfa(*big)
+    cstr.cstr_table_build(wide, h_big, -1)
+    check_table(wide, big, vb2, vo2, states=[0, 1, 32767, 32768, 32999])
+
+
+def test_one_call_form():
+    dfa = regex_to_dfa("(ab|c)*d")
+    vb, vo = vocab_from_strings([b"a", b"b", b"ab", b"c", b"cd", b"abc", b"d"])
+    h = cstr.cstr_load_dfa(*dfa)
+    table = cstr.cstr_build_token_table(h, vb, vo, eos_id=-1)
+    check_table(table, dfa, vb, vo)
+
+
+@pytest.mark.parametrize("name", ["api_1k", "json_32k"])
+def test_config_full(name):
+    dfa = config_dfas(name)[0]
+    vb, vo = config_vocab(name)
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo)
+
+
+def test_config_schema40_128k():
+    dfa = config_dfas("schema40_128k")[0]
+    vb, vo = config_vocab("schema40_128k")
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo, slab=123)
+
+
+@pytest.mark.parametrize("name", ["string_256k", "random10k_256k"])
+def test_config_256k_sampled_states(name):
+    # Full-size build; the oracle recomputes whole rows for a sample of states
+    # (first, last, slab edges, random), each row being 256,000 transitions.
+    dfa = config_dfas(name)[0]
+    vb, vo = config_vocab(name)
+    (table,) = gpu_tables([dfa], vb, vo)
+    S = dfa[0].shape[0]
+    rng = np.random.default_rng(1)
+    sample = sorted(set([0, 1, 15, 16, 17, S - 17, S - 2, S - 1] + rng.integers(0, S, size=40).tolist()))
+    check_table(table, dfa, vb, vo, states=sample)
+    # popcount of every mask row equals the count of live entries, for a slab of rows
+    nxt, mask = cstr.cstr_table_download(table, 100, 132)
+    live = (nxt >= 0).sum(axis=1)
+    pop = np.unpackbits(mask.view(np.uint8), axis=1).sum(axis=1)
+    assert np.array_equal(live, pop)
