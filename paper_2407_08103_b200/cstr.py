@@ -197,7 +197,7 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
     ld = logits.stride(0) if vocab_ld is None else vocab_ld
     batch = logits.shape[0]
     for name, t in (("masked_out", masked_out), ("noise", noise)):
-        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != ld or t.shape[0] != batch):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0) or t.shape[0] != batch):
             raise ValueError("%s must have the layout of logits" % name)
     if masked_out.dtype != logits.dtype:
         raise TypeError("masked_out must have the dtype of logits")
