@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the constrained decoding step (and the token-table build).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  A "step" is one constrained decoding step (mask from
+state, -inf penalty, arg-max, next state) for the whole batch of the
+``string_256k`` workload: vocabulary 256,000 x batch 512, fp32 logits,
+8,195-state string-literal DFA.  Logits cycle through a pool of seeded
+tensors, each larger than the L2 cache; rows that finish are restarted at the
+start state so every row stays active.  With N > 1 every rank runs an
+independent replica (the path has no exchange step).
+
+``--impl reference`` times the CPU oracle on the same workload instead.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOAD = "string_256k"
+METRIC = "constrained_step_logits_per_s"
+UNIT = "logits/s"
+POOL = 4
+BYTES_PER_LOGIT_F32_GREEDY = 4 + 4 + 1.0 / 8.0    # read + masked write + mask bit
+BYTES_PER_TRANSITION = 2 + 1.0 / 8.0              # int16 next entry + mask bit, stores only
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2560)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=12.0,
+                    help="CPU time budget of the oracle baseline leg")
+    ap.add_argument("--skip-build-bench", action="store_true")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def workload_inputs(rank: int, batch: int):
+    """Seeded host inputs: DFA, vocabulary, pool of logits tensors (rows keyed by global row id)."""
+    from synth import normal_logits
+    from synth.configs import CONFIGS, config_dfas, config_vocab
+    w = CONFIGS[WORKLOAD]
+    dfa = config_dfas(WORKLOAD)[0]
+    vb, vo = config_vocab(WORKLOAD)
+    return w, dfa, vb, vo
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock, power and clock-event reasons through NVML (read-only)."""
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []      # (t, sm_mhz, reasons_bitmask, power_w)
+        self.stop_flag = threading.Event()
+        self.ok = False
+        self.sm_max = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as exc:  # pragma: no cover - depends on the box
+            self.err = repr(exc)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag.is_set():
+            try:
+                sm = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.samples.append((time.perf_counter(), sm, rs, pw))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["unavailable"]}
+        nv = self.nv
+        sel = [s for s in self.samples if t0 <= s[0] <= t1]
+        window = "timed region"
+        if len(sel) < 3:
+            sel, window = self.samples, "whole run (timed region shorter than 3 samples)"
+        names = {
+            nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksEventReasonHwPowerBrakeSlowdown: "hw_power_brake_slowdown",
+            nv.nvmlClocksEventReasonApplicationsClocksSetting: "applications_clocks_setting",
+            nv.nvmlClocksEventReasonSyncBoost: "sync_boost",
+        }
+        seen = 0
+        for s in sel:
+            seen |= s[2]
+        reasons = [n for bit, n in names.items() if seen & bit]
+        return {"sm_mhz": float(np.median([s[1] for s in sel])), "sm_max_mhz": self.sm_max,
+                "reasons": reasons, "power_w_max": max(s[3] for s in sel), "samples": len(sel),
+                "window": window}
+
+
+def time_oracle(w, dfa, vb, vo, pools, budget_s: float, max_steps: int):
+    """The oracle as it stands, all host threads, whole-batch steps until the
+    time budget is used (at least 2 steps).  Returns (logits/s, cores, sample text, s/step)."""
+    import oracle
+    threads = oracle.max_threads()
+    B, V = pools[0].shape
+    states = np.full(B, dfa[2], dtype=np.int32)
+    oracle.step([dfa], vb, vo, pools[0][:8], states[:8], threads=threads)   # load + warm
+    done, t0 = 0, time.perf_counter()
+    while done < max_steps and (done < 2 or time.perf_counter() - t0 < budget_s):
+        res = oracle.step([dfa], vb, vo, pools[done % len(pools)], states, threads=threads)
+        states = np.where(res["states"] < 0, dfa[2], res["states"]).astype(np.int32)
+        done += 1
+    dt = time.perf_counter() - t0
+    sample = "%d whole-batch steps (%d rows x %d tokens) of %s, %.1f s" % (done, B, V, WORKLOAD, dt)
+    return B * V * done / dt, threads, sample, dt / done
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from synth import normal_logits
+    w, dfa, vb, vo = workload_inputs(0, 0)
+    V = vo.size - 1
+    B = w.batch
+    import oracle
+    oracle.build()
+    pools = [normal_logits(w.logits_seed, k, range(B), V) for k in range(2)]
+    threads = oracle.max_threads()
+    states = np.full(B, dfa[2], dtype=np.int32)
+    # bounded sample: each "step" of this arm is one whole-batch oracle step
+    steps = max(1, min(args.steps, 40))
+    warm = max(1, min(args.warmup, 3))
+    for i in range(warm):
+        oracle.step([dfa], vb, vo, pools[i % 2], states, threads=threads)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        res = oracle.step([dfa], vb, vo, pools[i % 2], states, threads=threads)
+        states = np.where(res["states"] < 0, dfa[2], res["states"]).astype(np.int32)
+    dt = time.perf_counter() - t0
+    value = B * V * steps / dt
+    sample = "%d whole-batch oracle steps (%d rows x %d tokens) of %s" % (steps, B, V, WORKLOAD)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": dt / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "vocab": V, "batch": B, "dfa_states": int(dfa[0].shape[0]),
+                   "sampler": "greedy", "note": "CPU oracle, host cores only"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2407_08103_b200 import build as libbuild
+    from paper_2407_08103_b200 import cstr
+    from paper_2407_08103_b200.decode import ConstrainedDecoder
+    from synth import normal_logits
+    libbuild.build_library()
+
+    w, dfa, vb, vo = workload_inputs(rank, 0)
+    V = vo.size - 1
+    B = w.batch
+    S = int(dfa[0].shape[0])
+    K, W = args.steps, max(args.warmup, 3)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- set-up: vocabulary, DFA, table (the table build is timed below) ----
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    h_dfa = cstr.cstr_load_dfa(*dfa)
+    table = cstr.cstr_table_create(vocab, S)
+    build_ms = []
+    for _ in range(4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        cstr.cstr_table_build(table, h_dfa, -1, stream)
+        e1.record(stream)
+        e1.synchronize()
+        build_ms.append(e0.elapsed_time(e1))
+    t_e2e0 = time.perf_counter()
+    h2 = cstr.cstr_load_dfa(*dfa)          # end to end: DFA upload + build, host clock
+    cstr.cstr_table_build(table, h2, -1, stream)
+    torch.cuda.synchronize()
+    build_e2e_ms = (time.perf_counter() - t_e2e0) * 1e3
+
+    # ---- inputs: pinned host pool (rows keyed by global row id), device pool ----
+    host_pool = [torch.empty((B, V), dtype=torch.float32).pin_memory() for _ in range(POOL)]
+    for k in range(POOL):
+        normal_logits(w.logits_seed, k, range(rank * B, rank * B + B), V, out=host_pool[k].numpy())
+    dev_pool = [t.to(dev, non_blocking=True) for t in host_pool]
+    out_bufs = [torch.empty((B, V), dtype=torch.float32, device=dev) for _ in range(2)]
+    dec = ConstrainedDecoder(table, B, device=dev)
+    start_vec = torch.full((B,), int(dfa[2]), dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+
+    def one_step(i, logits):
+        dec.step(logits, masked_out=out_bufs[i & 1], stream=stream)
+        # continuous batching: a finished row is replaced by a fresh sequence
+        torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    # ---- device-resident timing ------------------------------------------
+    for i in range(W):
+        one_step(i, dev_pool[i % POOL])
+    dec.status()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_dev0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(K):
+        one_step(i, dev_pool[i % POOL])
+    e1.record(stream)
+    barrier()
+    t_dev1 = time.perf_counter()
+    dev_ms = max_over_ranks(e0.elapsed_time(e1))
+    bad, empty = dec.status()
+
+    # duration of the step kernel alone (events around each launch; the restart
+    # op runs outside the bracket), for the roofline
+    ks = min(K, 128)
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(ks)]
+    for i in range(ks):
+        pairs[i][0].record(stream)
+        dec.step(dev_pool[i % POOL], masked_out=out_bufs[i & 1], stream=stream)
+        pairs[i][1].record(stream)
+        torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
+    torch.cuda.synchronize()
+    kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    active_frac = float((dec.states >= 0).float().mean().item())
+
+    # ---- end to end: pinned host logits in, tokens + states out, every step ----
+    staging = [torch.empty((B, V), dtype=torch.float32, device=dev) for _ in range(2)]
+    h_tok = torch.empty(B, dtype=torch.int32).pin_memory()
+    h_st = torch.empty(B, dtype=torch.int32).pin_memory()
+    Ke = min(K, 64)
+    dec.reset()
+
+    def e2e_step(i):
+        buf = staging[i & 1]
+        buf.copy_(host_pool[i % POOL], non_blocking=True)
+        one_step(i, buf)
+        h_tok.copy_(dec.tokens, non_blocking=True)
+        h_st.copy_(dec.states, non_blocking=True)
+        stream.synchronize()               # the sampling loop needs the tokens on the host
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(Ke):
+        e2e_step(i)
+    f1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(f0.elapsed_time(f1))
+    sampler.stop_flag.set()
+    sampler.join(timeout=2)
+    clocks = sampler.summary(t_dev0, t_dev1)
+
+    # ---- table-build scaling workload: random 10,000-state DFA ------------
+    build_random = None
+    if not args.skip_build_bench and rank == 0:
+        from synth import random_range_dfa
+        rd = random_range_dfa(10000, seed=2)
+        h_rd = cstr.cstr_load_dfa(*rd)
+        t_rd = cstr.cstr_table_create(vocab, 10000)
+        ms = []
+        for _ in range(4):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            cstr.cstr_table_build(t_rd, h_rd, -1, stream)
+            a1.record(stream)
+            a1.synchronize()
+            ms.append(a0.elapsed_time(a1))
+        build_random = ms[1:]
+        del t_rd, h_rd
+
+    # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1) --------
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu_baseline:
+        pools = [host_pool[k].numpy() for k in range(2)]
+        v, cores, sample, _ = time_oracle(w, dfa, vb, vo, pools, args.cpu_seconds, 400)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_hbm_peak()
+    logits_per_step = B * V * world
+    value = logits_per_step * K / (dev_ms * 1e-3)
+    step_bytes = B * V * BYTES_PER_LOGIT_F32_GREEDY
+    achieved = step_bytes / (kernel_ms * 1e-3) / 1e9
+    bt = np.array(build_ms[1:])
+    transitions = S * V
+
+    def build_entry(ms_list, s_states, workload):
+        ms_best = float(np.mean(ms_list))
+        tps = s_states * V / (ms_best * 1e-3)
+        gbs = s_states * V * BYTES_PER_TRANSITION / (ms_best * 1e-3) / 1e9
+        return {"workload": workload, "dfa_states": s_states, "vocab": V, "ms": ms_best,
+                "value": tps, "unit": "transitions/s",
+                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                             "frac": gbs / peak, "traffic": None,
+                             "note": "stores of next (int16) + mask only; of %s copy rate" % peak_kind}}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "vocab": V, "batch": B, "dfa_states": S,
+                   "sampler": "greedy", "logits": "fp32 N(0,1), pool of %d seeded tensors" % POOL,
+                   "l2": "inputs larger than L2 (each logits tensor %.0f MB, rotated)" % (B * V * 4 / 1e6),
+                   "rows": "finished rows restart at the start state (all rows active)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "e2e": {"value": logits_per_step * Ke / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * 8, "steps": Ke,
+                "ms_per_step": e2e_ms / Ke,
+                "note": "pinned host logits -> device, cstr_step, tokens+states -> host, sync per step"},
+        "gpu_launches": K,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None,
+                     "kernel": "step_vec_kernel<fp32, greedy>", "kernel_ms": kernel_ms,
+                     "bytes_per_launch": step_bytes, "peak_kind": "of %s" % peak_kind,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "active_row_fraction_at_end": active_frac},
+        "cpu_baseline": cpu,
+        "table_build": [build_entry(bt, S, WORKLOAD)] +
+                       ([build_entry(build_random, 10000, "random10k_256k (DFA 0)")] if build_random else []),
+        "table_build_e2e_ms": build_e2e_ms,
+        "status_rows": {"bad_state": bad, "empty_mask": empty},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -484,7 +484,10 @@ extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
     a.masked_out = masked_out;
     a.accept_out = accept_out;
     a.batch = batch;
-    a.ws = ws;
+    a.cell = ws->cell;
+    a.ticket = ws->ticket;
+    a.counters = ws->counters;
+    a.device = ws->device;
     return cstr_launch_step(a, (cudaStream_t)cuda_stream);
 }
 

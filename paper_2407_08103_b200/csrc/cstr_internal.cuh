@@ -84,6 +84,10 @@ struct cstr_step_args {
     void *masked_out;
     uint8_t *accept_out;
     int32_t batch;
-    cstr_workspace *ws;
+    // scratch, zero on entry and left zero by the kernel (see cstr_step.cu)
+    unsigned long long *cell;      // DEVICE [batch]
+    unsigned int *ticket;          // DEVICE [batch]
+    unsigned long long *counters;  // DEVICE [2]
+    int device;
 };
 int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream);

@@ -384,9 +384,9 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     p.states = a.states;
     p.tokens = a.tokens_out;
     p.accept_out = a.accept_out;
-    p.cell = a.ws->cell;
-    p.ticket = a.ws->ticket;
-    p.counters = a.ws->counters;
+    p.cell = a.cell;
+    p.ticket = a.ticket;
+    p.counters = a.counters;
     p.ld = a.ld;
     p.V = t0->V;
     p.n_tables = a.n_tables;
@@ -397,7 +397,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     const int total_tiles = (p.V + tile - 1) / tile;
     // 8 tiles (one per warp) per CTA when there is enough work to fill the
     // machine a few times over, fewer for small batches.
-    const long long want_ctas = 4LL * sm_count(a.ws->device);
+    const long long want_ctas = 4LL * sm_count(a.device);
     int tiles_per_cta = 8;
     while (tiles_per_cta > 1 &&
            (long long)a.batch * ((total_tiles + tiles_per_cta - 1) / tiles_per_cta) < want_ctas)
