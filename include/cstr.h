@@ -190,6 +190,40 @@ int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t
 int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t *bad_state_rows,
                      int64_t *empty_mask_rows);
 
+/*
+ * cstr_step without any allocation, for callers that cannot create a
+ * workspace.  (The paper has no counterpart; this is a deployment aid.)
+ *
+ * Some hosts of this library may not call the CUDA allocator once they are
+ * running: an inference server that hands all free device memory to its
+ * KV-cache pool at start-up, so that a later cudaMalloc can fail; a plug-in
+ * that must live inside a memory budget fixed by its host process; a
+ * latency-critical decode loop that cannot afford cudaMalloc's device-wide
+ * synchronisation.  For them the per-row scratch of the step is a fixed array
+ * inside the library image: about 48 KB of device memory on every GPU that
+ * loads libcstr, held until the process exits, enough for
+ * CSTR_STATIC_MAX_BATCH rows.
+ *
+ * Arguments, semantics and results are exactly those of cstr_step, without the
+ * workspace.  The call allocates nothing (no cudaMalloc / cudaFree, no
+ * allocating library routine); it enqueues one small memset and the step
+ * kernel on cuda_stream.  batch > CSTR_STATIC_MAX_BATCH is rejected with
+ * CSTR_ERR_SHAPE.  The status counters of cstr_step_status are not available
+ * here; a row's token of -1 carries the same information.
+ *
+ * The first call on each device looks up the array's device address (with
+ * that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents, so each call clears it first; two calls that may overlap on the
+ * GPU (different streams without an ordering between them) race on it - order
+ * them, or use cstr_step with one workspace per stream.
+ */
+#define CSTR_STATIC_MAX_BATCH 4096
+int cstr_step_static(const cstr_table_t *const *tables, int32_t n_tables,
+                     const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
+                     const float *noise, int32_t *states, int32_t *tokens_out, void *masked_out,
+                     uint8_t *accept_out, int32_t batch, void *cuda_stream);
+
 /* Message for the calling thread's most recent error ("" if none). */
 const char *cstr_last_error(void);
 

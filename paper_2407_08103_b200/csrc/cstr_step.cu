@@ -13,6 +13,9 @@
 // resets the scratch.  Nobody waits on anybody.
 #include <cuda_bf16.h>
 #include <math_constants.h>
+#include <string.h>
+
+#include <mutex>
 
 #include "cstr_internal.cuh"
 
@@ -434,4 +437,107 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     }
     CSTR_CUDA_TRY(cudaGetLastError());
     return CSTR_OK;
+}
+
+// ---- allocation-free variant -------------------------------------------------
+//
+// Same kernels, but the per-row scratch (cells, tickets, counters) lives in one
+// fixed array that is part of the loaded library image, so the call never asks
+// the CUDA allocator for anything.
+
+namespace {
+
+constexpr int kStaticRows = CSTR_STATIC_MAX_BATCH;
+// [0, kStaticRows) cells (u64) | tickets (u32, two per u64) | 2 counters
+constexpr size_t kStaticWords = (size_t)kStaticRows + (size_t)kStaticRows / 2 + 2;
+
+static __device__ __align__(256) unsigned long long g_static_scratch[kStaticWords];
+
+// Device address of g_static_scratch per device, resolved on first use.  In
+// host code the symbol's name is only a handle for the runtime, not a device
+// address, so it must never be passed to a kernel directly.
+std::mutex g_static_mutex;
+unsigned long long *g_static_ptr[64] = {nullptr};
+
+}  // namespace
+
+extern "C" int cstr_step_static(const cstr_table_t *const *tables, int32_t n_tables,
+                                const int32_t *row_table, const void *logits, int32_t dtype,
+                                int64_t ld, const float *noise, int32_t *states,
+                                int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
+                                int32_t batch, void *cuda_stream)
+{
+    if (!tables || !logits || !states || !tokens_out || !masked_out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_step_static: null pointer");
+    if (n_tables < 1 || n_tables > CSTR_MAX_TABLES)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_step_static: n_tables = %d, need 1..%d", n_tables,
+                         CSTR_MAX_TABLES);
+    if (dtype != CSTR_F32 && dtype != CSTR_BF16)
+        return cstr_fail(CSTR_ERR_DTYPE, "cstr_step_static: unknown dtype %d", dtype);
+    if (batch < 0)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_step_static: batch = %d", batch);
+    if (batch > kStaticRows)
+        return cstr_fail(CSTR_ERR_SHAPE,
+                         "cstr_step_static: batch %d exceeds the built-in scratch of %d rows; "
+                         "use cstr_step with a workspace for larger batches",
+                         batch, kStaticRows);
+    int device = -1;
+    CSTR_CUDA_TRY(cudaGetDevice(&device));
+    if (device < 0 || device >= 64)
+        return cstr_fail(CSTR_ERR_DEVICE, "cstr_step_static: device index %d not supported", device);
+    cstr_step_args a;
+    memset(&a, 0, sizeof a);
+    for (int32_t i = 0; i < n_tables; ++i) {
+        const cstr_table *t = tables[i];
+        if (!t)
+            return cstr_fail(CSTR_ERR_NULL, "cstr_step_static: tables[%d] is null", i);
+        if (t->device != device)
+            return cstr_fail(CSTR_ERR_DEVICE, "cstr_step_static: tables[%d] is on device %d, "
+                             "device %d is current", i, t->device, device);
+        if (t->n_states < 1)
+            return cstr_fail(CSTR_ERR_ARG, "cstr_step_static: tables[%d] has not been built", i);
+        if (t->V != tables[0]->V)
+            return cstr_fail(CSTR_ERR_SHAPE, "cstr_step_static: tables[%d] has V = %d, "
+                             "tables[0] has %d", i, t->V, tables[0]->V);
+        a.tables[i] = t;
+    }
+    if (ld < tables[0]->V)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_step_static: ld = %lld is below V = %d",
+                         (long long)ld, tables[0]->V);
+    if (batch == 0)
+        return CSTR_OK;
+
+    unsigned long long *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[device]) {
+            void *ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e != cudaSuccess || !ptr)
+                return cstr_fail(CSTR_ERR_CUDA, "cstr_step_static: cudaGetSymbolAddress: %s",
+                                 cudaGetErrorString(e));
+            g_static_ptr[device] = (unsigned long long *)ptr;
+        }
+        scratch = g_static_ptr[device];
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // The array keeps whatever the previous call (or an interrupted one) left.
+    CSTR_CUDA_TRY(cudaMemsetAsync(scratch, 0, kStaticWords * sizeof(unsigned long long), stream));
+
+    a.n_tables = n_tables;
+    a.row_table = row_table;
+    a.logits = logits;
+    a.dtype = dtype;
+    a.ld = ld;
+    a.noise = noise;
+    a.states = states;
+    a.tokens_out = tokens_out;
+    a.masked_out = masked_out;
+    a.accept_out = accept_out;
+    a.batch = batch;
+    a.cell = scratch;
+    a.ticket = (unsigned int *)(scratch + kStaticRows);
+    a.counters = scratch + kStaticRows + kStaticRows / 2;
+    a.device = device;
+    return cstr_launch_step(a, stream);
 }

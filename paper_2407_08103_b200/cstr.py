@@ -18,12 +18,13 @@ from .build import LIB_PATH
 CSTR_F32 = 0
 CSTR_BF16 = 1
 CSTR_MAX_TABLES = 16
+CSTR_STATIC_MAX_BATCH = 4096
 
 EXPORTS = [
     "cstr_load_dfa", "cstr_free_dfa", "cstr_load_vocab", "cstr_free_vocab",
     "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
-    "cstr_step", "cstr_step_status", "cstr_last_error",
+    "cstr_step", "cstr_step_status", "cstr_step_static", "cstr_last_error",
 ]
 
 _lib = None
@@ -213,6 +214,36 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
                            _dev_ptr(states), _dev_ptr(tokens_out), _dev_ptr(masked_out),
                            _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
                            _stream_ptr(stream)))
+
+
+def cstr_step_static(tables, logits, states, tokens_out, masked_out, noise=None, row_table=None,
+                     accept_out=None, stream=None) -> None:
+    """``cstr_step`` for callers that must not allocate: no workspace, the scratch
+    is a fixed array inside the library (at most ``CSTR_STATIC_MAX_BATCH`` rows;
+    calls that may overlap on the GPU must be ordered by the caller).  Same
+    tensors and results as ``cstr_step``."""
+    import torch
+    if isinstance(tables, Table):
+        tables = [tables]
+    if logits.dtype == torch.float32:
+        dtype = CSTR_F32
+    elif logits.dtype == torch.bfloat16:
+        dtype = CSTR_BF16
+    else:
+        raise TypeError("logits must be float32 or bfloat16")
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [B][ld] with unit inner stride")
+    batch = logits.shape[0]
+    for name, t in (("masked_out", masked_out), ("noise", noise)):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0)
+                              or t.shape[0] != batch):
+            raise ValueError("%s must have the layout of logits" % name)
+    arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
+    _check(lib().cstr_step_static(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
+                                  _dev_ptr(logits), ctypes.c_int32(dtype),
+                                  ctypes.c_int64(logits.stride(0)), _dev_ptr(noise),
+                                  _dev_ptr(states), _dev_ptr(tokens_out), _dev_ptr(masked_out),
+                                  _dev_ptr(accept_out), ctypes.c_int32(batch), _stream_ptr(stream)))
 
 
 def cstr_step_status(ws: Workspace, stream=None):
