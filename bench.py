@@ -46,7 +46,11 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0,
                     help="CPU time budget of the oracle baseline leg")
+    ap.add_argument("--case", default="full", choices=["full", "small"],
+                    help="small: batch 128 and a 515-state string-literal DFA over the same "
+                         "vocabulary (for profiler captures); its numbers are not bench values")
     ap.add_argument("--skip-build-bench", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -60,13 +64,18 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def workload_inputs(rank: int, batch: int):
-    """Seeded host inputs: DFA, vocabulary, pool of logits tensors (rows keyed by global row id)."""
-    from synth import normal_logits
+def workload_inputs(case: str = "full"):
+    """Seeded host inputs of the benchmark workload: recipe, DFA, vocabulary."""
+    import dataclasses
     from synth.configs import CONFIGS, config_dfas, config_vocab
     w = CONFIGS[WORKLOAD]
-    dfa = config_dfas(WORKLOAD)[0]
     vb, vo = config_vocab(WORKLOAD)
+    if case == "small":
+        from synth.regex_frontend import regex_to_dfa
+        w = dataclasses.replace(w, batch=128)
+        dfa = regex_to_dfa(w.regex.replace("{0,4096}", "{0,256}"))
+    else:
+        dfa = config_dfas(WORKLOAD)[0]
     return w, dfa, vb, vo
 
 
@@ -160,7 +169,7 @@ def run_reference(args):
     if rank != 0:
         return
     from synth import normal_logits
-    w, dfa, vb, vo = workload_inputs(0, 0)
+    w, dfa, vb, vo = workload_inputs(args.case)
     V = vo.size - 1
     B = w.batch
     import oracle
@@ -218,7 +227,7 @@ def main():
     from synth import normal_logits
     libbuild.build_library()
 
-    w, dfa, vb, vo = workload_inputs(rank, 0)
+    w, dfa, vb, vo = workload_inputs(args.case)
     V = vo.size - 1
     B = w.batch
     S = int(dfa[0].shape[0])
@@ -318,16 +327,18 @@ def main():
         h_st.copy_(dec.states, non_blocking=True)
         stream.synchronize()               # the sampling loop needs the tokens on the host
 
-    for i in range(3):
-        e2e_step(i)
-    barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(stream)
-    for i in range(Ke):
-        e2e_step(i)
-    f1.record(stream)
-    barrier()
-    e2e_ms = max_over_ranks(f0.elapsed_time(f1))
+    e2e_ms = float("nan")
+    if not args.skip_e2e:
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for i in range(Ke):
+            e2e_step(i)
+        f1.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(f0.elapsed_time(f1))
     sampler.stop_flag.set()
     sampler.join(timeout=2)
     clocks = sampler.summary(t_dev0, t_dev1)
@@ -380,19 +391,23 @@ def main():
                              "frac": gbs / peak, "traffic": None,
                              "note": "stores of next (int16) + mask only; of %s copy rate" % peak_kind}}
 
+    e2e = None
+    if not args.skip_e2e:
+        e2e = {"value": logits_per_step * Ke / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * 8, "steps": Ke,
+               "ms_per_step": e2e_ms / Ke,
+               "note": "pinned host logits -> device, cstr_step, tokens+states -> host, sync per step"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "vocab": V, "batch": B, "dfa_states": S,
+        "config": {"workload": WORKLOAD if args.case == "full" else WORKLOAD + " (small profiling case)",
+                   "vocab": V, "batch": B, "dfa_states": S,
                    "sampler": "greedy", "logits": "fp32 N(0,1), pool of %d seeded tensors" % POOL,
                    "l2": "inputs larger than L2 (each logits tensor %.0f MB, rotated)" % (B * V * 4 / 1e6),
                    "rows": "finished rows restart at the start state (all rows active)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
-        "e2e": {"value": logits_per_step * Ke / (e2e_ms * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * 8, "steps": Ke,
-                "ms_per_step": e2e_ms / Ke,
-                "note": "pinned host logits -> device, cstr_step, tokens+states -> host, sync per step"},
+        "e2e": e2e,
         "gpu_launches": K,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
