@@ -1,72 +1,217 @@
-// Token-table builder: next[q][v] = delta*(q, bytes(v)) and the allowed-token
+// Token-table builder: next[v][q] = delta*(q, bytes(v)) and the allowed-token
 // bitmask, for every DFA state q and vocabulary token v (Algorithm 1 composed
 // with the DFA as in Algorithm 2; Theorem 2 fixes the meaning).
 //
-// Work decomposition: a CTA owns 256 consecutive tokens (one per thread, the
-// first 16 bytes of the token held in four registers) and a block of
-// consecutive states; for each state every lane walks its own token through
-// the DFA, the warp votes the 32 results into one mask word with a ballot, and
-// the next-state entries go out as one coalesced row segment.  The DFA is read
-// through the read-only path (it stays resident in L1/L2: 512 bytes per state
-// as int16).
+// The detokenizing transducer of Algorithm 1 has a compact, trie-like form in
+// which tokens share the chain of their common prefix (Section 2.3, Figure 3).
+// The builder walks exactly that trie: tokens come in lexicographic order with
+// the length of the prefix each shares with its predecessor, and a warp that
+// owns a block of DFA states (one or more states per lane) keeps, per depth of
+// the current trie path, the state every lane has reached.  A token then costs
+// only the lookups of the bytes it does not share with the previous token.
+//
+//   - lane = state: every lane of a warp reads the same token, so there is no
+//     divergence on token length, and all control flow is warp-uniform;
+//   - the DFA is class-compressed and class-major (tt[class][state]) with a
+//     self-looping dead-sink column: a lookup is one indexed load, the first
+//     byte of a walk reads consecutive entries, and dead walks need no branch;
+//     it lives in shared memory when it fits, else it is gathered through L1/L2;
+//   - next-state entries leave as 64-byte state segments of the token's row;
+//     validity goes out as one ballot word per (token, 32-state block), which a
+//     second kernel bit-transposes into the state-major mask the step streams.
 #include "cstr_internal.cuh"
 
 namespace {
 
-constexpr int kBuildThreads = 256;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kDepth = CSTR_STACK_DEPTH;
 
-template <typename DT, typename NT>
-__global__ void __launch_bounds__(kBuildThreads)
-build_rows_kernel(const DT *__restrict__ dfa, int n_states, const uint8_t *__restrict__ accept,
-                  const uint4 *__restrict__ head, const uint32_t *__restrict__ len_arr,
-                  const uint8_t *__restrict__ bytes, const uint32_t *__restrict__ off, int V,
-                  int eos_id, NT *__restrict__ next, int64_t ldn, uint32_t *__restrict__ mask,
-                  int64_t ldw, int states_per_cta)
+struct BuildParams {
+    const void *tt;            // [n_classes][row]
+    const uint8_t *cls;        // [256]
+    const uint8_t *accept;     // [n_states]
+    const uint4 *desc;         // [V] sorted tokens
+    const uint8_t *bytes;      // raw vocabulary bytes
+    const uint32_t *off;       // [V + 1]
+    void *next;                // [V][lds]
+    uint32_t *maskT;           // [V][ldb]
+    long long row, lds, ldb;
+    int n_states, n_classes, V, eos_id;
+    int tokens_per_cta;
+    int table_in_smem;
+};
+
+// ST: entry type of the DFA table; NT: entry type of next; NS: states per lane.
+template <typename ST, typename NT, int NS>
+__global__ void __launch_bounds__(256)
+build_trie_kernel(const __grid_constant__ BuildParams p)
 {
-    const int v = blockIdx.x * kBuildThreads + threadIdx.x;
-    const bool in_vocab = v < V;
-    uint4 rec = make_uint4(0, 0, 0, 0);
-    uint32_t len = 0;
-    uint32_t begin = 0;
-    if (in_vocab) {
-        rec = head[v];
-        len = len_arr[v];
-        begin = off[v];
-    }
-    const uint32_t w[4] = {rec.x, rec.y, rec.z, rec.w};
-    const int q0 = blockIdx.y * states_per_cta;
-    const int q1 = min(n_states, q0 + states_per_cta);
-    const bool is_eos = in_vocab && v == eos_id;
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int sink = p.n_states;
 
-    for (int q = q0; q < q1; ++q) {
-        int s = (len > 0) ? q : CSTR_DEAD;
+    // shared memory: [class map 256 B][stack: nwarps x (kDepth+1) x NS x 32 ST][table]
+    uint8_t *s_cls = smem;
+    ST *s_stack = (ST *)(smem + 256) + (size_t)warp * (kDepth + 1) * NS * 32;
+    ST *s_tt = (ST *)(smem + 256) + (size_t)nwarps * (kDepth + 1) * NS * 32;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x)
+        s_cls[i] = p.cls[i];
+    const ST *tt = (const ST *)p.tt;
+    if (p.table_in_smem) {
+        const long long n16 = (long long)p.n_classes * p.row * (long long)sizeof(ST) / 16;
+        const uint4 *src = (const uint4 *)p.tt;
+        uint4 *dst = (uint4 *)s_tt;      // row is a multiple of 8 entries: whole 16-byte units
+        for (long long i = threadIdx.x; i < n16; i += blockDim.x)
+            dst[i] = __ldg(src + i);
+        tt = s_tt;
+    }
+    __syncthreads();
+
+    const int q0 = (blockIdx.x * nwarps + warp) * NS * 32;
+    if (q0 >= p.n_states)
+        return;                                          // whole warp out of range
+    int q[NS];
+    bool in_range[NS], acc[NS];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const bool go = (k < (int)len) && (s >= 0);
-            if (!__any_sync(0xffffffffu, go))
-                break;
-            if (go) {
-                const uint32_t b = (w[k >> 2] >> (8 * (k & 3))) & 0xffu;
-                s = (int)__ldg(dfa + (int64_t)s * 256 + b);
+    for (int j = 0; j < NS; ++j) {
+        q[j] = q0 + j * 32 + lane;
+        in_range[j] = q[j] < p.n_states;
+        acc[j] = in_range[j] && p.accept[q[j]] != 0;
+        s_stack[(0 * NS + j) * 32 + lane] = (ST)(in_range[j] ? q[j] : sink);
+    }
+    __syncwarp();
+
+    const int t_begin = blockIdx.y * p.tokens_per_cta;
+    const int t_end = min(p.V, t_begin + p.tokens_per_cta);
+    int cur[NS];
+#pragma unroll
+    for (int j = 0; j < NS; ++j)
+        cur[j] = in_range[j] ? q[j] : sink;
+    int depth = 0;                                       // depth of the path held in cur[]
+    NT *next = (NT *)p.next;
+
+    for (int i = t_begin; i < t_end; ++i) {
+        const uint4 d = __ldg(p.desc + i);               // same address in every lane
+        const int tok = (int)d.x;
+        const int n = (int)(d.y & 0xffffffu);
+        const int shared = (i == t_begin) ? 0 : (int)(d.y >> 24);
+        if (shared < depth) {                            // climb back to the shared prefix
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+                cur[j] = (int)s_stack[(shared * NS + j) * 32 + lane];
+        }
+        const bool inline_ok = (i != t_begin);           // d.z / d.w hold bytes shared..shared+7
+        const uint32_t begin = inline_ok ? 0u : __ldg(p.off + tok);
+        for (int k = shared; k < n; ++k) {
+            uint32_t b;
+            const int r = k - shared;
+            if (inline_ok && r < 8)
+                b = ((r < 4 ? d.z : d.w) >> (8 * (r & 3))) & 0xffu;
+            else
+                b = __ldg(p.bytes + (inline_ok ? __ldg(p.off + tok) : begin) + k);
+            const ST *rowp = tt + (long long)s_cls[b] * p.row;
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+                cur[j] = (int)rowp[cur[j]];
+            if (k + 1 <= kDepth) {
+#pragma unroll
+                for (int j = 0; j < NS; ++j)
+                    s_stack[((k + 1) * NS + j) * 32 + lane] = (ST)cur[j];
             }
         }
-        if (len > 16 && s >= 0) {       // rare: tokens longer than the packed head
-            for (uint32_t k = 16; k < len; ++k) {
-                s = (int)__ldg(dfa + (int64_t)s * 256 + bytes[begin + k]);
-                if (s < 0)
-                    break;
+        depth = n;
+        const bool is_eos = tok == p.eos_id;
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+            int s = (n > 0 && cur[j] != sink) ? cur[j] : CSTR_DEAD;
+            bool allowed = s >= 0;
+            if (is_eos) {                // allowed exactly in accepting states; finishes the row
+                allowed = acc[j];
+                s = CSTR_DEAD;
+            }
+            const uint32_t word = __ballot_sync(kFull, allowed && in_range[j]);
+            const int qb = q0 + j * 32;
+            if (qb < p.n_states) {
+                if (in_range[j])
+                    next[(long long)tok * p.lds + q[j]] = (NT)s;
+                if (lane == 0)
+                    p.maskT[(long long)tok * p.ldb + (qb >> 5)] = word;
             }
         }
-        bool allowed = s >= 0;
-        if (is_eos) {                   // allowed exactly in accepting states; finishes the row
-            allowed = accept[q] != 0;
-            s = CSTR_DEAD;
+    }
+}
+
+// mask[q][w] bit t = maskT[32 w + t][q / 32] bit (q % 32): 32 x 32 bit-matrix
+// transposes.  A CTA takes 1,024 tokens (32 mask words) x 8 state blocks; warp j
+// transposes the 32 tiles of state block j and each lane writes the 32
+// consecutive words of its state row (128 bytes).
+__global__ void __launch_bounds__(256)
+mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
+                      long long ldw, int n_states, int V)
+{
+    __shared__ uint32_t tile[8][1024];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int w0 = blockIdx.x * 32;
+    const int sb0 = blockIdx.y * 8;
+    for (int t = threadIdx.x; t < 1024; t += 256) {
+        const long long tokid = (long long)w0 * 32 + t;
+        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+        if (tokid < V) {
+            const uint4 *src = (const uint4 *)(maskT + tokid * ldb + sb0);   // ldb, sb0 multiples of 8
+            a = __ldg(src);
+            b = __ldg(src + 1);
         }
-        const uint32_t word = __ballot_sync(0xffffffffu, allowed && in_vocab);
-        if (in_vocab)
-            next[(int64_t)q * ldn + v] = (NT)s;
-        if ((threadIdx.x & 31) == 0 && in_vocab)
-            mask[(int64_t)q * ldw + (v >> 5)] = word;
+        tile[0][t] = a.x; tile[1][t] = a.y; tile[2][t] = a.z; tile[3][t] = a.w;
+        tile[4][t] = b.x; tile[5][t] = b.y; tile[6][t] = b.z; tile[7][t] = b.w;
+    }
+    __syncthreads();
+    const int q = (sb0 + warp) * 32 + lane;
+    if ((sb0 + warp) * 32 >= n_states)
+        return;
+    uint32_t outw[32];
+#pragma unroll
+    for (int wi = 0; wi < 32; ++wi) {
+        uint32_t x = tile[warp][wi * 32 + lane];         // row = token, bit = state
+        uint32_t m = 0x0000ffffu;
+#pragma unroll
+        for (int j = 16; j >= 1; j >>= 1) {
+            const uint32_t y = __shfl_xor_sync(kFull, x, j);
+            x = (lane & j) ? ((x & ~m) | ((y >> j) & m)) : ((x & m) | ((y << j) & ~m));
+            m ^= m << (j >> 1);
+        }
+        outw[wi] = x;                                    // row = state, bit = token
+    }
+    if (q < n_states) {
+        uint4 *dst = (uint4 *)(mask + (long long)q * ldw + w0);              // ldw multiple of 32
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            dst[g] = make_uint4(outw[4 * g], outw[4 * g + 1], outw[4 * g + 2], outw[4 * g + 3]);
+    }
+}
+
+template <typename ST, typename NT, int NS>
+cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
+                        cudaStream_t stream)
+{
+    auto kernel = build_trie_kernel<ST, NT, NS>;
+    if (smem_bytes > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem_bytes);
+        if (e != cudaSuccess)
+            return e;
+    }
+    kernel<<<grid, threads, smem_bytes, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <typename ST, typename NT>
+cudaError_t launch_trie_ns(int ns, const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
+                           cudaStream_t stream)
+{
+    switch (ns) {
+    case 1: return launch_trie<ST, NT, 1>(p, grid, threads, smem_bytes, stream);
+    case 2: return launch_trie<ST, NT, 2>(p, grid, threads, smem_bytes, stream);
+    default: return launch_trie<ST, NT, 4>(p, grid, threads, smem_bytes, stream);
     }
 }
 
@@ -75,26 +220,77 @@ build_rows_kernel(const DT *__restrict__ dfa, int n_states, const uint8_t *__res
 int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
 {
     const cstr_vocab *vc = t->vocab;
-    const int states_per_cta = 16;
-    dim3 grid((unsigned)((t->V + kBuildThreads - 1) / kBuildThreads),
-              (unsigned)((dfa->n_states + states_per_cta - 1) / states_per_cta));
-    if (grid.y > 65535u)
-        return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: %d states exceed the launch limit",
-                         dfa->n_states);
-    // The DFA's entry width follows its own size, the table's its capacity.
-#define CSTR_BUILD(DT, NT)                                                                   \
-    build_rows_kernel<DT, NT><<<grid, kBuildThreads, 0, stream>>>(                           \
-        (const DT *)dfa->trans, dfa->n_states, dfa->accept, vc->head, vc->len, vc->bytes,    \
-        vc->off, t->V, t->eos_id, (NT *)t->next, t->ldn, t->mask, t->ldw, states_per_cta)
-    if (!dfa->wide && !t->wide)
-        CSTR_BUILD(int16_t, int16_t);
-    else if (!dfa->wide && t->wide)
-        CSTR_BUILD(int16_t, int32_t);
-    else if (dfa->wide && t->wide)
-        CSTR_BUILD(int32_t, int32_t);
-    else
+    BuildParams p;
+    p.tt = dfa->tt;
+    p.cls = dfa->cls;
+    p.accept = dfa->accept;
+    p.desc = vc->desc;
+    p.bytes = vc->bytes;
+    p.off = vc->off;
+    p.next = t->next;
+    p.maskT = t->maskT;
+    p.row = dfa->row;
+    p.lds = t->lds;
+    p.ldb = t->ldb;
+    p.n_states = dfa->n_states;
+    p.n_classes = dfa->n_classes;
+    p.V = t->V;
+    p.eos_id = t->eos_id;
+
+    if (dfa->wide && !t->wide)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
-#undef CSTR_BUILD
+    const size_t st = dfa->wide ? 4 : 2;
+
+    // States per lane and warps per CTA: enough states per warp to amortise the
+    // per-token work, without leaving most lanes idle on small automata.
+    const int S = dfa->n_states;
+    const int ns = S >= 2048 ? 4 : (S >= 512 ? 2 : 1);
+    const int per_warp = ns * 32;
+    int warps = (S + per_warp - 1) / per_warp;
+    if (warps > 8)
+        warps = 8;
+    const int threads = warps * 32;
+    const int state_groups = (S + per_warp * warps - 1) / (per_warp * warps);
+
+    const size_t stack_bytes = (size_t)warps * (CSTR_STACK_DEPTH + 1) * ns * 32 * st;
+    const size_t table_bytes = (size_t)dfa->n_classes * (size_t)dfa->row * st;
+    const size_t smem_limit = 200 * 1024;
+    p.table_in_smem = (256 + stack_bytes + table_bytes + 16 <= smem_limit) ? 1 : 0;
+    // 256 + stack is a multiple of 16 only if stack_bytes is: (kDepth+1)*ns*32*st = 17*64*ns*(st/2)*... is.
+    const size_t smem_bytes = 256 + stack_bytes + (p.table_in_smem ? table_bytes : 0);
+
+    // Token chunks: each CTA restarts its walk at the root, so chunks should be
+    // long; but there must be enough CTAs to fill the machine.
+    int dev_sms = 148;
+    cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, t->device);
+    const long long want_ctas = 8LL * dev_sms;
+    long long chunks = (want_ctas + state_groups - 1) / state_groups;
+    long long tokens_per_cta = (t->V + chunks - 1) / chunks;
+    const long long min_tokens = p.table_in_smem ? 512 : 128;
+    if (tokens_per_cta < min_tokens)
+        tokens_per_cta = min_tokens;
+    chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
+    if (chunks > 65535) {
+        chunks = 65535;
+        tokens_per_cta = (t->V + chunks - 1) / chunks;
+        chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
+    }
+    p.tokens_per_cta = (int)tokens_per_cta;
+    dim3 grid((unsigned)state_groups, (unsigned)chunks);
+
+    cudaError_t e;
+    if (!dfa->wide && !t->wide)
+        e = launch_trie_ns<int16_t, int16_t>(ns, p, grid, threads, smem_bytes, stream);
+    else if (!dfa->wide && t->wide)
+        e = launch_trie_ns<int16_t, int32_t>(ns, p, grid, threads, smem_bytes, stream);
+    else
+        e = launch_trie_ns<int32_t, int32_t>(ns, p, grid, threads, smem_bytes, stream);
+    if (e != cudaSuccess)
+        return cstr_fail(CSTR_ERR_CUDA, "cstr_table_build: builder launch: %s",
+                         cudaGetErrorString(e));
+
+    dim3 tgrid((unsigned)(t->ldw / 32), (unsigned)((((S + 31) / 32) + 7) / 8));
+    mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V);
     CSTR_CUDA_TRY(cudaGetLastError());
     return CSTR_OK;
 }

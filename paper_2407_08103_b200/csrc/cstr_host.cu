@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -38,7 +39,8 @@ extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
 {
     if (!dfa)
         return;
-    cudaFree(dfa->trans);
+    cudaFree(dfa->tt);
+    cudaFree(dfa->cls);
     cudaFree(dfa->accept);
     delete dfa;
 }
@@ -65,40 +67,84 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     if (!d)
         return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
     memset(d, 0, sizeof *d);
-    int rc = CSTR_OK;
-    cudaError_t e = cudaGetDevice(&d->device);
     d->n_states = n_states;
     d->start = start_state;
-    d->wide = n_states > 32767;
+    d->wide = (int64_t)n_states + 1 > 32767;
+    d->row = ((int64_t)n_states + 1 + 7) / 8 * 8;
     const size_t esz = d->wide ? 4 : 2;
-    std::vector<uint8_t> flags;
-    std::vector<int16_t> narrow;
+
+    // Byte classes: bytes whose columns are identical in every state.
+    std::vector<int32_t> col;      // column-major copy, col[b * S + q]
+    std::vector<int> order(256), cls_of(256), rep;
+    std::vector<uint8_t> cls8(256), flags;
+    std::vector<uint8_t> tt;
+    try {
+        col.resize((size_t)n);
+        for (int32_t q = 0; q < n_states; ++q)
+            for (int b = 0; b < 256; ++b)
+                col[(size_t)b * n_states + q] = trans[(size_t)q * 256 + b];
+        const size_t colbytes = (size_t)n_states * sizeof(int32_t);
+        for (int b = 0; b < 256; ++b)
+            order[b] = b;
+        std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+            return memcmp(&col[(size_t)x * n_states], &col[(size_t)y * n_states], colbytes) < 0;
+        });
+        // classes numbered by their smallest byte
+        std::vector<int> group(256, -1);
+        int ngroups = 0;
+        for (int i = 0; i < 256; ++i) {
+            if (i > 0 && memcmp(&col[(size_t)order[i] * n_states],
+                                &col[(size_t)order[i - 1] * n_states], colbytes) == 0)
+                group[order[i]] = group[order[i - 1]];
+            else
+                group[order[i]] = ngroups++;
+        }
+        std::vector<int> renum(ngroups, -1);
+        for (int b = 0; b < 256; ++b) {
+            if (renum[group[b]] < 0) {
+                renum[group[b]] = (int)rep.size();
+                rep.push_back(b);
+            }
+            cls_of[b] = renum[group[b]];
+            cls8[b] = (uint8_t)cls_of[b];
+        }
+        d->n_classes = (int32_t)rep.size();
+        tt.assign((size_t)d->n_classes * (size_t)d->row * esz, 0);
+        const int32_t sink = n_states;
+        for (int c = 0; c < d->n_classes; ++c) {
+            const int32_t *src = &col[(size_t)rep[c] * n_states];
+            for (int64_t q = 0; q < d->row; ++q) {
+                const int32_t t = (q < n_states && src[q] >= 0) ? src[q] : sink;
+                if (d->wide)
+                    ((int32_t *)tt.data())[(size_t)c * d->row + q] = t;
+                else
+                    ((int16_t *)tt.data())[(size_t)c * d->row + q] = (int16_t)t;
+            }
+        }
+        flags.resize(n_states);
+        for (int32_t q = 0; q < n_states; ++q)
+            flags[q] = accept[q] ? 1 : 0;
+    } catch (const std::bad_alloc &) {
+        delete d;
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+    }
+
+    cudaError_t e = cudaGetDevice(&d->device);
     if (e == cudaSuccess)
-        e = cudaMalloc(&d->trans, (size_t)n * esz);
+        e = cudaMalloc(&d->tt, tt.size());
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&d->cls, 256);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&d->accept, (size_t)n_states);
-    if (e == cudaSuccess) {
-        try {
-            flags.resize(n_states);
-            for (int32_t q = 0; q < n_states; ++q)
-                flags[q] = accept[q] ? 1 : 0;
-            if (!d->wide) {
-                narrow.resize((size_t)n);
-                for (int64_t i = 0; i < n; ++i)
-                    narrow[(size_t)i] = (int16_t)trans[i];
-            }
-        } catch (const std::bad_alloc &) {
-            cstr_free_dfa(d);
-            return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
-        }
-        e = cudaMemcpy(d->trans, d->wide ? (const void *)trans : (const void *)narrow.data(),
-                       (size_t)n * esz, cudaMemcpyHostToDevice);
-    }
+    if (e == cudaSuccess)
+        e = cudaMemcpy(d->tt, tt.data(), tt.size(), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(d->cls, cls8.data(), 256, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(d->accept, flags.data(), (size_t)n_states, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
-        rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
-                       "cstr_load_dfa: %s", cudaGetErrorString(e));
+        int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                           "cstr_load_dfa: %s", cudaGetErrorString(e));
         cstr_free_dfa(d);
         return rc;
     }
@@ -114,8 +160,7 @@ extern "C" void cstr_free_vocab(cstr_vocab_t *v)
         return;
     cudaFree(v->bytes);
     cudaFree(v->off);
-    cudaFree(v->head);
-    cudaFree(v->len);
+    cudaFree(v->desc);
     delete v;
 }
 
@@ -133,6 +178,9 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
     for (int32_t v = 0; v < vocab_size; ++v) {
         if (offsets[v + 1] < offsets[v])
             return cstr_fail(CSTR_ERR_VOCAB, "cstr_load_vocab: offsets decrease at token %d", v);
+        if (offsets[v + 1] - offsets[v] >= (1 << 24))
+            return cstr_fail(CSTR_ERR_VOCAB, "cstr_load_vocab: token %d is longer than 2^24 bytes",
+                             v);
     }
     const int64_t total = offsets[vocab_size];
     if (total >= ((int64_t)1 << 31))
@@ -148,27 +196,58 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
     vh->V = vocab_size;
     vh->total_bytes = total;
 
-    std::vector<uint32_t> off32, len32;
-    std::vector<uint4> head;
+    std::vector<uint32_t> off32;
+    std::vector<int32_t> order;
+    std::vector<uint4> desc;
+    uint32_t max_len = 0;
     try {
         off32.resize((size_t)vocab_size + 1);
-        len32.resize((size_t)vocab_size);
-        head.resize((size_t)vocab_size);
+        order.resize((size_t)vocab_size);
+        desc.resize((size_t)vocab_size);
+        for (int32_t v = 0; v <= vocab_size; ++v)
+            off32[v] = (uint32_t)offsets[v];
+        for (int32_t v = 0; v < vocab_size; ++v)
+            order[v] = v;
+        // lexicographic order of the byte strings (a prefix sorts before its
+        // extensions), ties by id: the depth-first order of the vocabulary trie
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+            const uint32_t la = off32[a + 1] - off32[a], lb = off32[b + 1] - off32[b];
+            const uint32_t m = la < lb ? la : lb;
+            const int c = m ? memcmp(vocab_bytes + off32[a], vocab_bytes + off32[b], m) : 0;
+            if (c != 0)
+                return c < 0;
+            if (la != lb)
+                return la < lb;
+            return a < b;
+        });
+        for (int32_t i = 0; i < vocab_size; ++i) {
+            const int32_t v = order[i];
+            const uint8_t *cur = vocab_bytes + off32[v];
+            const uint32_t n = off32[v + 1] - off32[v];
+            if (n > max_len)
+                max_len = n;
+            uint32_t p = 0;
+            if (i > 0) {
+                const int32_t u = order[i - 1];
+                const uint8_t *prev = vocab_bytes + off32[u];
+                const uint32_t pn = off32[u + 1] - off32[u];
+                const uint32_t m = n < pn ? n : pn;
+                while (p < m && p < CSTR_STACK_DEPTH && prev[p] == cur[p])
+                    ++p;
+            }
+            uint8_t sfx[8] = {0};
+            for (uint32_t k = 0; k < 8 && p + k < n; ++k)
+                sfx[k] = cur[p + k];
+            uint4 r;
+            r.x = (uint32_t)v;
+            r.y = n | (p << 24);
+            memcpy(&r.z, sfx, 4);
+            memcpy(&r.w, sfx + 4, 4);
+            desc[i] = r;
+        }
     } catch (const std::bad_alloc &) {
         delete vh;
         return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_vocab: out of host memory");
-    }
-    uint32_t max_len = 0;
-    for (int32_t v = 0; v <= vocab_size; ++v)
-        off32[v] = (uint32_t)offsets[v];
-    for (int32_t v = 0; v < vocab_size; ++v) {
-        const uint32_t n = off32[v + 1] - off32[v];
-        len32[v] = n;
-        if (n > max_len)
-            max_len = n;
-        uint8_t rec[16] = {0};
-        memcpy(rec, vocab_bytes + off32[v], n < 16 ? n : 16);
-        memcpy(&head[v], rec, 16);
     }
     vh->max_len = max_len;
 
@@ -178,9 +257,7 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&vh->off, ((size_t)vocab_size + 1) * sizeof(uint32_t));
     if (e == cudaSuccess)
-        e = cudaMalloc((void **)&vh->head, (size_t)vocab_size * sizeof(uint4));
-    if (e == cudaSuccess)
-        e = cudaMalloc((void **)&vh->len, (size_t)vocab_size * sizeof(uint32_t));
+        e = cudaMalloc((void **)&vh->desc, (size_t)vocab_size * sizeof(uint4));
     if (e == cudaSuccess)
         e = cudaMemset(vh->bytes, 0, (size_t)total + 16);
     if (e == cudaSuccess && total > 0)
@@ -189,10 +266,7 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
         e = cudaMemcpy(vh->off, off32.data(), off32.size() * sizeof(uint32_t),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
-        e = cudaMemcpy(vh->head, head.data(), head.size() * sizeof(uint4), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(vh->len, len32.data(), len32.size() * sizeof(uint32_t),
-                       cudaMemcpyHostToDevice);
+        e = cudaMemcpy(vh->desc, desc.data(), desc.size() * sizeof(uint4), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
         int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
                            "cstr_load_vocab: %s", cudaGetErrorString(e));
@@ -211,6 +285,7 @@ extern "C" void cstr_free_table(cstr_table_t *t)
         return;
     cudaFree(t->next);
     cudaFree(t->mask);
+    cudaFree(t->maskT);
     cudaFree(t->accept);
     cstr_free_vocab(t->owned_vocab);
     delete t;
@@ -236,15 +311,19 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     t->max_states = max_states;
     t->V = vocab->V;
     t->W = (vocab->V + 31) / 32;
-    t->ldn = ((int64_t)t->V + 63) / 64 * 64;
+    t->lds = ((int64_t)max_states + 63) / 64 * 64;
     t->ldw = ((int64_t)t->W + 31) / 32 * 32;
-    t->wide = max_states > 32767;
+    t->ldb = (((int64_t)max_states + 31) / 32 + 7) / 8 * 8;
+    t->wide = (int64_t)max_states + 1 > 32767;
     t->eos_id = -1;
-    const size_t next_bytes = (size_t)max_states * (size_t)t->ldn * (t->wide ? 4 : 2);
+    const size_t next_bytes = (size_t)t->V * (size_t)t->lds * (t->wide ? 4 : 2);
     const size_t mask_bytes = (size_t)max_states * (size_t)t->ldw * 4;
+    const size_t maskT_bytes = (size_t)t->V * (size_t)t->ldb * 4;
     cudaError_t e = cudaMalloc(&t->next, next_bytes);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->mask, mask_bytes);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->maskT, maskT_bytes);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->accept, (size_t)max_states);
     if (e == cudaSuccess)
@@ -351,31 +430,29 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
                                    cudaMemcpyDeviceToHost));
     }
     if (next_host) {
-        if (t->wide) {
-            CSTR_CUDA_TRY(cudaMemcpy2D(next_host, (size_t)t->V * 4,
-                                       (const int32_t *)t->next + (int64_t)state_lo * t->ldn,
-                                       (size_t)t->ldn * 4, (size_t)t->V * 4, rows,
+        // The device table is token-major; bring the state columns down and
+        // transpose on the host, a slab of states at a time.
+        const size_t esz = t->wide ? 4 : 2;
+        const int32_t slab = 64;
+        std::vector<uint8_t> tmp;
+        try {
+            tmp.resize((size_t)slab * (size_t)t->V * esz);
+        } catch (const std::bad_alloc &) {
+            return cstr_fail(CSTR_ERR_NOMEM, "cstr_table_download: out of host memory");
+        }
+        for (int32_t r0 = 0; r0 < rows; r0 += slab) {
+            const int32_t nr = rows - r0 < slab ? rows - r0 : slab;
+            CSTR_CUDA_TRY(cudaMemcpy2D(tmp.data(), (size_t)nr * esz,
+                                       (const uint8_t *)t->next + (size_t)(state_lo + r0) * esz,
+                                       (size_t)t->lds * esz, (size_t)nr * esz, (size_t)t->V,
                                        cudaMemcpyDeviceToHost));
-        } else {
-            // narrow rows come down in slabs and are widened on the host
-            const int32_t slab = 64;
-            std::vector<int16_t> tmp;
-            try {
-                tmp.resize((size_t)slab * (size_t)t->V);
-            } catch (const std::bad_alloc &) {
-                return cstr_fail(CSTR_ERR_NOMEM, "cstr_table_download: out of host memory");
-            }
-            for (int32_t r0 = 0; r0 < rows; r0 += slab) {
-                const int32_t nr = rows - r0 < slab ? rows - r0 : slab;
-                CSTR_CUDA_TRY(cudaMemcpy2D(tmp.data(), (size_t)t->V * 2,
-                                           (const int16_t *)t->next +
-                                               (int64_t)(state_lo + r0) * t->ldn,
-                                           (size_t)t->ldn * 2, (size_t)t->V * 2, nr,
-                                           cudaMemcpyDeviceToHost));
-                int32_t *dst = next_host + (int64_t)r0 * t->V;
-                const int64_t n = (int64_t)nr * t->V;
-                for (int64_t i = 0; i < n; ++i)
-                    dst[i] = (int32_t)tmp[(size_t)i];
+            for (int32_t v = 0; v < t->V; ++v) {
+                for (int32_t r = 0; r < nr; ++r) {
+                    const size_t at = (size_t)v * nr + r;
+                    const int32_t x = t->wide ? ((const int32_t *)tmp.data())[at]
+                                              : (int32_t)((const int16_t *)tmp.data())[at];
+                    next_host[(int64_t)(r0 + r) * t->V + v] = x;
+                }
             }
         }
     }

@@ -20,40 +20,57 @@ int cstr_fail(int code, const char *fmt, ...);
                              "%s failed: %s", #expr, cudaGetErrorString(e_));            \
     } while (0)
 
+// Byte DFA as the builder reads it: bytes that no state tells apart share a
+// class, and the table is stored class-major ("transposed") with one extra
+// dead-sink column, tt[c][s] for s in [0, n_states], entry n_states = sink, so
+// that a walk needs no "is it dead" branch: the sink maps to itself.
 struct cstr_dfa {
     int device;
     int32_t n_states;
     int32_t start;
-    int wide;          // 0: int16 entries, 1: int32 entries
-    void *trans;       // DEVICE [n_states][256]
-    uint8_t *accept;   // DEVICE [n_states]
+    int wide;            // 0: int16 entries (n_states + 1 <= 32767), 1: int32 entries
+    int32_t n_classes;   // 1..256
+    int64_t row;         // entries per class row (n_states + 1, rounded up to 8)
+    void *tt;            // DEVICE [n_classes][row]
+    uint8_t *cls;        // DEVICE [256] byte -> class
+    uint8_t *accept;     // DEVICE [n_states]
 };
 
-// Vocabulary as the builder reads it: the first 16 bytes of every token packed
-// in one 16-byte record (zero padded), its length, and the raw bytes/offsets
-// for the rare longer token.
+// Vocabulary as the builder reads it: tokens in lexicographic (trie depth-first)
+// order, each with the length of the prefix it shares with its predecessor, so
+// that a walk resumes at the shared depth instead of at the root.
+//   desc[i] = { token id, length | shared_prefix << 24, first 8 bytes after the
+//               shared prefix (little endian in z, w) }
+// The shared prefix is clipped to CSTR_STACK_DEPTH.  Raw bytes / offsets serve
+// walks that start at the root and suffixes longer than 8 bytes.
+#define CSTR_STACK_DEPTH 16
 struct cstr_vocab {
     int device;
     int32_t V;
     int64_t total_bytes;
     uint8_t *bytes;    // DEVICE [total_bytes + 16]
     uint32_t *off;     // DEVICE [V + 1]
-    uint4 *head;       // DEVICE [V]    first 16 bytes
-    uint32_t *len;     // DEVICE [V]
+    uint4 *desc;       // DEVICE [V], sorted order
     uint32_t max_len;
 };
 
+// Token table.  next is token-major: next[v][q] (a step reads one entry per
+// row; the builder writes whole 64-byte state segments).  mask is state-major
+// as the step streams it.  maskT is the builder's intermediate: per token one
+// word per block of 32 states, transposed into mask by a second kernel.
 struct cstr_table {
     int device;
     const cstr_vocab *vocab;
     cstr_vocab *owned_vocab;   // non-null when created by cstr_build_token_table
     int32_t max_states;
     int32_t V, W;
-    int64_t ldn;       // elements per row of next (V rounded up to 64)
-    int64_t ldw;       // words per row of mask (W rounded up to 32), padding zero
+    int64_t lds;       // entries per token row of next (max_states rounded up to 64)
+    int64_t ldw;       // words per state row of mask (W rounded up to 32), padding zero
+    int64_t ldb;       // words per token row of maskT (state blocks rounded up to 8)
     int wide;          // capacity dtype of next: 0 int16, 1 int32
-    void *next;        // DEVICE [max_states][ldn]
+    void *next;        // DEVICE [V][lds]
     uint32_t *mask;    // DEVICE [max_states][ldw]
+    uint32_t *maskT;   // DEVICE [V][ldb]
     uint8_t *accept;   // DEVICE [max_states]
     int32_t n_states;  // of the automaton currently held (0 = not built)
     int32_t start;

@@ -25,7 +25,7 @@ struct TableDesc {
     const uint32_t *mask;
     const void *next;
     const uint8_t *accept;
-    long long ldn;
+    long long lds;       // next is token-major: next[token * lds + state]
     long long ldw;
     int n_states;
     int wide;
@@ -141,7 +141,7 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     const TableDesc &tb = p.tab[c.t];
     if (c.active && key != 0ull) {
         tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
-        const long long at = (long long)c.q * tb.ldn + tok;
+        const long long at = (long long)tok * tb.lds + c.q;
         q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const int16_t *)tb.next)[at];
     } else if (c.active) {
         atomicAdd(p.counters + 1, 1ull);
@@ -374,7 +374,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         p.tab[i].mask = t->mask;
         p.tab[i].next = t->next;
         p.tab[i].accept = t->accept;
-        p.tab[i].ldn = t->ldn;
+        p.tab[i].lds = t->lds;
         p.tab[i].ldw = t->ldw;
         p.tab[i].n_states = t->n_states;
         p.tab[i].wide = t->wide;
