@@ -35,119 +35,146 @@ struct BuildParams {
     const uint32_t *off;       // [V + 1]
     void *next;                // [V][lds]
     uint32_t *maskT;           // [V][ldb]
-    long long row, lds, ldb;
+    long long lds, ldb;
+    int row;                   // entries per class row of tt
     int n_states, n_classes, V, eos_id;
     int tokens_per_cta;
-    int table_in_smem;
 };
 
-// ST: entry type of the DFA table; NT: entry type of next; NS: states per lane.
-template <typename ST, typename NT, int NS>
+// NS consecutive entries moved as one aligned unit (one vector load / store).
+template <typename T, int NS>
+struct alignas(sizeof(T) * NS) Pack {
+    T v[NS];
+};
+
+// ST: entry type of the DFA table; NT: entry type of next; NS: states per lane;
+// SMEM: the class-major DFA table is staged in shared memory.
+// Lane l of the warp that owns states [q0, q0 + 32 NS) holds the NS consecutive
+// states q0 + NS l + j.  Ballot j therefore carries state q0 + NS l + j in bit l;
+// it is stored as word (q0 / 32 + j) of the token's maskT row and un-permuted
+// by the transpose kernel.
+template <typename ST, typename NT, int NS, bool SMEM>
 __global__ void __launch_bounds__(256)
 build_trie_kernel(const __grid_constant__ BuildParams p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    typedef Pack<ST, NS> SPack;
+    typedef Pack<NT, NS> NPack;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int sink = p.n_states;
 
-    // shared memory: [class map 256 B][stack: nwarps x (kDepth+1) x NS x 32 ST][table]
-    uint8_t *s_cls = smem;
-    ST *s_stack = (ST *)(smem + 256) + (size_t)warp * (kDepth + 1) * NS * 32;
-    ST *s_tt = (ST *)(smem + 256) + (size_t)nwarps * (kDepth + 1) * NS * 32;
+    // shared memory: [row offset per byte: 256 x u32][stack: nwarps x (kDepth+1) x 32 SPack][table]
+    uint32_t *s_rowoff = (uint32_t *)smem;
+    SPack *s_stack = (SPack *)(smem + 1024) + (size_t)warp * (kDepth + 1) * 32 + lane;
+    ST *s_tt = (ST *)(smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack));
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
-        s_cls[i] = p.cls[i];
-    const ST *tt = (const ST *)p.tt;
-    if (p.table_in_smem) {
-        const long long n16 = (long long)p.n_classes * p.row * (long long)sizeof(ST) / 16;
+        s_rowoff[i] = (uint32_t)p.cls[i] * (uint32_t)p.row;
+    if (SMEM) {
+        const int n16 = (int)((long long)p.n_classes * p.row * (long long)sizeof(ST) / 16);
         const uint4 *src = (const uint4 *)p.tt;
         uint4 *dst = (uint4 *)s_tt;      // row is a multiple of 8 entries: whole 16-byte units
-        for (long long i = threadIdx.x; i < n16; i += blockDim.x)
+        for (int i = threadIdx.x; i < n16; i += blockDim.x)
             dst[i] = __ldg(src + i);
-        tt = s_tt;
     }
     __syncthreads();
+    const ST *g_tt = (const ST *)p.tt;
 
     const int q0 = (blockIdx.x * nwarps + warp) * NS * 32;
     if (q0 >= p.n_states)
         return;                                          // whole warp out of range
-    int q[NS];
-    bool in_range[NS], acc[NS];
+    const int qbase = q0 + NS * lane;
+    int cur[NS];
+    unsigned accbits = 0, inbits = 0;
+    SPack root;
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
-        q[j] = q0 + j * 32 + lane;
-        in_range[j] = q[j] < p.n_states;
-        acc[j] = in_range[j] && p.accept[q[j]] != 0;
-        s_stack[(0 * NS + j) * 32 + lane] = (ST)(in_range[j] ? q[j] : sink);
+        const bool in = qbase + j < p.n_states;
+        inbits |= (unsigned)in << j;
+        accbits |= (unsigned)(in && p.accept[qbase + j] != 0) << j;
+        cur[j] = in ? qbase + j : sink;
+        root.v[j] = (ST)cur[j];
     }
+    s_stack[0] = root;
     __syncwarp();
 
     const int t_begin = blockIdx.y * p.tokens_per_cta;
     const int t_end = min(p.V, t_begin + p.tokens_per_cta);
-    int cur[NS];
-#pragma unroll
-    for (int j = 0; j < NS; ++j)
-        cur[j] = in_range[j] ? q[j] : sink;
     int depth = 0;                                       // depth of the path held in cur[]
-    NT *next = (NT *)p.next;
+    NPack outv;
+    uint32_t words[NS];
+    bool prev_eos = true;                                // forces the first token's outputs
 
+    uint4 d_next = __ldg(p.desc + t_begin);              // same address in every lane
     for (int i = t_begin; i < t_end; ++i) {
-        const uint4 d = __ldg(p.desc + i);               // same address in every lane
+        const uint4 d = d_next;
+        if (i + 1 < t_end)
+            d_next = __ldg(p.desc + i + 1);
         const int tok = (int)d.x;
         const int n = (int)(d.y & 0xffffffu);
-        const int shared = (i == t_begin) ? 0 : (int)(d.y >> 24);
+        const bool first = (i == t_begin);
+        const int shared = first ? 0 : (int)(d.y >> 24);
         if (shared < depth) {                            // climb back to the shared prefix
+            const SPack at = s_stack[shared * 32];
 #pragma unroll
             for (int j = 0; j < NS; ++j)
-                cur[j] = (int)s_stack[(shared * NS + j) * 32 + lane];
+                cur[j] = (int)at.v[j];
         }
-        const bool inline_ok = (i != t_begin);           // d.z / d.w hold bytes shared..shared+7
-        const uint32_t begin = inline_ok ? 0u : __ldg(p.off + tok);
         for (int k = shared; k < n; ++k) {
             uint32_t b;
             const int r = k - shared;
-            if (inline_ok && r < 8)
-                b = ((r < 4 ? d.z : d.w) >> (8 * (r & 3))) & 0xffu;
+            if (!first && r < 8)
+                b = ((r < 4 ? d.z : d.w) >> (8 * (r & 3))) & 0xffu;   // bytes shared .. shared+7
             else
-                b = __ldg(p.bytes + (inline_ok ? __ldg(p.off + tok) : begin) + k);
-            const ST *rowp = tt + (long long)s_cls[b] * p.row;
+                b = __ldg(p.bytes + __ldg(p.off + tok) + k);
+            const uint32_t ro = s_rowoff[b];
+            SPack at;
 #pragma unroll
-            for (int j = 0; j < NS; ++j)
-                cur[j] = (int)rowp[cur[j]];
-            if (k + 1 <= kDepth) {
-#pragma unroll
-                for (int j = 0; j < NS; ++j)
-                    s_stack[((k + 1) * NS + j) * 32 + lane] = (ST)cur[j];
+            for (int j = 0; j < NS; ++j) {
+                cur[j] = SMEM ? (int)s_tt[ro + (uint32_t)cur[j]]
+                              : (int)__ldg(g_tt + ro + (uint32_t)cur[j]);
+                at.v[j] = (ST)cur[j];
             }
+            if (k < kDepth)
+                s_stack[(k + 1) * 32] = at;
         }
         depth = n;
         const bool is_eos = tok == p.eos_id;
+        // A token with no byte of its own equals its predecessor: same outputs.
+        if (n != shared || first || is_eos || prev_eos) {
 #pragma unroll
-        for (int j = 0; j < NS; ++j) {
-            int s = (n > 0 && cur[j] != sink) ? cur[j] : CSTR_DEAD;
-            bool allowed = s >= 0;
-            if (is_eos) {                // allowed exactly in accepting states; finishes the row
-                allowed = acc[j];
-                s = CSTR_DEAD;
+            for (int j = 0; j < NS; ++j) {
+                int s = (n > 0 && cur[j] != sink) ? cur[j] : CSTR_DEAD;
+                bool allowed = s >= 0;
+                if (is_eos) {            // allowed exactly in accepting states; finishes the row
+                    allowed = (accbits >> j) & 1u;
+                    s = CSTR_DEAD;
+                }
+                words[j] = __ballot_sync(kFull, allowed && ((inbits >> j) & 1u));
+                outv.v[j] = (NT)s;
             }
-            const uint32_t word = __ballot_sync(kFull, allowed && in_range[j]);
-            const int qb = q0 + j * 32;
-            if (qb < p.n_states) {
-                if (in_range[j])
-                    next[(long long)tok * p.lds + q[j]] = (NT)s;
-                if (lane == 0)
-                    p.maskT[(long long)tok * p.ldb + (qb >> 5)] = word;
-            }
+        }
+        prev_eos = is_eos;
+        NT *nrow = (NT *)p.next + (long long)tok * p.lds + qbase;
+        *(NPack *)nrow = outv;                           // lds is a multiple of 128: in bounds
+        if (lane < NS) {                                 // (q0 >> 5) + NS <= lds / 32 < ldb
+            uint32_t mine = words[0];
+#pragma unroll
+            for (int j = 1; j < NS; ++j)
+                mine = (lane == j) ? words[j] : mine;
+            p.maskT[(long long)tok * p.ldb + (q0 >> 5) + lane] = mine;
         }
     }
 }
 
-// mask[q][w] bit t = maskT[32 w + t][q / 32] bit (q % 32): 32 x 32 bit-matrix
-// transposes.  A CTA takes 1,024 tokens (32 mask words) x 8 state blocks; warp j
-// transposes the 32 tiles of state block j and each lane writes the 32
-// consecutive words of its state row (128 bytes).
+// mask[q][w] bit t = validity of token 32 w + t in state q, gathered from the
+// per-token ballot words: 32 x 32 bit-matrix transposes.  A CTA takes 1,024
+// tokens (32 mask words) x 8 ballot words; warp j transposes the 32 tiles of
+// ballot word sb0 + j and each lane writes the 32 consecutive words of its
+// state row (128 bytes).  Ballot word k of a block of 32 NS states holds state
+// NS l + k of the block in bit l.
 __global__ void __launch_bounds__(256)
 mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
-                      long long ldw, int n_states, int V)
+                      long long ldw, int n_states, int V, int ns)
 {
     __shared__ uint32_t tile[8][1024];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -165,13 +192,15 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
         tile[4][t] = b.x; tile[5][t] = b.y; tile[6][t] = b.z; tile[7][t] = b.w;
     }
     __syncthreads();
-    const int q = (sb0 + warp) * 32 + lane;
-    if ((sb0 + warp) * 32 >= n_states)
+    const int sbw = sb0 + warp;
+    const int first_state = (sbw / ns) * (ns * 32) + (sbw % ns);
+    if (first_state >= n_states)
         return;
+    const int q = first_state + ns * lane;
     uint32_t outw[32];
 #pragma unroll
     for (int wi = 0; wi < 32; ++wi) {
-        uint32_t x = tile[warp][wi * 32 + lane];         // row = token, bit = state
+        uint32_t x = tile[warp][wi * 32 + lane];         // row = token, bit = state slot
         uint32_t m = 0x0000ffffu;
 #pragma unroll
         for (int j = 16; j >= 1; j >>= 1) {
@@ -179,7 +208,7 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
             x = (lane & j) ? ((x & ~m) | ((y >> j) & m)) : ((x & m) | ((y << j) & ~m));
             m ^= m << (j >> 1);
         }
-        outw[wi] = x;                                    // row = state, bit = token
+        outw[wi] = x;                                    // row = state slot, bit = token
     }
     if (q < n_states) {
         uint4 *dst = (uint4 *)(mask + (long long)q * ldw + w0);              // ldw multiple of 32
@@ -189,11 +218,11 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
     }
 }
 
-template <typename ST, typename NT, int NS>
+template <typename ST, typename NT, int NS, bool SMEM>
 cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
                         cudaStream_t stream)
 {
-    auto kernel = build_trie_kernel<ST, NT, NS>;
+    auto kernel = build_trie_kernel<ST, NT, NS, SMEM>;
     if (smem_bytes > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem_bytes);
@@ -205,14 +234,18 @@ cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t sme
 }
 
 template <typename ST, typename NT>
-cudaError_t launch_trie_ns(int ns, const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
-                           cudaStream_t stream)
+cudaError_t launch_trie_ns(int ns, bool in_smem, const BuildParams &p, dim3 grid, int threads,
+                           size_t smem_bytes, cudaStream_t stream)
 {
+#define CSTR_CASE(N)                                                                          \
+    return in_smem ? launch_trie<ST, NT, N, true>(p, grid, threads, smem_bytes, stream)       \
+                   : launch_trie<ST, NT, N, false>(p, grid, threads, smem_bytes, stream)
     switch (ns) {
-    case 1: return launch_trie<ST, NT, 1>(p, grid, threads, smem_bytes, stream);
-    case 2: return launch_trie<ST, NT, 2>(p, grid, threads, smem_bytes, stream);
-    default: return launch_trie<ST, NT, 4>(p, grid, threads, smem_bytes, stream);
+    case 1: CSTR_CASE(1);
+    case 2: CSTR_CASE(2);
+    default: CSTR_CASE(4);
     }
+#undef CSTR_CASE
 }
 
 }  // namespace
@@ -229,7 +262,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     p.off = vc->off;
     p.next = t->next;
     p.maskT = t->maskT;
-    p.row = dfa->row;
+    p.row = (int)dfa->row;
     p.lds = t->lds;
     p.ldb = t->ldb;
     p.n_states = dfa->n_states;
@@ -252,12 +285,11 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     const int threads = warps * 32;
     const int state_groups = (S + per_warp * warps - 1) / (per_warp * warps);
 
-    const size_t stack_bytes = (size_t)warps * (CSTR_STACK_DEPTH + 1) * ns * 32 * st;
+    const size_t stack_bytes = (size_t)warps * (CSTR_STACK_DEPTH + 1) * ns * 32 * st;   // x16 bytes
     const size_t table_bytes = (size_t)dfa->n_classes * (size_t)dfa->row * st;
     const size_t smem_limit = 200 * 1024;
-    p.table_in_smem = (256 + stack_bytes + table_bytes + 16 <= smem_limit) ? 1 : 0;
-    // 256 + stack is a multiple of 16 only if stack_bytes is: (kDepth+1)*ns*32*st = 17*64*ns*(st/2)*... is.
-    const size_t smem_bytes = 256 + stack_bytes + (p.table_in_smem ? table_bytes : 0);
+    const bool in_smem = 1024 + stack_bytes + table_bytes <= smem_limit;
+    const size_t smem_bytes = 1024 + stack_bytes + (in_smem ? table_bytes : 0);
 
     // Token chunks: each CTA restarts its walk at the root, so chunks should be
     // long; but there must be enough CTAs to fill the machine.
@@ -266,7 +298,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     const long long want_ctas = 8LL * dev_sms;
     long long chunks = (want_ctas + state_groups - 1) / state_groups;
     long long tokens_per_cta = (t->V + chunks - 1) / chunks;
-    const long long min_tokens = p.table_in_smem ? 512 : 128;
+    const long long min_tokens = in_smem ? 512 : 128;
     if (tokens_per_cta < min_tokens)
         tokens_per_cta = min_tokens;
     chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
@@ -280,17 +312,19 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
 
     cudaError_t e;
     if (!dfa->wide && !t->wide)
-        e = launch_trie_ns<int16_t, int16_t>(ns, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int16_t, int16_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
     else if (!dfa->wide && t->wide)
-        e = launch_trie_ns<int16_t, int32_t>(ns, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int16_t, int32_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
     else
-        e = launch_trie_ns<int32_t, int32_t>(ns, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int32_t, int32_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
     if (e != cudaSuccess)
         return cstr_fail(CSTR_ERR_CUDA, "cstr_table_build: builder launch: %s",
                          cudaGetErrorString(e));
 
-    dim3 tgrid((unsigned)(t->ldw / 32), (unsigned)((((S + 31) / 32) + 7) / 8));
-    mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V);
+    const int ballot_words = ((S + per_warp - 1) / per_warp) * ns;
+    dim3 tgrid((unsigned)(t->ldw / 32), (unsigned)((ballot_words + 7) / 8));
+    mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
+                                                     ns);
     CSTR_CUDA_TRY(cudaGetLastError());
     return CSTR_OK;
 }

@@ -311,9 +311,9 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     t->max_states = max_states;
     t->V = vocab->V;
     t->W = (vocab->V + 31) / 32;
-    t->lds = ((int64_t)max_states + 63) / 64 * 64;
+    t->lds = ((int64_t)max_states + 127) / 128 * 128;
     t->ldw = ((int64_t)t->W + 31) / 32 * 32;
-    t->ldb = (((int64_t)max_states + 31) / 32 + 7) / 8 * 8;
+    t->ldb = t->lds / 32 + 8 - (t->lds / 32) % 8;   // a multiple of 8, above lds / 32
     t->wide = (int64_t)max_states + 1 > 32767;
     t->eos_id = -1;
     const size_t next_bytes = (size_t)t->V * (size_t)t->lds * (t->wide ? 4 : 2);

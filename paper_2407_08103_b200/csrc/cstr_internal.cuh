@@ -64,7 +64,7 @@ struct cstr_table {
     cstr_vocab *owned_vocab;   // non-null when created by cstr_build_token_table
     int32_t max_states;
     int32_t V, W;
-    int64_t lds;       // entries per token row of next (max_states rounded up to 64)
+    int64_t lds;       // entries per token row of next (max_states rounded up to 128)
     int64_t ldw;       // words per state row of mask (W rounded up to 32), padding zero
     int64_t ldb;       // words per token row of maskT (state blocks rounded up to 8)
     int wide;          // capacity dtype of next: 0 int16, 1 int32
