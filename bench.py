@@ -47,7 +47,7 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=12.0,
                     help="CPU time budget of the oracle baseline leg")
     ap.add_argument("--case", default="full", choices=["full", "small"],
-                    help="small: batch 128 and a 2,051-state string-literal DFA over the same "
+                    help="small: batch 128 and a 4,099-state string-literal DFA over the same "
                          "vocabulary (for profiler captures); its numbers are not bench values")
     ap.add_argument("--skip-build-bench", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -73,7 +73,7 @@ def workload_inputs(case: str = "full"):
     if case == "small":
         from synth.regex_frontend import regex_to_dfa
         w = dataclasses.replace(w, batch=128)
-        dfa = regex_to_dfa(w.regex.replace("{0,4096}", "{0,1024}"))
+        dfa = regex_to_dfa(w.regex.replace("{0,4096}", "{0,2048}"))
     else:
         dfa = config_dfas(WORKLOAD)[0]
     return w, dfa, vb, vo

@@ -39,13 +39,56 @@ struct BuildParams {
     int row;                   // entries per class row of tt
     int n_states, n_classes, V, eos_id;
     int tokens_per_cta;
+    int warps_s;               // warps of a CTA that split its states ...
+    int warps_t;               // ... times warps that split its token chunk
 };
 
-// NS consecutive entries moved as one aligned unit (one vector load / store).
-template <typename T, int NS>
-struct alignas(sizeof(T) * NS) Pack {
-    T v[NS];
-};
+// NS consecutive table entries per lane travel as one aligned unit (one vector
+// load / store).  States are handled as unsigned values (entry types are read
+// as uint16 / uint32; "no edge" is all ones), which keeps every conversion a
+// plain bit operation.
+template <int BYTES>
+struct Unit;
+template <> struct Unit<2> { typedef unsigned short type; };
+template <> struct Unit<4> { typedef unsigned int type; };
+template <> struct Unit<8> { typedef uint2 type; };
+template <> struct Unit<16> { typedef uint4 type; };
+
+template <int ESZ, int NS>
+__device__ __forceinline__ typename Unit<ESZ * NS>::type pack_entries(const unsigned (&v)[NS])
+{
+    typename Unit<ESZ * NS>::type u;
+    if constexpr (ESZ == 2) {
+        if constexpr (NS == 1) u = (unsigned short)v[0];
+        if constexpr (NS == 2) u = v[0] | (v[1] << 16);            // values are below 2^16
+        if constexpr (NS == 4) u = make_uint2(v[0] | (v[1] << 16), v[2] | (v[3] << 16));
+        if constexpr (NS == 8) u = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16),
+                                              v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+    } else {
+        if constexpr (NS == 1) u = v[0];
+        if constexpr (NS == 2) u = make_uint2(v[0], v[1]);
+        if constexpr (NS == 4) u = make_uint4(v[0], v[1], v[2], v[3]);
+    }
+    return u;
+}
+
+template <int ESZ, int NS>
+__device__ __forceinline__ void unpack_entries(typename Unit<ESZ * NS>::type u, unsigned (&v)[NS])
+{
+    if constexpr (ESZ == 2) {
+        if constexpr (NS == 1) v[0] = u;
+        if constexpr (NS == 2) { v[0] = u & 0xffffu; v[1] = u >> 16; }
+        if constexpr (NS == 4) { v[0] = u.x & 0xffffu; v[1] = u.x >> 16; v[2] = u.y & 0xffffu; v[3] = u.y >> 16; }
+        if constexpr (NS == 8) {
+            v[0] = u.x & 0xffffu; v[1] = u.x >> 16; v[2] = u.y & 0xffffu; v[3] = u.y >> 16;
+            v[4] = u.z & 0xffffu; v[5] = u.z >> 16; v[6] = u.w & 0xffffu; v[7] = u.w >> 16;
+        }
+    } else {
+        if constexpr (NS == 1) v[0] = u;
+        if constexpr (NS == 2) { v[0] = u.x; v[1] = u.y; }
+        if constexpr (NS == 4) { v[0] = u.x; v[1] = u.y; v[2] = u.z; v[3] = u.w; }
+    }
+}
 
 // ST: entry type of the DFA table; NT: entry type of next; NS: states per lane;
 // SMEM: the class-major DFA table is staged in shared memory.
@@ -54,114 +97,121 @@ struct alignas(sizeof(T) * NS) Pack {
 // it is stored as word (q0 / 32 + j) of the token's maskT row and un-permuted
 // by the transpose kernel.
 template <typename ST, typename NT, int NS, bool SMEM>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 build_trie_kernel(const __grid_constant__ BuildParams p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    typedef Pack<ST, NS> SPack;
-    typedef Pack<NT, NS> NPack;
+    typedef typename Unit<sizeof(ST)>::type SU;                 // unsigned view of a table entry
+    typedef typename Unit<sizeof(ST) * NS>::type SPack;
+    typedef typename Unit<sizeof(NT) * NS>::type NPack;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int sink = p.n_states;
+    const unsigned sink = (unsigned)CSTR_PERM(p.n_states);      // all ids below are permuted
 
     // shared memory: [row offset per byte: 256 x u32][stack: nwarps x (kDepth+1) x 32 SPack][table]
     uint32_t *s_rowoff = (uint32_t *)smem;
     SPack *s_stack = (SPack *)(smem + 1024) + (size_t)warp * (kDepth + 1) * 32 + lane;
-    ST *s_tt = (ST *)(smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack));
+    SU *s_tt = (SU *)(smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack));
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
         s_rowoff[i] = (uint32_t)p.cls[i] * (uint32_t)p.row;
     if (SMEM) {
         const int n16 = (int)((long long)p.n_classes * p.row * (long long)sizeof(ST) / 16);
         const uint4 *src = (const uint4 *)p.tt;
-        uint4 *dst = (uint4 *)s_tt;      // row is a multiple of 8 entries: whole 16-byte units
+        uint4 *dst = (uint4 *)s_tt;      // row is a multiple of 256 entries: whole 16-byte units
         for (int i = threadIdx.x; i < n16; i += blockDim.x)
             dst[i] = __ldg(src + i);
     }
     __syncthreads();
-    const ST *g_tt = (const ST *)p.tt;
+    const SU *g_tt = (const SU *)p.tt;
 
-    const int q0 = (blockIdx.x * nwarps + warp) * NS * 32;
+    const int warp_s = warp % p.warps_s, warp_t = warp / p.warps_s;
+    const int q0 = (blockIdx.x * p.warps_s + warp_s) * NS * 32;
     if (q0 >= p.n_states)
         return;                                          // whole warp out of range
     const int qbase = q0 + NS * lane;
-    int cur[NS];
-    unsigned accbits = 0, inbits = 0;
-    SPack root;
+    unsigned cur[NS];
+    unsigned accbits = 0;
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
         const bool in = qbase + j < p.n_states;
-        inbits |= (unsigned)in << j;
         accbits |= (unsigned)(in && p.accept[qbase + j] != 0) << j;
-        cur[j] = in ? qbase + j : sink;
-        root.v[j] = (ST)cur[j];
+        cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) : sink;
     }
-    s_stack[0] = root;
+    s_stack[0] = pack_entries<sizeof(ST), NS>(cur);
     __syncwarp();
 
-    const int t_begin = blockIdx.y * p.tokens_per_cta;
-    const int t_end = min(p.V, t_begin + p.tokens_per_cta);
+    const int c_begin = blockIdx.y * p.tokens_per_cta;
+    const int c_end = min(p.V, c_begin + p.tokens_per_cta);
+    const int per_t = (c_end - c_begin + p.warps_t - 1) / p.warps_t;
+    const int t_begin = c_begin + warp_t * per_t;
+    const int t_end = min(c_end, t_begin + per_t);
+    if (t_begin >= t_end)
+        return;
     int depth = 0;                                       // depth of the path held in cur[]
-    NPack outv;
+    unsigned outs[NS];
     uint32_t words[NS];
+    NPack outp;
     bool prev_eos = true;                                // forces the first token's outputs
+    NT *const next_lane = (NT *)p.next + qbase;
+    uint32_t *const maskT_lane = p.maskT + (q0 >> 5) + (lane < NS ? lane : 0);
 
     uint4 d_next = __ldg(p.desc + t_begin);              // same address in every lane
     for (int i = t_begin; i < t_end; ++i) {
         const uint4 d = d_next;
         if (i + 1 < t_end)
             d_next = __ldg(p.desc + i + 1);
-        const int tok = (int)d.x;
+        const unsigned tok = d.x;
         const int n = (int)(d.y & 0xffffffu);
         const bool first = (i == t_begin);
         const int shared = first ? 0 : (int)(d.y >> 24);
-        if (shared < depth) {                            // climb back to the shared prefix
-            const SPack at = s_stack[shared * 32];
+        if (shared < depth)                              // climb back to the shared prefix
+            unpack_entries<sizeof(ST), NS>(s_stack[shared * 32], cur);
+        unsigned long long inl = ((unsigned long long)d.w << 32) | d.z;   // bytes shared .. shared+7
+        for (int k = shared; k < n; ++k) {
+            unsigned b;
+            if (!first && k - shared < 8) {
+                b = (unsigned)inl & 0xffu;
+                inl >>= 8;
+            } else {
+                b = __ldg(p.bytes + __ldg(p.off + tok) + k);
+            }
+            const uint32_t ro = s_rowoff[b];
 #pragma unroll
             for (int j = 0; j < NS; ++j)
-                cur[j] = (int)at.v[j];
-        }
-        for (int k = shared; k < n; ++k) {
-            uint32_t b;
-            const int r = k - shared;
-            if (!first && r < 8)
-                b = ((r < 4 ? d.z : d.w) >> (8 * (r & 3))) & 0xffu;   // bytes shared .. shared+7
-            else
-                b = __ldg(p.bytes + __ldg(p.off + tok) + k);
-            const uint32_t ro = s_rowoff[b];
-            SPack at;
-#pragma unroll
-            for (int j = 0; j < NS; ++j) {
-                cur[j] = SMEM ? (int)s_tt[ro + (uint32_t)cur[j]]
-                              : (int)__ldg(g_tt + ro + (uint32_t)cur[j]);
-                at.v[j] = (ST)cur[j];
-            }
+                cur[j] = SMEM ? (unsigned)s_tt[ro + cur[j]] : (unsigned)__ldg(g_tt + ro + cur[j]);
             if (k < kDepth)
-                s_stack[(k + 1) * 32] = at;
+                s_stack[(k + 1) * 32] = pack_entries<sizeof(ST), NS>(cur);
         }
         depth = n;
-        const bool is_eos = tok == p.eos_id;
+        const bool is_eos = (int)tok == p.eos_id;
         // A token with no byte of its own equals its predecessor: same outputs.
+        // "No edge" is written as the sink index itself (the step and the
+        // download map it to -1), so live walks go out unconverted; lanes past
+        // the last state sit in the sink from the start.
         if (n != shared || first || is_eos || prev_eos) {
-#pragma unroll
-            for (int j = 0; j < NS; ++j) {
-                int s = (n > 0 && cur[j] != sink) ? cur[j] : CSTR_DEAD;
-                bool allowed = s >= 0;
-                if (is_eos) {            // allowed exactly in accepting states; finishes the row
-                    allowed = (accbits >> j) & 1u;
-                    s = CSTR_DEAD;
+            if (n == 0 || is_eos) {      // empty token: no edge.  EOS: allowed exactly in
+#pragma unroll                           // accepting states and finishes the row.
+                for (int j = 0; j < NS; ++j) {
+                    outs[j] = sink;
+                    words[j] = __ballot_sync(kFull, is_eos && ((accbits >> j) & 1u));
                 }
-                words[j] = __ballot_sync(kFull, allowed && ((inbits >> j) & 1u));
-                outv.v[j] = (NT)s;
+            } else {
+#pragma unroll
+                for (int j = 0; j < NS; ++j) {
+                    outs[j] = cur[j];
+                    words[j] = __ballot_sync(kFull, cur[j] != sink);
+                }
             }
+            outp = pack_entries<sizeof(NT), NS>(outs);
         }
         prev_eos = is_eos;
-        NT *nrow = (NT *)p.next + (long long)tok * p.lds + qbase;
-        *(NPack *)nrow = outv;                           // lds is a multiple of 128: in bounds
+        // lds is a multiple of 256 states: the whole unit is inside the token's row
+        *(NPack *)(next_lane + (size_t)tok * (size_t)p.lds) = outp;
         if (lane < NS) {                                 // (q0 >> 5) + NS <= lds / 32 < ldb
             uint32_t mine = words[0];
 #pragma unroll
             for (int j = 1; j < NS; ++j)
                 mine = (lane == j) ? words[j] : mine;
-            p.maskT[(long long)tok * p.ldb + (q0 >> 5) + lane] = mine;
+            maskT_lane[(size_t)tok * (size_t)p.ldb] = mine;
         }
     }
 }
@@ -243,7 +293,13 @@ cudaError_t launch_trie_ns(int ns, bool in_smem, const BuildParams &p, dim3 grid
     switch (ns) {
     case 1: CSTR_CASE(1);
     case 2: CSTR_CASE(2);
-    default: CSTR_CASE(4);
+    case 4: CSTR_CASE(4);
+    default:
+        if constexpr (sizeof(NT) == 2) {
+            CSTR_CASE(8);
+        } else {
+            CSTR_CASE(4);
+        }
     }
 #undef CSTR_CASE
 }
@@ -274,31 +330,51 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
     const size_t st = dfa->wide ? 4 : 2;
 
-    // States per lane and warps per CTA: enough states per warp to amortise the
-    // per-token work, without leaving most lanes idle on small automata.
+    // States per lane: enough states per warp to amortise the per-token work,
+    // without leaving most lanes idle on small automata.
     const int S = dfa->n_states;
-    const int ns = S >= 2048 ? 4 : (S >= 512 ? 2 : 1);
+    int ns = S >= 4096 ? 8 : (S >= 1024 ? 4 : (S >= 256 ? 2 : 1));
+    if (ns == 8 && t->wide)
+        ns = 4;                        // a lane's unit of next is at most 16 bytes
     const int per_warp = ns * 32;
-    int warps = (S + per_warp - 1) / per_warp;
-    if (warps > 8)
-        warps = 8;
-    const int threads = warps * 32;
-    const int state_groups = (S + per_warp * warps - 1) / (per_warp * warps);
+    const int state_warps = (S + per_warp - 1) / per_warp;
 
-    const size_t stack_bytes = (size_t)warps * (CSTR_STACK_DEPTH + 1) * ns * 32 * st;   // x16 bytes
+    // Warps per CTA from the shared-memory budget: the table (when it fits) is
+    // shared by all warps of a CTA, each warp adds its per-depth stack.  Aim
+    // for two resident CTAs per SM, fall back to one big CTA for large tables.
+    const size_t stack_per_warp = (size_t)(CSTR_STACK_DEPTH + 1) * ns * 32 * st;
     const size_t table_bytes = (size_t)dfa->n_classes * (size_t)dfa->row * st;
-    const size_t smem_limit = 200 * 1024;
-    const bool in_smem = 1024 + stack_bytes + table_bytes <= smem_limit;
-    const size_t smem_bytes = 1024 + stack_bytes + (in_smem ? table_bytes : 0);
+    const size_t cta_max = 200 * 1024, cta_half = 108 * 1024;
+    const bool in_smem = 1024 + 4 * stack_per_warp + table_bytes <= cta_max;
+    const size_t fixed = 1024 + (in_smem ? table_bytes : 0);
+    size_t budget = in_smem ? cta_half : 48 * 1024;
+    if (fixed + 8 * stack_per_warp > budget)
+        budget = cta_max;
+    int max_warps = (int)((budget - fixed) / stack_per_warp);
+    if (max_warps > 16)
+        max_warps = 16;
+    if (max_warps < 1)
+        max_warps = 1;
+    int state_groups = (state_warps + max_warps - 1) / max_warps;
+    const int warps_s = (state_warps + state_groups - 1) / state_groups;   // balanced groups
+    state_groups = (state_warps + warps_s - 1) / warps_s;
+    int warps_t = max_warps / warps_s;
+    if (warps_t < 1)
+        warps_t = 1;
+    const int warps = warps_s * warps_t;
+    const int threads = warps * 32;
+    const size_t smem_bytes = fixed + (size_t)warps * stack_per_warp;
+    p.warps_s = warps_s;
+    p.warps_t = warps_t;
 
-    // Token chunks: each CTA restarts its walk at the root, so chunks should be
-    // long; but there must be enough CTAs to fill the machine.
+    // Token chunks: every warp restarts its walk at the root of the trie, so a
+    // warp's share should be long; but there must be enough CTAs for the machine.
     int dev_sms = 148;
     cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, t->device);
     const long long want_ctas = 8LL * dev_sms;
     long long chunks = (want_ctas + state_groups - 1) / state_groups;
     long long tokens_per_cta = (t->V + chunks - 1) / chunks;
-    const long long min_tokens = in_smem ? 512 : 128;
+    const long long min_tokens = (long long)warps_t * (in_smem ? 256 : 128);
     if (tokens_per_cta < min_tokens)
         tokens_per_cta = min_tokens;
     chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;

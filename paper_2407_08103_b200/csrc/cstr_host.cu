@@ -70,7 +70,7 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     d->n_states = n_states;
     d->start = start_state;
     d->wide = (int64_t)n_states + 1 > 32767;
-    d->row = ((int64_t)n_states + 1 + 7) / 8 * 8;
+    d->row = ((int64_t)n_states + 1 + 255) / 256 * 256;
     const size_t esz = d->wide ? 4 : 2;
 
     // Byte classes: bytes whose columns are identical in every state.
@@ -115,10 +115,11 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
             const int32_t *src = &col[(size_t)rep[c] * n_states];
             for (int64_t q = 0; q < d->row; ++q) {
                 const int32_t t = (q < n_states && src[q] >= 0) ? src[q] : sink;
+                const size_t at = (size_t)c * d->row + (size_t)CSTR_PERM(q);
                 if (d->wide)
-                    ((int32_t *)tt.data())[(size_t)c * d->row + q] = t;
+                    ((uint32_t *)tt.data())[at] = (uint32_t)CSTR_PERM(t);
                 else
-                    ((int16_t *)tt.data())[(size_t)c * d->row + q] = (int16_t)t;
+                    ((uint16_t *)tt.data())[at] = (uint16_t)CSTR_PERM(t);
             }
         }
         flags.resize(n_states);
@@ -311,7 +312,7 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     t->max_states = max_states;
     t->V = vocab->V;
     t->W = (vocab->V + 31) / 32;
-    t->lds = ((int64_t)max_states + 127) / 128 * 128;
+    t->lds = ((int64_t)max_states + 255) / 256 * 256;
     t->ldw = ((int64_t)t->W + 31) / 32 * 32;
     t->ldb = t->lds / 32 + 8 - (t->lds / 32) % 8;   // a multiple of 8, above lds / 32
     t->wide = (int64_t)max_states + 1 > 32767;
@@ -450,8 +451,10 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
                 for (int32_t r = 0; r < nr; ++r) {
                     const size_t at = (size_t)v * nr + r;
                     const int32_t x = t->wide ? ((const int32_t *)tmp.data())[at]
-                                              : (int32_t)((const int16_t *)tmp.data())[at];
-                    next_host[(int64_t)(r0 + r) * t->V + v] = x;
+                                              : (int32_t)((const uint16_t *)tmp.data())[at];
+                    // device entries are permuted ids; the sink n_states means "no edge"
+                    const int32_t u = CSTR_UNPERM(x);
+                    next_host[(int64_t)(r0 + r) * t->V + v] = (u == t->n_states) ? -1 : u;
                 }
             }
         }

@@ -20,17 +20,27 @@ int cstr_fail(int code, const char *fmt, ...);
                              "%s failed: %s", #expr, cudaGetErrorString(e_));            \
     } while (0)
 
+// State ids inside the builder's tables are permuted within blocks of 256:
+// state 256 b + 8 l + j sits at slot 256 b + 32 j + l.  A warp whose lane l
+// owns the 8 consecutive states 8 l .. 8 l + 7 then reads 32 consecutive slots
+// per lookup round (no shared-memory bank conflicts) as long as the walk keeps
+// neighbouring states neighbours, which counters and literal chains do.
+#define CSTR_PERM(s) (((s) & ~255) | (((s) & 7) << 5) | (((s) >> 3) & 31))
+#define CSTR_UNPERM(v) (((v) & ~255) | (((v) & 31) << 3) | (((v) >> 5) & 7))
+
 // Byte DFA as the builder reads it: bytes that no state tells apart share a
-// class, and the table is stored class-major ("transposed") with one extra
-// dead-sink column, tt[c][s] for s in [0, n_states], entry n_states = sink, so
-// that a walk needs no "is it dead" branch: the sink maps to itself.
+// class, and the table is stored class-major ("transposed") in permuted slots,
+// holding permuted targets, with a dead sink (state n_states) that maps to
+// itself, so that a walk needs no "is it dead" branch:
+//     tt[c][PERM(s)] = PERM(target of s on class c, or n_states)
+// for s in [0, row), row = n_states + 1 rounded up to 256.
 struct cstr_dfa {
     int device;
     int32_t n_states;
     int32_t start;
     int wide;            // 0: int16 entries (n_states + 1 <= 32767), 1: int32 entries
     int32_t n_classes;   // 1..256
-    int64_t row;         // entries per class row (n_states + 1, rounded up to 8)
+    int64_t row;         // entries per class row (n_states + 1, rounded up to 256)
     void *tt;            // DEVICE [n_classes][row]
     uint8_t *cls;        // DEVICE [256] byte -> class
     uint8_t *accept;     // DEVICE [n_states]
@@ -43,7 +53,7 @@ struct cstr_dfa {
 //               shared prefix (little endian in z, w) }
 // The shared prefix is clipped to CSTR_STACK_DEPTH.  Raw bytes / offsets serve
 // walks that start at the root and suffixes longer than 8 bytes.
-#define CSTR_STACK_DEPTH 16
+#define CSTR_STACK_DEPTH 8
 struct cstr_vocab {
     int device;
     int32_t V;
@@ -55,7 +65,8 @@ struct cstr_vocab {
 };
 
 // Token table.  next is token-major: next[v][q] (a step reads one entry per
-// row; the builder writes whole 64-byte state segments).  mask is state-major
+// row; the builder writes whole state segments); entries are unsigned permuted
+// state ids (CSTR_PERM), "no edge" being the permuted sink CSTR_PERM(n_states).  mask is state-major
 // as the step streams it.  maskT is the builder's intermediate: per token one
 // word per block of 32 states, transposed into mask by a second kernel.
 struct cstr_table {
@@ -64,7 +75,7 @@ struct cstr_table {
     cstr_vocab *owned_vocab;   // non-null when created by cstr_build_token_table
     int32_t max_states;
     int32_t V, W;
-    int64_t lds;       // entries per token row of next (max_states rounded up to 128)
+    int64_t lds;       // entries per token row of next (max_states rounded up to 256)
     int64_t ldw;       // words per state row of mask (W rounded up to 32), padding zero
     int64_t ldb;       // words per token row of maskT (state blocks rounded up to 8)
     int wide;          // capacity dtype of next: 0 int16, 1 int32

@@ -142,7 +142,9 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     if (c.active && key != 0ull) {
         tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
         const long long at = (long long)tok * tb.lds + c.q;
-        q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const int16_t *)tb.next)[at];
+        q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const uint16_t *)tb.next)[at];
+        q2 = CSTR_UNPERM(q2);                           // entries are permuted ids ...
+        q2 = (q2 == tb.n_states) ? CSTR_DEAD : q2;      // ... and the sink n_states means "no edge"
     } else if (c.active) {
         atomicAdd(p.counters + 1, 1ull);
     } else if (c.q != -1) {
