@@ -101,42 +101,50 @@ __global__ void __launch_bounds__(512)
 build_trie_kernel(const __grid_constant__ BuildParams p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    typedef typename Unit<sizeof(ST)>::type SU;                 // unsigned view of a table entry
-    typedef typename Unit<sizeof(ST) * NS>::type SPack;
+    constexpr int ESZ = (int)sizeof(ST);
+    typedef typename Unit<ESZ>::type SU;                        // unsigned view of a table entry
+    typedef typename Unit<ESZ * NS>::type SPack;
     typedef typename Unit<sizeof(NT) * NS>::type NPack;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const unsigned sink = (unsigned)CSTR_PERM(p.n_states);      // all ids below are permuted
+    // Every state id below is a "code": the byte offset of the state's slot in
+    // a class row, ESZ * PERM(state).  Table entries hold codes, so a lookup is
+    // one add and one load; next[] stores codes too (decoded where it is read).
+    const unsigned sink = (unsigned)CSTR_PERM(p.n_states) * ESZ;
 
-    // shared memory: [row offset per byte: 256 x u32][stack: nwarps x (kDepth+1) x 32 SPack][table]
+    // shared memory: [row byte offset per byte value: 256 x u32]
+    //                [stack: nwarps x (kDepth+1) x 32 SPack][table]
     uint32_t *s_rowoff = (uint32_t *)smem;
     SPack *s_stack = (SPack *)(smem + 1024) + (size_t)warp * (kDepth + 1) * 32 + lane;
-    SU *s_tt = (SU *)(smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack));
+    const unsigned char *s_tt = smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack);
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
-        s_rowoff[i] = (uint32_t)p.cls[i] * (uint32_t)p.row;
+        s_rowoff[i] = (uint32_t)p.cls[i] * (uint32_t)p.row * ESZ;
     if (SMEM) {
-        const int n16 = (int)((long long)p.n_classes * p.row * (long long)sizeof(ST) / 16);
+        const int n16 = (int)((long long)p.n_classes * p.row * ESZ / 16);
         const uint4 *src = (const uint4 *)p.tt;
         uint4 *dst = (uint4 *)s_tt;      // row is a multiple of 256 entries: whole 16-byte units
         for (int i = threadIdx.x; i < n16; i += blockDim.x)
             dst[i] = __ldg(src + i);
     }
     __syncthreads();
-    const SU *g_tt = (const SU *)p.tt;
+    const unsigned char *g_tt = (const unsigned char *)p.tt;
 
     const int warp_s = warp % p.warps_s, warp_t = warp / p.warps_s;
     const int q0 = (blockIdx.x * p.warps_s + warp_s) * NS * 32;
     if (q0 >= p.n_states)
         return;                                          // whole warp out of range
     const int qbase = q0 + NS * lane;
-    unsigned cur[NS];
+    unsigned cur[NS], sinks[NS];
     unsigned accbits = 0;
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
         const bool in = qbase + j < p.n_states;
         accbits |= (unsigned)(in && p.accept[qbase + j] != 0) << j;
-        cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) : sink;
+        cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) * ESZ : sink;
+        sinks[j] = sink;
     }
-    s_stack[0] = pack_entries<sizeof(ST), NS>(cur);
+    SPack pk = pack_entries<ESZ, NS>(cur);               // cur[] in packed form, kept in step
+    const NPack dead_out = pack_entries<sizeof(NT), NS>(sinks);
+    s_stack[0] = pk;
     __syncwarp();
 
     const int c_begin = blockIdx.y * p.tokens_per_cta;
@@ -147,12 +155,11 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     if (t_begin >= t_end)
         return;
     int depth = 0;                                       // depth of the path held in cur[]
-    unsigned outs[NS];
-    uint32_t words[NS];
-    NPack outp;
+    uint32_t words[NS > 4 ? NS : 4] = {0u, 0u, 0u, 0u};
+    NPack outp = dead_out;
     bool prev_eos = true;                                // forces the first token's outputs
     NT *const next_lane = (NT *)p.next + qbase;
-    uint32_t *const maskT_lane = p.maskT + (q0 >> 5) + (lane < NS ? lane : 0);
+    uint32_t *const maskT_warp = p.maskT + (q0 >> 5);
 
     uint4 d_next = __ldg(p.desc + t_begin);              // same address in every lane
     for (int i = t_begin; i < t_end; ++i) {
@@ -163,8 +170,10 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
         const int n = (int)(d.y & 0xffffffu);
         const bool first = (i == t_begin);
         const int shared = first ? 0 : (int)(d.y >> 24);
-        if (shared < depth)                              // climb back to the shared prefix
-            unpack_entries<sizeof(ST), NS>(s_stack[shared * 32], cur);
+        if (shared < depth) {                            // climb back to the shared prefix
+            pk = s_stack[shared * 32];
+            unpack_entries<ESZ, NS>(pk, cur);
+        }
         unsigned long long inl = ((unsigned long long)d.w << 32) | d.z;   // bytes shared .. shared+7
         for (int k = shared; k < n; ++k) {
             unsigned b;
@@ -175,43 +184,52 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
                 b = __ldg(p.bytes + __ldg(p.off + tok) + k);
             }
             const uint32_t ro = s_rowoff[b];
+            if (SMEM) {
+                const unsigned char *rowp = s_tt + ro;
 #pragma unroll
-            for (int j = 0; j < NS; ++j)
-                cur[j] = SMEM ? (unsigned)s_tt[ro + cur[j]] : (unsigned)__ldg(g_tt + ro + cur[j]);
+                for (int j = 0; j < NS; ++j)
+                    cur[j] = (unsigned)*(const SU *)(rowp + cur[j]);
+            } else {
+                const unsigned char *rowp = g_tt + ro;
+#pragma unroll
+                for (int j = 0; j < NS; ++j)
+                    cur[j] = (unsigned)__ldg((const SU *)(rowp + cur[j]));
+            }
+            pk = pack_entries<ESZ, NS>(cur);
             if (k < kDepth)
-                s_stack[(k + 1) * 32] = pack_entries<sizeof(ST), NS>(cur);
+                s_stack[(k + 1) * 32] = pk;
         }
         depth = n;
         const bool is_eos = (int)tok == p.eos_id;
         // A token with no byte of its own equals its predecessor: same outputs.
-        // "No edge" is written as the sink index itself (the step and the
-        // download map it to -1), so live walks go out unconverted; lanes past
-        // the last state sit in the sink from the start.
+        // "No edge" goes out as the sink's own code (decoded to -1 by readers),
+        // so live walks are stored as they are; lanes past the last state sit
+        // in the sink from the start.
         if (n != shared || first || is_eos || prev_eos) {
             if (n == 0 || is_eos) {      // empty token: no edge.  EOS: allowed exactly in
-#pragma unroll                           // accepting states and finishes the row.
-                for (int j = 0; j < NS; ++j) {
-                    outs[j] = sink;
-                    words[j] = __ballot_sync(kFull, is_eos && ((accbits >> j) & 1u));
-                }
-            } else {
+                outp = dead_out;         // accepting states, and it finishes the row.
 #pragma unroll
-                for (int j = 0; j < NS; ++j) {
-                    outs[j] = cur[j];
+                for (int j = 0; j < NS; ++j)
+                    words[j] = __ballot_sync(kFull, is_eos && ((accbits >> j) & 1u));
+            } else {
+                if constexpr (sizeof(NT) == sizeof(ST))
+                    outp = pk;
+                else
+                    outp = pack_entries<sizeof(NT), NS>(cur);
+#pragma unroll
+                for (int j = 0; j < NS; ++j)
                     words[j] = __ballot_sync(kFull, cur[j] != sink);
-                }
             }
-            outp = pack_entries<sizeof(NT), NS>(outs);
         }
         prev_eos = is_eos;
         // lds is a multiple of 256 states: the whole unit is inside the token's row
         *(NPack *)(next_lane + (size_t)tok * (size_t)p.lds) = outp;
-        if (lane < NS) {                                 // (q0 >> 5) + NS <= lds / 32 < ldb
-            uint32_t mine = words[0];
-#pragma unroll
-            for (int j = 1; j < NS; ++j)
-                mine = (lane == j) ? words[j] : mine;
-            maskT_lane[(size_t)tok * (size_t)p.ldb] = mine;
+        if (lane == 0) {                 // ballots are warp-uniform; (q0 >> 5) + NS <= lds / 32 < ldb
+            uint32_t *mrow = maskT_warp + (size_t)tok * (size_t)p.ldb;       // NS-word aligned
+            if constexpr (NS == 1) *mrow = words[0];
+            if constexpr (NS == 2) *(uint2 *)mrow = make_uint2(words[0], words[1]);
+            if constexpr (NS >= 4) *(uint4 *)mrow = make_uint4(words[0], words[1], words[2], words[3]);
+            if constexpr (NS == 8) *(uint4 *)(mrow + 4) = make_uint4(words[4], words[5], words[6], words[7]);
         }
     }
 }

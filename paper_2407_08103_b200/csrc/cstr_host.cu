@@ -116,10 +116,11 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
             for (int64_t q = 0; q < d->row; ++q) {
                 const int32_t t = (q < n_states && src[q] >= 0) ? src[q] : sink;
                 const size_t at = (size_t)c * d->row + (size_t)CSTR_PERM(q);
+                // entries are codes: the byte offset of the target's slot in a row
                 if (d->wide)
-                    ((uint32_t *)tt.data())[at] = (uint32_t)CSTR_PERM(t);
+                    ((uint32_t *)tt.data())[at] = (uint32_t)CSTR_PERM(t) * 4u;
                 else
-                    ((uint16_t *)tt.data())[at] = (uint16_t)CSTR_PERM(t);
+                    ((uint16_t *)tt.data())[at] = (uint16_t)(CSTR_PERM(t) * 2);
             }
         }
         flags.resize(n_states);
@@ -362,6 +363,7 @@ extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int3
     table->n_states = dfa->n_states;
     table->start = dfa->start;
     table->eos_id = eos_id;
+    table->code_shift = dfa->wide ? 2 : 1;
     CSTR_CUDA_TRY(cudaMemcpyAsync(table->accept, dfa->accept, (size_t)dfa->n_states,
                                   cudaMemcpyDeviceToDevice, stream));
     return cstr_launch_build(table, dfa, stream);
@@ -452,8 +454,8 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
                     const size_t at = (size_t)v * nr + r;
                     const int32_t x = t->wide ? ((const int32_t *)tmp.data())[at]
                                               : (int32_t)((const uint16_t *)tmp.data())[at];
-                    // device entries are permuted ids; the sink n_states means "no edge"
-                    const int32_t u = CSTR_UNPERM(x);
+                    // device entries are codes of permuted ids; the sink n_states means "no edge"
+                    const int32_t u = CSTR_UNPERM(x >> t->code_shift);
                     next_host[(int64_t)(r0 + r) * t->V + v] = (u == t->n_states) ? -1 : u;
                 }
             }

@@ -32,7 +32,8 @@ int cstr_fail(int code, const char *fmt, ...);
 // class, and the table is stored class-major ("transposed") in permuted slots,
 // holding permuted targets, with a dead sink (state n_states) that maps to
 // itself, so that a walk needs no "is it dead" branch:
-//     tt[c][PERM(s)] = PERM(target of s on class c, or n_states)
+//     tt[c][PERM(s)] = code(target of s on class c, or n_states),
+//     code(t) = PERM(t) * sizeof(entry): the byte offset of t's slot in a row,
 // for s in [0, row), row = n_states + 1 rounded up to 256.
 struct cstr_dfa {
     int device;
@@ -65,8 +66,9 @@ struct cstr_vocab {
 };
 
 // Token table.  next is token-major: next[v][q] (a step reads one entry per
-// row; the builder writes whole state segments); entries are unsigned permuted
-// state ids (CSTR_PERM), "no edge" being the permuted sink CSTR_PERM(n_states).  mask is state-major
+// row; the builder writes whole state segments); entries are the unsigned
+// codes the builder walks with (CSTR_PERM(state) << code_shift), "no edge"
+// being the code of the sink state n_states.  mask is state-major
 // as the step streams it.  maskT is the builder's intermediate: per token one
 // word per block of 32 states, transposed into mask by a second kernel.
 struct cstr_table {
@@ -86,6 +88,7 @@ struct cstr_table {
     int32_t n_states;  // of the automaton currently held (0 = not built)
     int32_t start;
     int32_t eos_id;
+    int32_t code_shift; // next entries are CSTR_PERM(state) << code_shift (1: 16-bit DFA, 2: 32-bit)
 };
 
 struct cstr_workspace {

@@ -29,6 +29,7 @@ struct TableDesc {
     long long ldw;
     int n_states;
     int wide;
+    int code_shift;
 };
 
 struct StepParams {
@@ -143,7 +144,8 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
         tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
         const long long at = (long long)tok * tb.lds + c.q;
         q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const uint16_t *)tb.next)[at];
-        q2 = CSTR_UNPERM(q2);                           // entries are permuted ids ...
+        q2 = q2 >> tb.code_shift;                       // entries are codes of permuted ids ...
+        q2 = CSTR_UNPERM(q2);
         q2 = (q2 == tb.n_states) ? CSTR_DEAD : q2;      // ... and the sink n_states means "no edge"
     } else if (c.active) {
         atomicAdd(p.counters + 1, 1ull);
@@ -380,6 +382,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         p.tab[i].ldw = t->ldw;
         p.tab[i].n_states = t->n_states;
         p.tab[i].wide = t->wide;
+        p.tab[i].code_shift = t->code_shift;
     }
     const cstr_table *t0 = a.tables[0];
     p.row_table = a.row_table;
