@@ -51,6 +51,8 @@ def parse_args():
                          "vocabulary (for profiler captures); its numbers are not bench values")
     ap.add_argument("--skip-build-bench", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-other-workloads", action="store_true",
+                    help="do not time the four other workloads (reported under 'other_workloads')")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -162,6 +164,84 @@ def time_oracle(w, dfa, vb, vo, pools, budget_s: float, max_steps: int):
     dt = time.perf_counter() - t0
     sample = "%d whole-batch steps (%d rows x %d tokens) of %s, %.1f s" % (done, B, V, WORKLOAD, dt)
     return B * V * done / dt, threads, sample, dt / done
+
+
+def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak, steps=48):
+    """Step-kernel and table-build timing of one of the other workloads: device
+    generated seeded logits (timing only; parity is covered by the tests), a
+    pool of tensors larger than twice the L2 where the batch allows, finished
+    rows restarted, events around each step launch."""
+    from synth.configs import CONFIGS, config_dfas, config_vocab, row_table_for
+    w = CONFIGS[name]
+    dfas = config_dfas(name)
+    vb, vo = config_vocab(name)
+    V, B = vo.size - 1, w.batch
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    tables, handles, build_ms = [], [], []
+    for d in dfas:
+        h = cstr.cstr_load_dfa(*d)
+        t = cstr.cstr_table_create(vocab, d[0].shape[0])
+        for rep in range(3 if len(tables) == 0 else 1):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            cstr.cstr_table_build(t, h, -1, stream)
+            a1.record(stream)
+            a1.synchronize()
+            if len(tables) == 0 and rep > 0:
+                build_ms.append(a0.elapsed_time(a1))
+        tables.append(t)
+        handles.append(h)
+    esz = 4 if w.dtype == "f32" else 2
+    tdtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    tensor_bytes = B * V * esz
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    pool_n = int(max(2, min(256, -(-2 * l2 // tensor_bytes))))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.logits_seed)
+    pool = [(torch.randn((B, V), generator=gen, device=dev, dtype=torch.float32) * w.sigma).to(tdtype)
+            for _ in range(pool_n)]
+    noise = None
+    if w.gumbel:
+        gen.manual_seed(w.noise_seed)
+        noise = []
+        for _ in range(min(pool_n, 2)):
+            u = torch.rand((B, V), generator=gen, device=dev, dtype=torch.float32).clamp_(1e-20, 1 - 1e-7)
+            noise.append(-torch.log(-torch.log(u)))
+    row_table = row_table_for(w, B)
+    dec = ConstrainedDecoder(tables, B, row_table=row_table, device=dev)
+    start_vec = dec.states.clone()
+    out = [torch.empty((B, V), dtype=tdtype, device=dev) for _ in range(2)]
+    pairs = []
+    for i in range(steps + 4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        dec.step(pool[i % pool_n], noise=None if noise is None else noise[i % len(noise)],
+                 masked_out=out[i & 1], stream=stream)
+        e1.record(stream)
+        torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
+        if i >= 4:
+            pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    bytes_per_logit = 2 * esz + (4 if w.gumbel else 0) + 1.0 / 8.0
+    step_bytes = B * V * bytes_per_logit
+    gbs = step_bytes / (kernel_ms * 1e-3) / 1e9
+    S0 = int(dfas[0][0].shape[0])
+    bms = float(np.mean(build_ms))
+    bgbs = S0 * V * BYTES_PER_TRANSITION / (bms * 1e-3) / 1e9
+    hbm_honest = pool_n * tensor_bytes >= 2 * l2
+    return {
+        "workload": name, "vocab": V, "batch": B, "dfa_states": [int(d[0].shape[0]) for d in dfas],
+        "dtype": w.dtype, "sampler": "gumbel-max" if w.gumbel else "greedy",
+        "tables": len(tables), "step_kernel_ms": kernel_ms,
+        "logits_per_s": B * V / (kernel_ms * 1e-3),
+        "roofline": {"bound": "hbm" if hbm_honest else "launch latency (working set sits in L2)",
+                     "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "traffic": None, "bytes_per_logit": bytes_per_logit,
+                     "logits_pool": "%d tensors x %.1f MB" % (pool_n, tensor_bytes / 1e6)},
+        "table_build": {"dfa_states": S0, "ms": bms, "transitions_per_s": S0 * V / (bms * 1e-3),
+                        "store_gbs": bgbs, "frac_of_hbm_peak": bgbs / peak},
+    }
 
 
 def run_reference(args):
@@ -361,6 +441,18 @@ def main():
         build_random = ms[1:]
         del t_rd, h_rd
 
+    # ---- the other four workloads (single-GPU runs only) --------------------
+    others = None
+    if rank == 0 and world == 1 and not args.skip_other_workloads and args.case == "full":
+        del dev_pool, staging, out_bufs
+        torch.cuda.empty_cache()
+        peak_now, _ = measured_hbm_peak()
+        others = []
+        for name in ("api_1k", "json_32k", "schema40_128k", "random10k_256k"):
+            others.append(time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream,
+                                              peak_now))
+            torch.cuda.empty_cache()
+
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1) --------
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
@@ -420,6 +512,7 @@ def main():
         "table_build": [build_entry(bt, S, WORKLOAD)] +
                        ([build_entry(build_random, 10000, "random10k_256k (DFA 0)")] if build_random else []),
         "table_build_e2e_ms": build_e2e_ms,
+        "other_workloads": others,
         "status_rows": {"bad_state": bad, "empty_mask": empty},
     }
     print(json.dumps(line))
