@@ -159,54 +159,72 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
 }
 
 // ---- per-vector processing ------------------------------------------------
+//
+// The streaming loop tracks the winner at vector granularity only: the largest
+// candidate of each 16-byte vector (NaN where nothing in it can win) and the
+// first vector that holds the running maximum.  Which element of that vector
+// it is gets resolved once per warp after the loop (refine_winner), which
+// keeps the per-logit work to two selects and one max.
 
-// fp32: 4 logits per 16-byte vector, 4 mask bits.
-__device__ __forceinline__ float4 apply_f32(float4 x, const float4 *nz, unsigned bits, int idx,
-                                            Best &b)
+struct VBest {
+    float v;
+    int vec;   // token index of the winning vector's first element; -1: none yet
+};
+
+__device__ __forceinline__ void vconsider(VBest &b, float m, int tok)
 {
-    const float ninf = -CUDART_INF_F, qnan = CUDART_NAN_F;
-    float in[4] = {x.x, x.y, x.z, x.w};
-    float out[4];
-    float add[4] = {0.f, 0.f, 0.f, 0.f};
-    if (nz) {
-        add[0] = nz->x; add[1] = nz->y; add[2] = nz->z; add[3] = nz->w;
-    }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const bool ok = (bits >> e) & 1u;
-        out[e] = ok ? in[e] : ninf;
-        const float s = nz ? in[e] + add[e] : in[e];
-        consider(b, ok ? s : qnan, idx + e);
-    }
-    return make_float4(out[0], out[1], out[2], out[3]);
+    const bool take = (m > b.v) || (b.vec < 0 && m == m);
+    b.v = take ? m : b.v;
+    b.vec = take ? tok : b.vec;
 }
 
-// bf16: 8 logits per 16-byte vector, 8 mask bits; noise comes as two float4.
-__device__ __forceinline__ uint4 apply_bf16(uint4 x, const float4 *nz, unsigned bits, int idx,
-                                            Best &b)
+// fp32: 4 logits per 16-byte vector, mask bits in bits[3:0].
+template <bool NOISE>
+__device__ __forceinline__ uint4 apply_f32(uint4 xu, float4 nz, unsigned bits, float &m)
+{
+    const float ninf = -CUDART_INF_F, qnan = CUDART_NAN_F;
+    const float x[4] = {__uint_as_float(xu.x), __uint_as_float(xu.y), __uint_as_float(xu.z),
+                        __uint_as_float(xu.w)};
+    const float add[4] = {nz.x, nz.y, nz.z, nz.w};
+    float o[4], c[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const bool ok = bits & (1u << e);
+        o[e] = ok ? x[e] : ninf;
+        const float s = NOISE ? x[e] + add[e] : x[e];
+        c[e] = ok ? s : qnan;
+    }
+    m = fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3]));      // fmaxf skips NaN operands
+    return make_uint4(__float_as_uint(o[0]), __float_as_uint(o[1]), __float_as_uint(o[2]),
+                      __float_as_uint(o[3]));
+}
+
+// bf16: 8 logits per 16-byte vector, mask bits in bits[7:0]; noise as two float4.
+template <bool NOISE>
+__device__ __forceinline__ uint4 apply_bf16(uint4 xu, float4 nza, float4 nzb, unsigned bits,
+                                            float &m)
 {
     const float qnan = CUDART_NAN_F;
-    unsigned in[4] = {x.x, x.y, x.z, x.w};
-    unsigned out[4];
-    float add[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (nz) {
-        add[0] = nz[0].x; add[1] = nz[0].y; add[2] = nz[0].z; add[3] = nz[0].w;
-        add[4] = nz[1].x; add[5] = nz[1].y; add[6] = nz[1].z; add[7] = nz[1].w;
-    }
+    const unsigned w[4] = {xu.x, xu.y, xu.z, xu.w};
+    const float add[8] = {nza.x, nza.y, nza.z, nza.w, nzb.x, nzb.y, nzb.z, nzb.w};
+    unsigned o[4];
+    float c[8];
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
-        const bool ok0 = (bits >> (2 * h)) & 1u, ok1 = (bits >> (2 * h + 1)) & 1u;
-        const unsigned lo = in[h] & 0xffffu, hi = in[h] & 0xffff0000u;
-        out[h] = (ok0 ? lo : 0xff80u) | (ok1 ? hi : 0xff800000u);
-        float f0 = __uint_as_float(lo << 16), f1 = __uint_as_float(hi);   // exact widening
-        if (nz) {
+        const bool ok0 = bits & (1u << (2 * h)), ok1 = bits & (2u << (2 * h));
+        const unsigned s0 = ok0 ? w[h] : 0xff80ff80u, s1 = ok1 ? w[h] : 0xff80ff80u;
+        o[h] = __byte_perm(s0, s1, 0x7610);               // low half from s0, high half from s1
+        float f0 = __uint_as_float(w[h] << 16), f1 = __uint_as_float(w[h] & 0xffff0000u);
+        if (NOISE) {
             f0 = f0 + add[2 * h];
             f1 = f1 + add[2 * h + 1];
         }
-        consider(b, ok0 ? f0 : qnan, idx + 2 * h);
-        consider(b, ok1 ? f1 : qnan, idx + 2 * h + 1);
+        c[2 * h] = ok0 ? f0 : qnan;
+        c[2 * h + 1] = ok1 ? f1 : qnan;
     }
-    return make_uint4(out[0], out[1], out[2], out[3]);
+    m = fmaxf(fmaxf(fmaxf(c[0], c[1]), fmaxf(c[2], c[3])),
+              fmaxf(fmaxf(c[4], c[5]), fmaxf(c[6], c[7])));
+    return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // Scalar element, shared by the vector kernel's ragged tail and the scalar kernel.
@@ -260,7 +278,8 @@ step_vec_kernel(const __grid_constant__ StepParams p)
     const int tile_end = min(total_tiles, (c.chunk + 1) * p.tiles_per_cta);
     const int Vv = p.V - p.V % VEC;                 // tokens covered by whole vectors
 
-    Best b = {-CUDART_INF_F, -1};
+    VBest vb = {-CUDART_INF_F, -1};
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
 
     for (int tile = c.chunk * p.tiles_per_cta + warp; tile < tile_end; tile += nwarps) {
         const int tok0 = tile * TILE;
@@ -295,13 +314,13 @@ step_vec_kernel(const __grid_constant__ StepParams p)
             for (int j = 0; j < kUnroll; ++j) {
                 const int tok = tok0 + (j * 32 + lane) * VEC;
                 if (BF16) {
-                    nz[2 * j] = nz[2 * j + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    nz[2 * j] = nz[2 * j + 1] = zero4;
                     if (tok < Vv) {
                         nz[2 * j] = __ldcs(nzrow + tok / 4);
                         nz[2 * j + 1] = __ldcs(nzrow + tok / 4 + 1);
                     }
                 } else {
-                    nz[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    nz[j] = zero4;
                     if (tok < Vv)
                         nz[j] = __ldcs(nzrow + tok / 4);
                 }
@@ -312,25 +331,60 @@ step_vec_kernel(const __grid_constant__ StepParams p)
             const int tok = tok0 + (j * 32 + lane) * VEC;
             const int word_in_tile = j * VEC + lane / LANES_PER_WORD;
             const uint32_t word = __shfl_sync(kFull, mw[word_in_tile / 32], word_in_tile % 32);
-            const unsigned bits = (word >> ((lane % LANES_PER_WORD) * VEC)) & ((1u << VEC) - 1u);
+            const unsigned bits = word >> ((lane % LANES_PER_WORD) * VEC);   // low VEC bits count
             if (tok < Vv) {
-                if (BF16) {
-                    const uint4 o = apply_bf16(x[j], NOISE ? &nz[2 * j] : nullptr, bits, tok, b);
-                    __stcs(out + tok / VEC, o);
-                } else {
-                    const float4 xf = make_float4(__uint_as_float(x[j].x), __uint_as_float(x[j].y),
-                                                  __uint_as_float(x[j].z), __uint_as_float(x[j].w));
-                    const float4 o = apply_f32(xf, NOISE ? &nz[j] : nullptr, bits, tok, b);
-                    __stcs(out + tok / VEC,
-                           make_uint4(__float_as_uint(o.x), __float_as_uint(o.y),
-                                      __float_as_uint(o.z), __float_as_uint(o.w)));
-                }
+                float m;
+                uint4 o;
+                if (BF16)
+                    o = apply_bf16<NOISE>(x[j], NOISE ? nz[2 * j] : zero4,
+                                          NOISE ? nz[2 * j + 1] : zero4, bits, m);
+                else
+                    o = apply_f32<NOISE>(x[j], NOISE ? nz[j] : zero4, bits, m);
+                __stcs(out + tok / VEC, o);
+                vconsider(vb, m, tok);
             }
         }
     }
+
+    // Winner among the warp's vectors (every lane ends with the same pair), then
+    // the element inside that vector: lanes 0..VEC-1 re-read one logit each (an
+    // allowed logit is unchanged even when the step runs in place).
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(kFull, vb.v, off);
+        const int oi = __shfl_xor_sync(kFull, vb.vec, off);
+        const bool take = oi >= 0 && (vb.vec < 0 || ov > vb.v || (ov == vb.v && oi < vb.vec));
+        vb.v = take ? ov : vb.v;
+        vb.vec = take ? oi : vb.vec;
+    }
+    Best b = {-CUDART_INF_F, -1};
+    if (vb.vec >= 0) {                              // warp-uniform
+        __syncwarp();
+        bool match = false;
+        if (lane < VEC) {
+            const int i = vb.vec + lane;
+            const bool ok = (c.mrow[i >> 5] >> (i & 31)) & 1u;
+            float f;
+            if (BF16)
+                f = __uint_as_float((unsigned)((const unsigned short *)p.logits)[row_off + i] << 16);
+            else
+                f = ((const float *)p.logits)[row_off + i];
+            if (NOISE)
+                f = f + p.noise[row_off + i];
+            match = ok && f == vb.v;
+        }
+        const unsigned hits = __ballot_sync(kFull, match);
+        if (hits != 0u && lane == 0) {
+            b.v = vb.v;
+            b.i = vb.vec + __ffs((int)hits) - 1;
+        }
+    }
     // ragged tail (V not a multiple of the vector width): highest indices of the row
-    if (c.chunk == p.nchunks - 1 && warp == 0 && Vv + lane < p.V)
-        apply_one<BF16>(p, c, row_off, Vv + lane, b);
+    if (c.chunk == p.nchunks - 1 && warp == 0 && Vv + lane < p.V) {
+        Best tb = {-CUDART_INF_F, -1};
+        apply_one<BF16>(p, c, row_off, Vv + lane, tb);
+        merge(b, tb.v, tb.i);
+    }
 
     finish_row(p, c, b);
 }
@@ -403,10 +457,12 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     const int esz = bf16 ? 2 : 4;
     const int tile = 32 * (bf16 ? 8 : 4) * kUnroll;
     const int total_tiles = (p.V + tile - 1) / tile;
-    // 8 tiles (one per warp) per CTA when there is enough work to fill the
-    // machine a few times over, fewer for small batches.
+    // 16 tiles (two per warp) per CTA when there is enough work to fill the
+    // machine a few times over - measured best on B200: one tile per warp leaves
+    // the per-warp set-up and reduction dominant, more tiles per CTA unbalance
+    // the row tails - and fewer for small batches.
     const long long want_ctas = 4LL * sm_count(a.device);
-    int tiles_per_cta = 8;
+    int tiles_per_cta = 16;
     while (tiles_per_cta > 1 &&
            (long long)a.batch * ((total_tiles + tiles_per_cta - 1) / tiles_per_cta) < want_ctas)
         tiles_per_cta >>= 1;
