@@ -49,9 +49,12 @@ struct StepParams {
     int n_tables;
     int nchunks;         // CTAs per row
     int tiles_per_cta;
+    int tile_tokens;     // tokens per warp tile of the launched kernel
 };
 
-constexpr int kUnroll = 8;          // 16-byte vectors in flight per lane per tile
+// 16-byte vectors in flight per lane per tile: 8 for the greedy kernels, 4 when a
+// noise stream is read as well (keeps the register count at four CTAs per SM).
+__host__ __device__ constexpr int unroll_for(bool noise) { return noise ? 4 : 8; }
 constexpr unsigned kFull = 0xffffffffu;
 
 struct Best {
@@ -263,9 +266,10 @@ __global__ void __launch_bounds__(256)
 step_vec_kernel(const __grid_constant__ StepParams p)
 {
     constexpr int VEC = BF16 ? 8 : 4;               // logits per 16-byte vector
+    constexpr int kUnroll = unroll_for(NOISE);
     constexpr int TILE = 32 * VEC * kUnroll;        // tokens per warp tile
-    constexpr int WORDS = TILE / 32;                // mask words per tile (32 or 64)
-    constexpr int WPL = WORDS / 32;                 // mask words per lane per tile
+    constexpr int WORDS = TILE / 32;                // mask words per tile (16, 32 or 64)
+    constexpr int WPL = WORDS >= 32 ? WORDS / 32 : 1;   // mask words per lane per tile
     constexpr int LANES_PER_WORD = 32 / VEC;
 
     const RowCtx c = row_context(p);
@@ -298,7 +302,7 @@ step_vec_kernel(const __grid_constant__ StepParams p)
 #pragma unroll
         for (int i = 0; i < WPL; ++i) {
             const long long widx = (long long)tile * WORDS + i * 32 + lane;
-            mw[i] = (widx < p.tab[c.t].ldw) ? __ldg(c.mrow + widx) : 0u;
+            mw[i] = (i * 32 + lane < WORDS && widx < p.tab[c.t].ldw) ? __ldg(c.mrow + widx) : 0u;
         }
         uint4 x[kUnroll];
         float4 nz[NOISE ? kUnroll * (BF16 ? 2 : 1) : 1];
@@ -395,12 +399,10 @@ template <bool BF16>
 __global__ void __launch_bounds__(256)
 step_scalar_kernel(const __grid_constant__ StepParams p)
 {
-    constexpr int VEC = BF16 ? 8 : 4;
-    constexpr int TILE = 32 * VEC * kUnroll;
     const RowCtx c = row_context(p);
     const long long row_off = (long long)c.r * p.ld;
-    const long long begin = (long long)c.chunk * p.tiles_per_cta * TILE;
-    const int end = (int)min((long long)p.V, begin + (long long)p.tiles_per_cta * TILE);
+    const long long begin = (long long)c.chunk * p.tiles_per_cta * p.tile_tokens;
+    const int end = (int)min((long long)p.V, begin + (long long)p.tiles_per_cta * p.tile_tokens);
     Best b = {-CUDART_INF_F, -1};
     for (int i = (int)begin + threadIdx.x; i < end; i += blockDim.x)
         apply_one<BF16>(p, c, row_off, i, b);
@@ -455,7 +457,8 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
 
     const bool bf16 = a.dtype == CSTR_BF16;
     const int esz = bf16 ? 2 : 4;
-    const int tile = 32 * (bf16 ? 8 : 4) * kUnroll;
+    const int tile = 32 * (bf16 ? 8 : 4) * unroll_for(a.noise != nullptr);
+    p.tile_tokens = tile;
     const int total_tiles = (p.V + tile - 1) / tile;
     // 16 tiles (two per warp) per CTA when there is enough work to fill the
     // machine a few times over - measured best on B200: one tile per warp leaves
