@@ -36,6 +36,10 @@ POOL = 4
 BYTES_PER_LOGIT_F32_GREEDY = 4 + 4 + 1.0 / 8.0    # read + masked write + mask bit
 BYTES_PER_TRANSITION = 2 + 1.0 / 8.0              # int16 next entry + mask bit, stores only
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one full-size step launch (512 x 256,000 fp32),
+# from the ncu capture summarised in profiles/step_vec_kernel_fp32_full_size_traffic.md; set to
+# None whenever step_vec_kernel changes until the capture is repeated.
+STEP_TRAFFIC_BYTES = 993.9e6
 
 
 def parse_args():
@@ -427,9 +431,10 @@ def main():
     build_random = None
     if not args.skip_build_bench and rank == 0:
         from synth import random_range_dfa
-        rd = random_range_dfa(10000, seed=2)
+        n_rd = 10000 if args.case == "full" else 4096
+        rd = random_range_dfa(n_rd, seed=2)
         h_rd = cstr.cstr_load_dfa(*rd)
-        t_rd = cstr.cstr_table_create(vocab, 10000)
+        t_rd = cstr.cstr_table_create(vocab, n_rd)
         ms = []
         for _ in range(4):
             a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -503,14 +508,18 @@ def main():
         "gpu_launches": K,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None,
+                     "frac": achieved / peak,
+                     "traffic": STEP_TRAFFIC_BYTES if args.case == "full" else None,
                      "kernel": "step_vec_kernel<fp32, greedy>", "kernel_ms": kernel_ms,
                      "bytes_per_launch": step_bytes, "peak_kind": "of %s" % peak_kind,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "active_row_fraction_at_end": active_frac},
         "cpu_baseline": cpu,
         "table_build": [build_entry(bt, S, WORKLOAD)] +
-                       ([build_entry(build_random, 10000, "random10k_256k (DFA 0)")] if build_random else []),
+                       ([build_entry(build_random, 10000 if args.case == "full" else 4096,
+                                     "random10k_256k (DFA 0)" if args.case == "full"
+                                     else "random 4,096-state DFA (small profiling case)")]
+                        if build_random else []),
         "table_build_e2e_ms": build_e2e_ms,
         "other_workloads": others,
         "status_rows": {"bad_state": bad, "empty_mask": empty},

@@ -63,8 +63,9 @@ typedef struct cstr_workspace cstr_workspace_t; /* per-stream scratch of cstr_st
  *   trans        HOST  int32 [n_states][256], target state or -1 (no edge)
  *   accept       HOST  uint8 [n_states], non-zero = final state
  *   n_states     >= 1;  start_state in [0, n_states)
- * Validates every target, copies to the device (int16 entries when
- * n_states <= 32767, else int32) and returns the handle in *out.
+ * Validates every target, merges bytes that no state tells apart into
+ * classes, and copies the class-major table to the device (16-bit entries up
+ * to 32766 states, else 32-bit); returns the handle in *out.
  * Synchronous; allocates device memory.
  */
 int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
