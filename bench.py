@@ -85,6 +85,27 @@ def workload_inputs(case: str = "full"):
     return w, dfa, vb, vo
 
 
+def global_rows(rank: int, batch: int):
+    """Row ids of this replica: every rank decodes its own `batch` rows (weak scaling)."""
+    return range(rank * batch, rank * batch + batch)
+
+
+def reduce_max(x: float, world: int, device) -> float:
+    """Maximum of a per-rank number over all ranks (the slowest rank sets the time)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(units_per_rank_step: int, world: int, steps: int, max_ms: float) -> float:
+    """Units all ranks processed divided by the slowest rank's device time."""
+    return units_per_rank_step * world * steps / (max_ms * 1e-3)
+
+
 class ClockSampler(threading.Thread):
     """Polls SM clock, power and clock-event reasons through NVML (read-only)."""
 
@@ -324,11 +345,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max(x, world, dev)
 
     # ---- set-up: vocabulary, DFA, table (the table build is timed below) ----
     vocab = cstr.cstr_load_vocab(vb, vo)
@@ -351,7 +368,7 @@ def main():
     # ---- inputs: pinned host pool (rows keyed by global row id), device pool ----
     host_pool = [torch.empty((B, V), dtype=torch.float32).pin_memory() for _ in range(POOL)]
     for k in range(POOL):
-        normal_logits(w.logits_seed, k, range(rank * B, rank * B + B), V, out=host_pool[k].numpy())
+        normal_logits(w.logits_seed, k, global_rows(rank, B), V, out=host_pool[k].numpy())
     dev_pool = [t.to(dev, non_blocking=True) for t in host_pool]
     out_bufs = [torch.empty((B, V), dtype=torch.float32, device=dev) for _ in range(2)]
     dec = ConstrainedDecoder(table, B, device=dev)
@@ -472,7 +489,7 @@ def main():
 
     peak, peak_kind = measured_hbm_peak()
     logits_per_step = B * V * world
-    value = logits_per_step * K / (dev_ms * 1e-3)
+    value = whole_job_throughput(B * V, world, K, dev_ms)
     step_bytes = B * V * BYTES_PER_LOGIT_F32_GREEDY
     achieved = step_bytes / (kernel_ms * 1e-3) / 1e9
     bt = np.array(build_ms[1:])
