@@ -64,9 +64,23 @@ def _check_dfa(trans, accept):
     return trans, accept
 
 
+def _check_terminals(term_trans, token_sets, S, V):
+    if term_trans is None:
+        return None, 0, None
+    term_trans = np.ascontiguousarray(term_trans, dtype=np.int32)
+    assert term_trans.ndim == 2 and term_trans.shape[0] == S and term_trans.shape[1] <= 32
+    token_sets = np.ascontiguousarray(token_sets, dtype=np.uint32)
+    assert token_sets.shape == (V,)
+    return term_trans, term_trans.shape[1], token_sets
+
+
 def token_table(trans, accept, vocab_bytes, offsets, eos_id: int = -1,
-                q_lo: int = 0, q_hi: int | None = None, threads: int = 1):
-    """Returns (next int32 [q_hi-q_lo][V], mask uint32 [q_hi-q_lo][ceil(V/32)])."""
+                q_lo: int = 0, q_hi: int | None = None, threads: int = 1,
+                term_trans=None, token_sets=None):
+    """Returns (next int32 [q_hi-q_lo][V], mask uint32 [q_hi-q_lo][ceil(V/32)]).
+
+    ``term_trans`` int32 ``[S][T]`` (terminal-label edges, -1 = none) and
+    ``token_sets`` uint32 ``[V]`` (bit t: token belongs to label t) are optional."""
     lib = _load()
     trans, accept = _check_dfa(trans, accept)
     vocab_bytes = np.ascontiguousarray(vocab_bytes, dtype=np.uint8)
@@ -78,7 +92,9 @@ def token_table(trans, accept, vocab_bytes, offsets, eos_id: int = -1,
     W = (V + 31) // 32
     nxt = np.empty((q_hi - q_lo, V), dtype=np.int32)
     mask = np.empty((q_hi - q_lo, W), dtype=np.uint32)
-    lib.oracle_token_table(_ptr(trans), _ptr(accept), ctypes.c_int32(S), _ptr(vocab_bytes),
+    term_trans, n_term, token_sets = _check_terminals(term_trans, token_sets, S, V)
+    lib.oracle_token_table(_ptr(trans), _ptr(accept), ctypes.c_int32(S), _ptr(term_trans),
+                           ctypes.c_int32(n_term), _ptr(token_sets), _ptr(vocab_bytes),
                            _ptr(offsets), ctypes.c_int32(V), ctypes.c_int32(eos_id),
                            ctypes.c_int32(q_lo), ctypes.c_int32(q_hi), _ptr(nxt), _ptr(mask),
                            ctypes.c_int32(threads))
@@ -86,10 +102,12 @@ def token_table(trans, accept, vocab_bytes, offsets, eos_id: int = -1,
 
 
 def step(dfas, vocab_bytes, offsets, logits, states, noise=None, row_table=None,
-         eos_id: int = -1, vocab_size: int | None = None, threads: int = 1):
+         eos_id: int = -1, vocab_size: int | None = None, threads: int = 1,
+         term_trans=None, token_sets=None):
     """One constrained decoding step on the CPU.
 
-    dfas: list of (trans, accept[, start]).  logits: float32 ``[B][ld]`` or uint16
+    dfas: list of (trans, accept[, start]); ``term_trans``: matching list of
+    terminal-edge tables (or None), ``token_sets`` uint32 ``[V]``.  logits: float32 ``[B][ld]`` or uint16
     (bfloat16 bit patterns) ``[B][ld]``.  states: int32 ``[B]`` (not modified).
     Returns dict(tokens, states, masked, accept, bad_state_rows, empty_mask_rows);
     ``masked`` columns past the vocabulary keep the input values.
@@ -118,12 +136,20 @@ def step(dfas, vocab_bytes, offsets, logits, states, noise=None, row_table=None,
         assert noise.shape == logits.shape
     if row_table is not None:
         row_table = np.ascontiguousarray(row_table, dtype=np.int32)
+    term_ptrs, n_term, sets = None, None, None
+    if term_trans is not None:
+        terms = [np.ascontiguousarray(t, dtype=np.int32) for t in term_trans]
+        term_ptrs = TransArr(*[t.ctypes.data for t in terms])
+        n_term = np.array([t.shape[1] for t in terms], dtype=np.int32)
+        sets = np.ascontiguousarray(token_sets, dtype=np.uint32)
+        assert sets.shape == (offsets.size - 1,)
     st = np.array(states, dtype=np.int32, copy=True)
     tokens = np.empty(B, dtype=np.int32)
     masked = logits.copy()
     acc_out = np.empty(B, dtype=np.uint8)
     counters = np.zeros(2, dtype=np.int64)
-    lib.oracle_step(trans_ptrs, acc_ptrs, _ptr(n_states), ctypes.c_int32(n), _ptr(row_table),
+    lib.oracle_step(trans_ptrs, acc_ptrs, _ptr(n_states), term_ptrs, _ptr(n_term), _ptr(sets),
+                    ctypes.c_int32(n), _ptr(row_table),
                     _ptr(vocab_bytes), _ptr(offsets), ctypes.c_int32(V), ctypes.c_int32(eos_id),
                     _ptr(logits), ctypes.c_int32(dtype), ctypes.c_int64(ld), _ptr(noise),
                     _ptr(st), _ptr(tokens), _ptr(masked), _ptr(acc_out), ctypes.c_int32(B),

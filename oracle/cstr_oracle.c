@@ -14,6 +14,15 @@
  *     tokens outside A become -infinity; a token is selected; q moves along
  *     its edge.
  *
+ *   - Section 2.5.1, terminal labels: a state may also have edges labelled with
+ *     terminal labels (symbols outside the byte alphabet), each label standing
+ *     for a pre-computed set of tokens.  Such an edge allows every token of the
+ *     label's set ("terminal masks are applied en masse"); when the selected
+ *     token has no ordinary edge, the terminal edge of the first label (fixed
+ *     precedence: ascending label index) whose set holds the token is taken
+ *     ("prefer normal token edges when available, and otherwise follow a ...
+ *     precedence ordering over terminal labels").
+ *
  * Readings the paper leaves open (kept identical in the library under test):
  *   - a token of zero length never has an edge (Algorithm 1 emits the last
  *     character of every token, so it assumes |v| >= 1);
@@ -54,21 +63,47 @@ static int32_t walk_token(const int32_t *trans, int32_t q, const uint8_t *bytes,
     return s;
 }
 
+/* A DFA with optional terminal-label edges: term[q * n_term + t] = target or -1. */
+typedef struct {
+    const int32_t *trans;
+    const uint8_t *accept;
+    const int32_t *term;   /* may be NULL when n_term == 0 */
+    int32_t n_term;
+} dfa_view;
+
+/* First terminal edge of q, in label order, whose token set holds v (tmask bit). */
+static int32_t terminal_edge(const dfa_view *d, int32_t q, const uint32_t *tmask, int32_t v)
+{
+    if (d->n_term == 0 || !tmask)
+        return DEAD;
+    for (int32_t t = 0; t < d->n_term; ++t) {
+        int32_t target = d->term[(int64_t)q * d->n_term + t];
+        if (target >= 0 && ((tmask[v] >> t) & 1u))
+            return target;
+    }
+    return DEAD;
+}
+
 /* Edge of the token automaton: target state of token v from state q, or DEAD. */
-static int32_t token_edge(const int32_t *trans, const uint8_t *accept, int32_t q,
-                          const uint8_t *bytes, const int64_t *off, int32_t v, int32_t eos_id)
+static int32_t token_edge(const dfa_view *d, int32_t q, const uint8_t *bytes, const int64_t *off,
+                          const uint32_t *tmask, int32_t v, int32_t eos_id)
 {
     if (v == eos_id)
         return DEAD; /* taking EOS finishes the row; whether it is allowed is separate */
-    return walk_token(trans, q, bytes, off[v], off[v + 1]);
+    if (off[v + 1] <= off[v])
+        return DEAD; /* empty token: no edge of either kind */
+    int32_t s = walk_token(d->trans, q, bytes, off[v], off[v + 1]);
+    if (s >= 0)
+        return s;    /* ordinary edges come first */
+    return terminal_edge(d, q, tmask, v);
 }
 
-static int token_allowed(const int32_t *trans, const uint8_t *accept, int32_t q,
-                         const uint8_t *bytes, const int64_t *off, int32_t v, int32_t eos_id)
+static int token_allowed(const dfa_view *d, int32_t q, const uint8_t *bytes, const int64_t *off,
+                         const uint32_t *tmask, int32_t v, int32_t eos_id)
 {
     if (v == eos_id)
-        return accept[q] != 0;
-    return walk_token(trans, q, bytes, off[v], off[v + 1]) >= 0;
+        return d->accept[q] != 0;
+    return token_edge(d, q, bytes, off, tmask, v, eos_id) >= 0;
 }
 
 int oracle_max_threads(void)
@@ -87,11 +122,13 @@ int oracle_max_threads(void)
  * W = ceil(V / 32); unused high bits of the last word are 0.
  */
 void oracle_token_table(const int32_t *trans, const uint8_t *accept, int32_t n_states,
+                        const int32_t *term_trans, int32_t n_term, const uint32_t *tmask,
                         const uint8_t *bytes, const int64_t *off, int32_t V, int32_t eos_id,
                         int32_t q_lo, int32_t q_hi, int32_t *next_out, uint32_t *mask_out,
                         int32_t threads)
 {
     const int64_t W = ((int64_t)V + 31) / 32;
+    const dfa_view d = {trans, accept, term_trans, term_trans ? n_term : 0};
     (void)n_states;
 #pragma omp parallel for num_threads(threads) schedule(static)
     for (int32_t q = q_lo; q < q_hi; ++q) {
@@ -99,8 +136,8 @@ void oracle_token_table(const int32_t *trans, const uint8_t *accept, int32_t n_s
         uint32_t *mrow = mask_out + (int64_t)(q - q_lo) * W;
         memset(mrow, 0, (size_t)W * sizeof(uint32_t));
         for (int32_t v = 0; v < V; ++v) {
-            nrow[v] = token_edge(trans, accept, q, bytes, off, v, eos_id);
-            if (token_allowed(trans, accept, q, bytes, off, v, eos_id))
+            nrow[v] = token_edge(&d, q, bytes, off, tmask, v, eos_id);
+            if (token_allowed(&d, q, bytes, off, tmask, v, eos_id))
                 mrow[v >> 5] |= (uint32_t)1 << (v & 31);
         }
     }
@@ -118,7 +155,9 @@ static float bf16_to_float(uint16_t b)
  * One constrained decoding step for `batch` rows (Algorithm 2, loop body).
  *
  * tables: n_tables DFAs given as arrays of pointers (trans[t], accept[t],
- * n_states[t]); row r uses table row_table[r] (or 0 when row_table is NULL).
+ * n_states[t], and optionally term_trans[t] with n_term[t] labels; tmask[v] has
+ * bit t set iff token v belongs to the set of label t); row r uses table
+ * row_table[r] (or 0 when row_table is NULL).
  * logits: [batch][ld] fp32 (dtype 0) or bf16 bit patterns (dtype 1);
  * noise: [batch][ld] fp32 or NULL.  masked_out: same shape/dtype as logits,
  * columns >= V are not written.  states: in/out.  counters[0] += rows whose
@@ -126,7 +165,9 @@ static float bf16_to_float(uint16_t b)
  * selectable token.
  */
 void oracle_step(const int32_t *const *trans, const uint8_t *const *accept,
-                 const int32_t *n_states, int32_t n_tables, const int32_t *row_table,
+                 const int32_t *n_states, const int32_t *const *term_trans,
+                 const int32_t *n_term, const uint32_t *tmask, int32_t n_tables,
+                 const int32_t *row_table,
                  const uint8_t *bytes, const int64_t *off, int32_t V, int32_t eos_id,
                  const void *logits, int32_t dtype, int64_t ld, const float *noise,
                  int32_t *states, int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
@@ -145,10 +186,17 @@ void oracle_step(const int32_t *const *trans, const uint8_t *const *accept,
         int active = (t >= 0 && t < n_tables && q >= 0 && q < n_states[t]);
         if (!active && q != -1)
             bad += 1;
+        dfa_view d = {0, 0, 0, 0};
+        if (active) {
+            d.trans = trans[t];
+            d.accept = accept[t];
+            d.term = term_trans ? term_trans[t] : 0;
+            d.n_term = (term_trans && term_trans[t]) ? n_term[t] : 0;
+        }
         float best = -INFINITY;
         int32_t best_v = -1;
         for (int32_t v = 0; v < V; ++v) {
-            int ok = active && token_allowed(trans[t], accept[t], q, bytes, off, v, eos_id);
+            int ok = active && token_allowed(&d, q, bytes, off, tmask, v, eos_id);
             if (!ok) {
                 if (dtype == 0)
                     of[v] = -INFINITY;
@@ -178,7 +226,7 @@ void oracle_step(const int32_t *const *trans, const uint8_t *const *accept,
         tokens_out[r] = best_v;
         int32_t q2 = DEAD;
         if (best_v >= 0)
-            q2 = token_edge(trans[t], accept[t], q, bytes, off, best_v, eos_id);
+            q2 = token_edge(&d, q, bytes, off, tmask, best_v, eos_id);
         states[r] = q2;
         if (accept_out)
             accept_out[r] = (q2 >= 0) ? (accept[t][q2] != 0) : 0;

@@ -39,9 +39,14 @@ _CHAR_ESCAPES = {"n": 10, "t": 9, "r": 13, "f": 12, "v": 11, "0": 0}
 _EVERY = frozenset(range(256))
 
 
-def parse(pattern: str):
+def parse(pattern: str, terminals=()):
+    """``terminals``: names of terminal labels; the empty named group
+    ``(?P<NAME>)`` stands for one edge labelled with symbol 256 + index of NAME
+    (Section 2.5.1: a terminal label is an input symbol outside the byte
+    alphabet, later matched by any token of a pre-computed set)."""
     pos = 0
     n = len(pattern)
+    terminals = list(terminals)
 
     def fail(msg):
         raise ValueError("bad regex %r at %d: %s" % (pattern, pos, msg))
@@ -102,6 +107,13 @@ def parse(pattern: str):
         ch = pattern[pos]
         pos += 1
         if ch == "(":
+            if pattern.startswith("?P<", pos):
+                close = pattern.find(">)", pos)
+                name = pattern[pos + 3:close] if close >= 0 else None
+                if name is None or name not in terminals:
+                    fail("unknown terminal label")
+                pos = close + 2
+                return ("set", frozenset([256 + terminals.index(name)]))
             if pattern.startswith("?:", pos):
                 pos += 2
             elif pos < n and pattern[pos] == "?":
@@ -282,8 +294,9 @@ def _closure(nfa: NFA, states):
 # subset construction
 # --------------------------------------------------------------------------
 
-def determinize(nfa: NFA):
-    """Returns (trans int32 [S][256] with -1 for "no edge", accept uint8 [S], start=0).
+def determinize(nfa: NFA, n_symbols: int = 256):
+    """Returns (trans int32 [S][n_symbols] with -1 for "no edge", accept uint8 [S], start=0).
+    Symbols 256.. are terminal labels.
 
     DFA states are epsilon-closed sets of NFA states, discovered breadth-first
     with bytes ascending.  Bytes that no edge label tells apart behave alike, so
@@ -294,7 +307,7 @@ def determinize(nfa: NFA):
     signature = {}
     group_of = []
     group_first = []
-    for b in range(256):
+    for b in range(n_symbols):
         sig = tuple(b in label for label in labels)
         if sig not in signature:
             signature[sig] = len(group_first)
@@ -324,15 +337,15 @@ def determinize(nfa: NFA):
                 ids[target] = len(order)
                 order.append(target)
             row_by_group.append(ids[target])
-        rows.append([row_by_group[group_of[b]] for b in range(256)])
-    trans = np.array(rows, dtype=np.int32).reshape(len(order), 256)
+        rows.append([row_by_group[group_of[b]] for b in range(n_symbols)])
+    trans = np.array(rows, dtype=np.int32).reshape(len(order), n_symbols)
     accept = np.array([nfa.final in s for s in order], dtype=np.uint8)
     return trans, accept, 0
 
 
 def trim(trans: np.ndarray, accept: np.ndarray, start: int):
     """Remove states that cannot reach an accepting state; renumber breadth-first."""
-    S = trans.shape[0]
+    S, A = trans.shape
     # backward reachability from the accepting states over reversed edges
     preds = [set() for _ in range(S)]
     for q in range(S):
@@ -347,30 +360,37 @@ def trim(trans: np.ndarray, accept: np.ndarray, start: int):
                 useful[q] = True
                 stack.append(q)
     if not useful[start]:
-        return np.full((1, 256), -1, dtype=np.int32), np.zeros(1, dtype=np.uint8), 0
+        return np.full((1, A), -1, dtype=np.int32), np.zeros(1, dtype=np.uint8), 0
     new_id = {start: 0}
     order = [start]
     head = 0
     while head < len(order):
         q = order[head]
         head += 1
-        for b in range(256):
+        for b in range(A):
             t = int(trans[q, b])
             if t >= 0 and useful[t] and t not in new_id:
                 new_id[t] = len(order)
                 order.append(t)
-    out = np.full((len(order), 256), -1, dtype=np.int32)
+    out = np.full((len(order), A), -1, dtype=np.int32)
     for i, q in enumerate(order):
-        for b in range(256):
+        for b in range(A):
             t = int(trans[q, b])
             if t >= 0 and useful[t]:
                 out[i, b] = new_id[t]
     return out, accept[order].astype(np.uint8), 0
 
 
-def compile_regex(pattern: str):
-    """regex -> Thompson NFA -> subset construction -> trim."""
-    return trim(*determinize(thompson(parse(pattern))))
+def compile_regex(pattern: str, terminals=()):
+    """regex -> Thompson NFA -> subset construction -> trim.  With terminal
+    labels the table has 256 + len(terminals) columns (split_terminals)."""
+    return trim(*determinize(thompson(parse(pattern, terminals)), 256 + len(terminals)))
+
+
+def split_terminals(trans):
+    """(byte transitions [S][256], terminal transitions [S][T])."""
+    trans = np.asarray(trans)
+    return np.ascontiguousarray(trans[:, :256]), np.ascontiguousarray(trans[:, 256:])
 
 
 def dfa_accepts(trans, accept, start, data: bytes) -> bool:
@@ -393,7 +413,7 @@ def dfa_equivalent(a, b) -> bool:
         qa = bool(ab[q]) if q >= 0 else False
         if pa != qa:
             return False
-        for byte in range(256):
+        for byte in range(ta.shape[1]):
             np_ = int(ta[p, byte]) if p >= 0 else -1
             nq = int(tb[q, byte]) if q >= 0 else -1
             if np_ < 0 and nq < 0:
