@@ -72,6 +72,23 @@ int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
                   int32_t start_state, cstr_dfa_t **out);
 void cstr_free_dfa(cstr_dfa_t *dfa);
 
+/*
+ * As cstr_load_dfa, for an automaton that also has edges labelled with
+ * terminal labels (Section 2.5.1, "Wildcard matching"): symbols outside the
+ * byte alphabet, each standing for a pre-computed set of tokens, written
+ * (?P<NAME>) in a regex.
+ *   term_trans   HOST  int32 [n_states][n_labels], target state or -1
+ *   n_labels     0..32; label t is bit t of the token sets given to
+ *                cstr_vocab_set_token_sets
+ * In the built table a state's terminal edges allow every token of their
+ * labels' sets on top of the ordinary tokens ("applied en masse"); a selected
+ * token follows its ordinary edge if it has one, else the terminal edge of the
+ * lowest label whose set holds it (the paper's precedence heuristic).
+ */
+int cstr_load_dfa_terminals(const int32_t *trans, const int32_t *term_trans, int32_t n_labels,
+                            const uint8_t *accept, int32_t n_states, int32_t start_state,
+                            cstr_dfa_t **out);
+
 /* ---------------------------------------------------------------- vocab */
 
 /*
@@ -91,6 +108,18 @@ int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offsets, int32_t 
                     cstr_vocab_t **out);
 void cstr_free_vocab(cstr_vocab_t *vocab);
 
+/*
+ * Attach the token sets of the terminal labels to a vocabulary (Section 2.5.1:
+ * "terminal labels ... map to pre-computed masks of valid tokens", e.g. the
+ * newline-free tokens for PARAGRAPH_TOKEN).  Prepared once per LM.
+ *   token_sets   HOST  uint32 [vocab_size]; bit t set iff the token belongs to
+ *                the set of label t
+ *   n_labels     1..32
+ * Replaces any sets attached before.  Synchronous; allocates device memory.
+ * Tokens of length 0 never match a label.
+ */
+int cstr_vocab_set_token_sets(cstr_vocab_t *vocab, const uint32_t *token_sets, int32_t n_labels);
+
 /* ---------------------------------------------------------------- table */
 
 /*
@@ -109,6 +138,9 @@ int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states, cstr_table_
  *                  bits of the last word are 0
  * If eos_id >= 0, that token's bytes are ignored: it is allowed exactly in
  * accepting states and leads to -1 ("finished").
+ * A DFA loaded with terminal labels needs a vocabulary with token sets for at
+ * least as many labels (else CSTR_ERR_SHAPE); its terminal edges are merged
+ * into mask and next as described at cstr_load_dfa_terminals.
  * Only enqueues kernels on cuda_stream: no allocation, no host synchronisation.
  * The table may be rebuilt any number of times (dfa->n_states <= max_states);
  * it must not be in use by a cstr_step that has not completed.

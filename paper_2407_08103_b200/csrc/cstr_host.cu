@@ -42,6 +42,9 @@ extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
     cudaFree(dfa->tt);
     cudaFree(dfa->cls);
     cudaFree(dfa->accept);
+    cudaFree(dfa->tstate);
+    cudaFree(dfa->tset);
+    cudaFree(dfa->ttarget);
     delete dfa;
 }
 
@@ -154,7 +157,104 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     return CSTR_OK;
 }
 
+extern "C" int cstr_load_dfa_terminals(const int32_t *trans, const int32_t *term_trans,
+                                       int32_t n_labels, const uint8_t *accept, int32_t n_states,
+                                       int32_t start_state, cstr_dfa_t **out)
+{
+    if (!out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_dfa_terminals: null pointer");
+    *out = nullptr;
+    if (n_labels < 0 || n_labels > 32)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa_terminals: n_labels = %d, need 0..32",
+                         n_labels);
+    if (n_labels > 0 && !term_trans)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_dfa_terminals: null term_trans");
+    if (n_states >= 1) {
+        for (int64_t i = 0; i < (int64_t)n_states * n_labels; ++i) {
+            if (term_trans[i] < -1 || term_trans[i] >= n_states)
+                return cstr_fail(CSTR_ERR_DFA,
+                                 "cstr_load_dfa_terminals: state %lld label %lld has target %d "
+                                 "outside [-1, %d)", (long long)(i / n_labels),
+                                 (long long)(i % n_labels), term_trans[i], n_states);
+        }
+    }
+    cstr_dfa *d = nullptr;
+    int rc = cstr_load_dfa(trans, accept, n_states, start_state, &d);
+    if (rc)
+        return rc;
+    d->n_labels = n_labels;
+    std::vector<int32_t> tstate;
+    std::vector<uint32_t> tset, ttarget;
+    try {
+        for (int32_t q = 0; q < n_states && n_labels > 0; ++q) {
+            uint32_t labels = 0;
+            for (int32_t t = 0; t < n_labels; ++t)
+                if (term_trans[(int64_t)q * n_labels + t] >= 0)
+                    labels |= 1u << t;
+            if (!labels)
+                continue;
+            tstate.push_back(q);
+            tset.push_back(labels);
+            for (int32_t t = 0; t < n_labels; ++t) {
+                const int32_t target = term_trans[(int64_t)q * n_labels + t];
+                const uint32_t code = (uint32_t)CSTR_PERM(target < 0 ? n_states : target)
+                                      << (d->wide ? 2 : 1);
+                ttarget.push_back(code);
+            }
+        }
+    } catch (const std::bad_alloc &) {
+        cstr_free_dfa(d);
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa_terminals: out of host memory");
+    }
+    d->n_term_states = (int32_t)tstate.size();
+    if (d->n_term_states > 0) {
+        cudaError_t e = cudaMalloc((void **)&d->tstate, tstate.size() * 4);
+        if (e == cudaSuccess)
+            e = cudaMalloc((void **)&d->tset, tset.size() * 4);
+        if (e == cudaSuccess)
+            e = cudaMalloc((void **)&d->ttarget, ttarget.size() * 4);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->tstate, tstate.data(), tstate.size() * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->tset, tset.data(), tset.size() * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->ttarget, ttarget.data(), ttarget.size() * 4, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                           "cstr_load_dfa_terminals: %s", cudaGetErrorString(e));
+            cstr_free_dfa(d);
+            return rc;
+        }
+    }
+    *out = d;
+    return CSTR_OK;
+}
+
 // ---------------------------------------------------------------- vocab
+
+extern "C" int cstr_vocab_set_token_sets(cstr_vocab_t *vocab, const uint32_t *token_sets,
+                                         int32_t n_labels)
+{
+    if (!vocab || !token_sets)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_vocab_set_token_sets: null pointer");
+    if (n_labels < 1 || n_labels > 32)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_vocab_set_token_sets: n_labels = %d, need 1..32",
+                         n_labels);
+    int rc = check_device(vocab->device, "vocabulary");
+    if (rc)
+        return rc;
+    uint32_t *dev = nullptr;
+    CSTR_CUDA_TRY(cudaMalloc((void **)&dev, (size_t)vocab->V * 4));
+    cudaError_t e = cudaMemcpy(dev, token_sets, (size_t)vocab->V * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(dev);
+        return cstr_fail(CSTR_ERR_CUDA, "cstr_vocab_set_token_sets: %s", cudaGetErrorString(e));
+    }
+    cudaFree(vocab->tsets);
+    vocab->tsets = dev;
+    vocab->n_labels = n_labels;
+    return CSTR_OK;
+}
 
 extern "C" void cstr_free_vocab(cstr_vocab_t *v)
 {
@@ -163,6 +263,7 @@ extern "C" void cstr_free_vocab(cstr_vocab_t *v)
     cudaFree(v->bytes);
     cudaFree(v->off);
     cudaFree(v->desc);
+    cudaFree(v->tsets);
     delete v;
 }
 
@@ -356,6 +457,11 @@ extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int3
     if (dfa->n_states > table->max_states)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA has %d states, table holds %d",
                          dfa->n_states, table->max_states);
+    if (dfa->n_term_states > 0 && table->vocab->n_labels < dfa->n_labels)
+        return cstr_fail(CSTR_ERR_SHAPE,
+                         "cstr_table_build: the DFA uses %d terminal labels, the vocabulary has "
+                         "token sets for %d (cstr_vocab_set_token_sets)", dfa->n_labels,
+                         table->vocab->n_labels);
     if (eos_id < -1 || eos_id >= table->V)
         return cstr_fail(CSTR_ERR_ARG, "cstr_table_build: eos_id %d outside [-1, %d)", eos_id,
                          table->V);

@@ -45,6 +45,12 @@ struct cstr_dfa {
     void *tt;            // DEVICE [n_classes][row]
     uint8_t *cls;        // DEVICE [256] byte -> class
     uint8_t *accept;     // DEVICE [n_states]
+    // terminal-label edges, kept only for the states that have any
+    int32_t n_labels;
+    int32_t n_term_states;
+    int32_t *tstate;     // DEVICE [n_term_states] state ids
+    uint32_t *tset;      // DEVICE [n_term_states] labels with an edge (bit set)
+    uint32_t *ttarget;   // DEVICE [n_term_states][n_labels] target codes
 };
 
 // Vocabulary as the builder reads it: tokens in lexicographic (trie depth-first)
@@ -63,6 +69,8 @@ struct cstr_vocab {
     uint32_t *off;     // DEVICE [V + 1]
     uint4 *desc;       // DEVICE [V], sorted order
     uint32_t max_len;
+    int32_t n_labels;  // terminal labels with a token set (0 = none attached)
+    uint32_t *tsets;   // DEVICE [V] bit t: token belongs to label t's set
 };
 
 // Token table.  next is token-major: next[v][q] (a step reads one entry per

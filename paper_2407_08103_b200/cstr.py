@@ -21,7 +21,8 @@ CSTR_MAX_TABLES = 16
 CSTR_STATIC_MAX_BATCH = 4096
 
 EXPORTS = [
-    "cstr_load_dfa", "cstr_free_dfa", "cstr_load_vocab", "cstr_free_vocab",
+    "cstr_load_dfa", "cstr_load_dfa_terminals", "cstr_free_dfa", "cstr_load_vocab",
+    "cstr_vocab_set_token_sets", "cstr_free_vocab",
     "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
     "cstr_step", "cstr_step_status", "cstr_step_static", "cstr_last_error",
@@ -122,13 +123,40 @@ def cstr_load_dfa(trans, accept, start_state=0) -> Dfa:
     return Dfa(out)
 
 
+def cstr_load_dfa_terminals(trans, term_trans, accept, start_state=0) -> Dfa:
+    """``trans`` int32 ``[S][256]``, ``term_trans`` int32 ``[S][n_labels]`` (terminal-label edges)."""
+    trans = np.ascontiguousarray(trans, dtype=np.int32)
+    term_trans = np.ascontiguousarray(term_trans, dtype=np.int32)
+    accept = np.ascontiguousarray(accept, dtype=np.uint8)
+    if trans.ndim != 2 or trans.shape[1] != 256 or accept.shape != (trans.shape[0],):
+        raise ValueError("trans must be [S][256] and accept [S]")
+    if term_trans.ndim != 2 or term_trans.shape[0] != trans.shape[0]:
+        raise ValueError("term_trans must be [S][n_labels]")
+    out = ctypes.c_void_p()
+    _check(lib().cstr_load_dfa_terminals(_np_ptr(trans), _np_ptr(term_trans),
+                                         ctypes.c_int32(term_trans.shape[1]), _np_ptr(accept),
+                                         ctypes.c_int32(trans.shape[0]),
+                                         ctypes.c_int32(start_state), ctypes.byref(out)))
+    return Dfa(out)
+
+
+def cstr_vocab_set_token_sets(vocab: Vocab, token_sets, n_labels: int) -> None:
+    """``token_sets`` uint32 ``[V]``: bit t set iff the token belongs to terminal label t's set."""
+    token_sets = np.ascontiguousarray(token_sets, dtype=np.uint32)
+    if token_sets.shape != (vocab.size,):
+        raise ValueError("token_sets must have one uint32 per token")
+    _check(lib().cstr_vocab_set_token_sets(vocab.ptr, _np_ptr(token_sets), ctypes.c_int32(n_labels)))
+
+
 def cstr_load_vocab(vocab_bytes, offsets) -> Vocab:
     vocab_bytes = np.ascontiguousarray(vocab_bytes, dtype=np.uint8)
     offsets = np.ascontiguousarray(offsets, dtype=np.int64)
     out = ctypes.c_void_p()
     _check(lib().cstr_load_vocab(_np_ptr(vocab_bytes), _np_ptr(offsets),
                                  ctypes.c_int32(offsets.size - 1), ctypes.byref(out)))
-    return Vocab(out)
+    v = Vocab(out)
+    v.size = int(offsets.size - 1)
+    return v
 
 
 def cstr_table_create(vocab: Vocab, max_states: int) -> Table:

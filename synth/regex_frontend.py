@@ -151,10 +151,11 @@ class _Terms:
 
 
 class _Parser:
-    def __init__(self, pattern: str, terms: _Terms):
+    def __init__(self, pattern: str, terms: _Terms, terminals=()):
         self.p = pattern
         self.i = 0
         self.T = terms
+        self.terminals = list(terminals)
 
     def error(self, msg):
         raise ValueError("regex error at %d in %r: %s" % (self.i, self.p, msg))
@@ -273,6 +274,14 @@ class _Parser:
         ch = self.peek()
         self.i += 1
         if ch == "(":
+            if self.p.startswith("?P<", self.i):
+                # empty named group = one edge carrying a terminal label (symbol 256 + index)
+                j = self.p.find(">)", self.i)
+                name = self.p[self.i + 3:j] if j >= 0 else None
+                if name is None or name not in self.terminals:
+                    self.error("unknown terminal label")
+                self.i = j + 2
+                return self.T.set(1 << (256 + self.terminals.index(name)))
             if self.p.startswith("?:", self.i):
                 self.i += 2
             elif self.peek() == "?":
@@ -293,13 +302,13 @@ class _Parser:
         return self.T.set(1 << self.byte_of(ch))
 
 
-def _byte_classes(terms: _Terms):
-    """Partition 0..255 into classes no byte set of the regex tells apart."""
+def _byte_classes(terms: _Terms, n_symbols: int = 256):
+    """Partition the symbols into classes no symbol set of the regex tells apart."""
     sets = sorted({node[1] for node in terms.t if node[0] == "set"})
     sig = {}
-    cls = np.zeros(256, dtype=np.int32)
+    cls = np.zeros(n_symbols, dtype=np.int32)
     reps = []
-    for b in range(256):
+    for b in range(n_symbols):
         s = tuple((m >> b) & 1 for m in sets)
         if s not in sig:
             sig[s] = len(reps)
@@ -398,11 +407,15 @@ def _trim_merge_renumber(tc: np.ndarray, acc: np.ndarray, start: int):
     return np.stack(rows), out_acc, 0
 
 
-def regex_to_dfa(pattern: str):
-    """Compile ``pattern`` to ``(trans int32 [S][256], accept uint8 [S], start)``."""
+def regex_to_dfa(pattern: str, terminals=()):
+    """Compile ``pattern`` to ``(trans int32 [S][256 + len(terminals)], accept uint8 [S], start)``.
+
+    ``terminals`` names the terminal labels the pattern may use as empty named
+    groups ``(?P<NAME>)`` (the paper's wildcard extension, Section 2.5.1); label
+    ``i`` is symbol ``256 + i``, its column holds the terminal edges."""
     T = _Terms()
-    root = _Parser(pattern, T).parse()
-    cls, reps = _byte_classes(T)
+    root = _Parser(pattern, T, terminals).parse()
+    cls, reps = _byte_classes(T, 256 + len(list(terminals)))
     # classes are numbered by their smallest byte, so class order == byte order
     index = {root: 0}
     queue = [root]

@@ -29,11 +29,17 @@ def bits_equal(a, b):
     return np.array_equal(a, b)
 
 
-def gpu_tables(dfas, vb, vo, eos_id=-1):
+def gpu_tables(dfas, vb, vo, eos_id=-1, term_trans=None, token_sets=None):
     vocab = cstr.cstr_load_vocab(vb, vo)
+    if token_sets is not None:
+        n_labels = max(max(t.shape[1] for t in term_trans), 1)
+        cstr.cstr_vocab_set_token_sets(vocab, token_sets, n_labels)
     tables = []
-    for d in dfas:
-        h = cstr.cstr_load_dfa(d[0], d[1], d[2])
+    for i, d in enumerate(dfas):
+        if term_trans is not None:
+            h = cstr.cstr_load_dfa_terminals(d[0], term_trans[i], d[1], d[2])
+        else:
+            h = cstr.cstr_load_dfa(d[0], d[1], d[2])
         t = cstr.cstr_table_create(vocab, d[0].shape[0])
         cstr.cstr_table_build(t, h, eos_id)
         tables.append(t)
@@ -41,7 +47,8 @@ def gpu_tables(dfas, vb, vo, eos_id=-1):
     return tables
 
 
-def check_table(table, dfa, vb, vo, states=None, eos_id=-1, slab=64, threads=None):
+def check_table(table, dfa, vb, vo, states=None, eos_id=-1, slab=64, threads=None,
+                term_trans=None, token_sets=None):
     """Compare downloaded rows of a built table with the oracle's, slab by slab."""
     threads = threads or min(oracle.max_threads(), 32)
     S = dfa[0].shape[0]
@@ -55,13 +62,14 @@ def check_table(table, dfa, vb, vo, states=None, eos_id=-1, slab=64, threads=Non
     for lo, hi in ranges:
         nxt, mask = cstr.cstr_table_download(table, lo, hi)
         o_next, o_mask = oracle.token_table(dfa[0], dfa[1], vb, vo, eos_id=eos_id, q_lo=lo, q_hi=hi,
-                                            threads=threads)
+                                            threads=threads, term_trans=term_trans,
+                                            token_sets=token_sets)
         assert np.array_equal(nxt, o_next), "next-state rows %d..%d differ" % (lo, hi)
         assert np.array_equal(mask, o_mask), "mask rows %d..%d differ" % (lo, hi)
 
 
 def run_step_both(dfas, tables, vb, vo, logits, states, noise=None, row_table=None, eos_id=-1,
-                  ws=None, in_place=False, accept=True):
+                  ws=None, in_place=False, accept=True, term_trans=None, token_sets=None):
     """One step on the GPU and on the oracle; asserts bit equality of every output."""
     B = logits.shape[0]
     ws = ws or cstr.cstr_workspace_create(B)
@@ -78,7 +86,8 @@ def run_step_both(dfas, tables, vb, vo, logits, states, noise=None, row_table=No
     bad, empty = cstr.cstr_step_status(ws)
     ref = oracle.step(dfas, vb, vo, logits, states, noise=noise, row_table=row_table,
                       eos_id=eos_id, vocab_size=vo.size - 1,
-                      threads=min(oracle.max_threads(), 32))
+                      threads=min(oracle.max_threads(), 32), term_trans=term_trans,
+                      token_sets=token_sets)
     V = vo.size - 1
     assert np.array_equal(d_tokens.cpu().numpy(), ref["tokens"])
     assert np.array_equal(d_states.cpu().numpy(), ref["states"])
