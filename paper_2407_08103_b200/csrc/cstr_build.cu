@@ -419,10 +419,13 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     // warp's share should be long; but there must be enough CTAs for the machine.
     int dev_sms = 148;
     cudaDeviceGetAttribute(&dev_sms, cudaDevAttrMultiProcessorCount, t->device);
-    const long long want_ctas = 8LL * dev_sms;
+    const long long want_ctas = (table_bytes <= 16 * 1024 && in_smem ? 32LL : 8LL) * dev_sms;
     long long chunks = (want_ctas + state_groups - 1) / state_groups;
     long long tokens_per_cta = (t->V + chunks - 1) / chunks;
-    const long long min_tokens = (long long)warps_t * (in_smem ? 256 : 128);
+    // (a CTA re-stages the table, so big tables want long chunks; small automata
+    // are latency-bound per token and want many short ones)
+    const long long min_tokens =
+        (long long)warps_t * (!in_smem ? 128 : (table_bytes <= 16 * 1024 ? 32 : 256));
     if (tokens_per_cta < min_tokens)
         tokens_per_cta = min_tokens;
     chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
