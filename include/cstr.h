@@ -216,6 +216,45 @@ int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t
               int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
 
 /*
+ * cstr_step that leaves the input states untouched and writes the new ones to
+ * states_out, so that a caller can keep "a full history of states instead of
+ * just one" (Section 4, Speculative decoding: the constraint must be
+ * rewindable because the target model may reject drafted tokens).
+ *   states_in   DEVICE int32 [batch]
+ *   states_out  DEVICE int32 [batch]; may equal states_in (then it is cstr_step)
+ * Everything else as in cstr_step.  The same call, over batch x (k + 1) rows
+ * whose states are the draft's history q_0 .. q_k of each sequence, penalises
+ * the target model's logits at all drafted positions at once with the masks
+ * the draft used ("sharing the penalties with the target model") and decodes
+ * the target's own token and next state at each position.
+ */
+int cstr_step_history(const cstr_table_t *const *tables, int32_t n_tables,
+                      const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
+                      const float *noise, const int32_t *states_in, int32_t *states_out,
+                      int32_t *tokens_out, void *masked_out, uint8_t *accept_out, int32_t batch,
+                      cstr_workspace_t *ws, void *cuda_stream);
+
+/*
+ * Greedy verification and rewind for speculative decoding (Section 4): keep
+ * the drafted tokens up to the first position where the target model's token
+ * differs, take the target's token there, and rewind the constraint to the
+ * state that follows it.
+ *   draft_tokens   DEVICE int32 [batch][k]      tokens of the approximation model
+ *   target_tokens  DEVICE int32 [batch][k + 1]  target's token at each drafted position
+ *                  (and one past the last), from cstr_step_history
+ *   target_states  DEVICE int32 [batch][k + 1]  target's next state at each position
+ *   n_accepted     DEVICE int32 [batch]         n = drafted tokens kept (0..k)
+ *   out_tokens     DEVICE int32 [batch][k + 1]  target_tokens[0..n], then -1
+ *   states         DEVICE int32 [batch]         target_states[n]: the rewound state
+ * The emitted sequence equals what constrained greedy decoding with the
+ * target model alone would produce.  Only enqueues one small kernel.
+ */
+int cstr_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,
+                      const int32_t *target_states, int32_t k, int32_t batch,
+                      int32_t *n_accepted, int32_t *out_tokens, int32_t *states,
+                      void *cuda_stream);
+
+/*
  * Rows since the last call whose input state or table index was out of range
  * (not counting -1), and active rows that had no selectable token.
  * Synchronises cuda_stream, then resets both counters.  Either pointer may be NULL.

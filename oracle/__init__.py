@@ -46,6 +46,7 @@ def _load():
         _lib.oracle_max_threads.restype = ctypes.c_int
         _lib.oracle_token_table.restype = None
         _lib.oracle_step.restype = None
+        _lib.oracle_accept_draft.restype = None
     return _lib
 
 
@@ -156,3 +157,21 @@ def step(dfas, vocab_bytes, offsets, logits, states, noise=None, row_table=None,
                     _ptr(counters), ctypes.c_int32(threads))
     return dict(tokens=tokens, states=st, masked=masked, accept=acc_out,
                 bad_state_rows=int(counters[0]), empty_mask_rows=int(counters[1]))
+
+
+def accept_draft(draft_tokens, target_tokens, target_states):
+    """Greedy verification + rewind.  int32 arrays ``[B][k]``, ``[B][k+1]``, ``[B][k+1]``;
+    returns (n_accepted [B], out_tokens [B][k+1], states [B])."""
+    lib = _load()
+    target_tokens = np.ascontiguousarray(target_tokens, dtype=np.int32)
+    target_states = np.ascontiguousarray(target_states, dtype=np.int32)
+    B, k1 = target_tokens.shape
+    draft_tokens = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(B, k1 - 1)
+    assert target_states.shape == (B, k1)
+    n_acc = np.empty(B, dtype=np.int32)
+    out = np.empty((B, k1), dtype=np.int32)
+    st = np.empty(B, dtype=np.int32)
+    lib.oracle_accept_draft(_ptr(draft_tokens), _ptr(target_tokens), _ptr(target_states),
+                            ctypes.c_int32(k1 - 1), ctypes.c_int32(B), _ptr(n_acc), _ptr(out),
+                            _ptr(st))
+    return n_acc, out, st

@@ -234,3 +234,31 @@ void oracle_step(const int32_t *const *trans, const uint8_t *const *accept,
     counters[0] += bad;
     counters[1] += empty;
 }
+
+/*
+ * Speculative decoding, greedy verification and rewind (Section 4): the target
+ * model accepts a prefix of the drafted tokens; the constraint, which tracked
+ * "a full history of states instead of just one", restarts from the state that
+ * follows the last token kept.  With greedy selection the kept prefix is the
+ * run of positions where the target's own (constrained) token equals the
+ * drafted one, and the target's token at the first disagreement (or after the
+ * last drafted position) is emitted as well.
+ *   draft[b][k], tgt_tok[b][k+1], tgt_state[b][k+1] ->
+ *   n_accepted[b], out_tokens[b][k+1] (tgt_tok[0..n], then -1), states[b] = tgt_state[n]
+ */
+void oracle_accept_draft(const int32_t *draft, const int32_t *tgt_tok, const int32_t *tgt_state,
+                         int32_t k, int32_t batch, int32_t *n_accepted, int32_t *out_tokens,
+                         int32_t *states)
+{
+    for (int32_t r = 0; r < batch; ++r) {
+        const int32_t *d = draft + (int64_t)r * k;
+        const int32_t *t = tgt_tok + (int64_t)r * (k + 1);
+        int32_t n = 0;
+        while (n < k && d[n] == t[n])
+            n += 1;
+        for (int32_t i = 0; i <= k; ++i)
+            out_tokens[(int64_t)r * (k + 1) + i] = (i <= n) ? t[i] : -1;
+        n_accepted[r] = n;
+        states[r] = tgt_state[(int64_t)r * (k + 1) + n];
+    }
+}

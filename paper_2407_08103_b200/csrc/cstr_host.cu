@@ -620,13 +620,13 @@ extern "C" int cstr_workspace_create(int32_t max_batch, cstr_workspace_t **out)
 
 // ----------------------------------------------------------------- step
 
-extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
-                         const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
-                         const float *noise, int32_t *states, int32_t *tokens_out,
-                         void *masked_out, uint8_t *accept_out, int32_t batch,
-                         cstr_workspace_t *ws, void *cuda_stream)
+static int step_common(const cstr_table_t *const *tables, int32_t n_tables,
+                       const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
+                       const float *noise, const int32_t *states, int32_t *states_out,
+                       int32_t *tokens_out, void *masked_out, uint8_t *accept_out, int32_t batch,
+                       cstr_workspace_t *ws, void *cuda_stream)
 {
-    if (!tables || !logits || !states || !tokens_out || !masked_out || !ws)
+    if (!tables || !logits || !states || !states_out || !tokens_out || !masked_out || !ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_step: null pointer");
     if (n_tables < 1 || n_tables > CSTR_MAX_TABLES)
         return cstr_fail(CSTR_ERR_ARG, "cstr_step: n_tables = %d, need 1..%d", n_tables,
@@ -668,6 +668,7 @@ extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
     a.ld = ld;
     a.noise = noise;
     a.states = states;
+    a.states_out = states_out;
     a.tokens_out = tokens_out;
     a.masked_out = masked_out;
     a.accept_out = accept_out;
@@ -677,6 +678,43 @@ extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
     a.counters = ws->counters;
     a.device = ws->device;
     return cstr_launch_step(a, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int cstr_step(const cstr_table_t *const *tables, int32_t n_tables,
+                         const int32_t *row_table, const void *logits, int32_t dtype, int64_t ld,
+                         const float *noise, int32_t *states, int32_t *tokens_out,
+                         void *masked_out, uint8_t *accept_out, int32_t batch,
+                         cstr_workspace_t *ws, void *cuda_stream)
+{
+    return step_common(tables, n_tables, row_table, logits, dtype, ld, noise, states, states,
+                       tokens_out, masked_out, accept_out, batch, ws, cuda_stream);
+}
+
+extern "C" int cstr_step_history(const cstr_table_t *const *tables, int32_t n_tables,
+                                 const int32_t *row_table, const void *logits, int32_t dtype,
+                                 int64_t ld, const float *noise, const int32_t *states_in,
+                                 int32_t *states_out, int32_t *tokens_out, void *masked_out,
+                                 uint8_t *accept_out, int32_t batch, cstr_workspace_t *ws,
+                                 void *cuda_stream)
+{
+    return step_common(tables, n_tables, row_table, logits, dtype, ld, noise, states_in,
+                       states_out, tokens_out, masked_out, accept_out, batch, ws, cuda_stream);
+}
+
+extern "C" int cstr_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,
+                                 const int32_t *target_states, int32_t k, int32_t batch,
+                                 int32_t *n_accepted, int32_t *out_tokens, int32_t *states,
+                                 void *cuda_stream)
+{
+    if (!target_tokens || !target_states || !n_accepted || !out_tokens || !states ||
+        (k > 0 && !draft_tokens))
+        return cstr_fail(CSTR_ERR_NULL, "cstr_accept_draft: null pointer");
+    if (k < 0 || batch < 0)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_accept_draft: k = %d, batch = %d", k, batch);
+    if (batch == 0)
+        return CSTR_OK;
+    return cstr_launch_accept(draft_tokens, target_tokens, target_states, k, batch, n_accepted,
+                              out_tokens, states, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t *bad_state_rows,

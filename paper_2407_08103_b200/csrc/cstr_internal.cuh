@@ -118,7 +118,8 @@ struct cstr_step_args {
     int32_t dtype;
     int64_t ld;
     const float *noise;
-    int32_t *states;
+    const int32_t *states;
+    int32_t *states_out;           // may equal states (in-place update)
     int32_t *tokens_out;
     void *masked_out;
     uint8_t *accept_out;
@@ -130,3 +131,6 @@ struct cstr_step_args {
     int device;
 };
 int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream);
+int cstr_launch_accept(const int32_t *draft, const int32_t *tgt_tok, const int32_t *tgt_state,
+                       int32_t k, int32_t batch, int32_t *n_accepted, int32_t *out_tokens,
+                       int32_t *states, cudaStream_t stream);

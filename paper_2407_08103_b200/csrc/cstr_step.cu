@@ -38,7 +38,8 @@ struct StepParams {
     const void *logits;
     const float *noise;
     void *out;
-    int32_t *states;
+    const int32_t *states;   // per-row state before the step
+    int32_t *states_out;     // state after the step (may be the same array)
     int32_t *tokens;
     uint8_t *accept_out;
     unsigned long long *cell;
@@ -156,7 +157,7 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
         atomicAdd(p.counters + 0, 1ull);
     }
     p.tokens[c.r] = tok;
-    p.states[c.r] = q2;
+    p.states_out[c.r] = q2;
     if (p.accept_out)
         p.accept_out[c.r] = (q2 >= 0) ? (uint8_t)(tb.accept[q2] != 0) : (uint8_t)0;
 }
@@ -446,6 +447,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     p.noise = a.noise;
     p.out = a.masked_out;
     p.states = a.states;
+    p.states_out = a.states_out;
     p.tokens = a.tokens_out;
     p.accept_out = a.accept_out;
     p.cell = a.cell;
@@ -499,6 +501,47 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         else
             step_scalar_kernel<false><<<grid, threads, 0, stream>>>(p);
     }
+    CSTR_CUDA_TRY(cudaGetLastError());
+    return CSTR_OK;
+}
+
+// ---- speculative decoding: accept / rewind ------------------------------------
+//
+// After the target model has been penalised and decoded at every drafted
+// position (one fused step over batch x (k + 1) rows whose states are the
+// draft's state history), each sequence keeps the drafted tokens up to the
+// first disagreement, takes the target's token there, and rewinds its
+// constraint state to the one that follows that token.
+
+namespace {
+
+__global__ void accept_draft_kernel(const int32_t *__restrict__ draft, const int32_t *__restrict__ tgt_tok,
+                                    const int32_t *__restrict__ tgt_state, int k, int batch,
+                                    int32_t *__restrict__ n_accepted, int32_t *__restrict__ out_tokens,
+                                    int32_t *__restrict__ states)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= batch)
+        return;
+    const int32_t *d = draft + (long long)r * k;
+    const int32_t *t = tgt_tok + (long long)r * (k + 1);
+    int n = 0;
+    while (n < k && d[n] == t[n])
+        ++n;
+    for (int i = 0; i <= k; ++i)
+        out_tokens[(long long)r * (k + 1) + i] = (i <= n) ? t[i] : -1;
+    n_accepted[r] = n;
+    states[r] = tgt_state[(long long)r * (k + 1) + n];
+}
+
+}  // namespace
+
+int cstr_launch_accept(const int32_t *draft, const int32_t *tgt_tok, const int32_t *tgt_state,
+                       int32_t k, int32_t batch, int32_t *n_accepted, int32_t *out_tokens,
+                       int32_t *states, cudaStream_t stream)
+{
+    accept_draft_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(draft, tgt_tok, tgt_state, k, batch,
+                                                                  n_accepted, out_tokens, states);
     CSTR_CUDA_TRY(cudaGetLastError());
     return CSTR_OK;
 }
@@ -595,6 +638,7 @@ extern "C" int cstr_step_static(const cstr_table_t *const *tables, int32_t n_tab
     a.ld = ld;
     a.noise = noise;
     a.states = states;
+    a.states_out = states;
     a.tokens_out = tokens_out;
     a.masked_out = masked_out;
     a.accept_out = accept_out;

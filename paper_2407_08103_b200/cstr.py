@@ -25,7 +25,8 @@ EXPORTS = [
     "cstr_vocab_set_token_sets", "cstr_free_vocab",
     "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
-    "cstr_step", "cstr_step_status", "cstr_step_static", "cstr_last_error",
+    "cstr_step", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
+    "cstr_step_static", "cstr_last_error",
 ]
 
 _lib = None
@@ -207,8 +208,10 @@ def cstr_workspace_create(max_batch: int) -> Workspace:
 
 
 def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noise=None,
-              row_table=None, accept_out=None, vocab_ld: int | None = None, stream=None) -> None:
-    """Enqueue one constrained decoding step.  All tensors are CUDA tensors:
+              row_table=None, accept_out=None, vocab_ld: int | None = None, stream=None,
+              states_out=None) -> None:
+    """Enqueue one constrained decoding step (``cstr_step``; with ``states_out`` given,
+    ``cstr_step_history``: ``states`` is left untouched).  All tensors are CUDA tensors:
     ``logits``/``masked_out`` ``[B][ld]`` float32 or bfloat16, ``noise`` float32
     ``[B][ld]`` or None, ``states``/``tokens_out``/``row_table`` int32 ``[B]``,
     ``accept_out`` uint8 ``[B]`` or None."""
@@ -232,16 +235,49 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
         raise TypeError("masked_out must have the dtype of logits")
     if noise is not None and noise.dtype != torch.float32:
         raise TypeError("noise must be float32")
-    for name, t, dt in (("states", states, torch.int32), ("tokens_out", tokens_out, torch.int32),
+    for name, t, dt in (("states", states, torch.int32), ("states_out", states_out, torch.int32),
+                        ("tokens_out", tokens_out, torch.int32),
                         ("row_table", row_table, torch.int32), ("accept_out", accept_out, torch.uint8)):
         if t is not None and (t.dtype != dt or t.numel() < batch or not t.is_contiguous()):
             raise ValueError("%s must be a contiguous %s tensor with one entry per row" % (name, dt))
     arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
-    _check(lib().cstr_step(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table), _dev_ptr(logits),
-                           ctypes.c_int32(dtype), ctypes.c_int64(ld), _dev_ptr(noise),
-                           _dev_ptr(states), _dev_ptr(tokens_out), _dev_ptr(masked_out),
-                           _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
-                           _stream_ptr(stream)))
+    if states_out is None:
+        _check(lib().cstr_step(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
+                               _dev_ptr(logits), ctypes.c_int32(dtype), ctypes.c_int64(ld),
+                               _dev_ptr(noise), _dev_ptr(states), _dev_ptr(tokens_out),
+                               _dev_ptr(masked_out), _dev_ptr(accept_out), ctypes.c_int32(batch),
+                               ws.ptr, _stream_ptr(stream)))
+    else:
+        _check(lib().cstr_step_history(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
+                                       _dev_ptr(logits), ctypes.c_int32(dtype), ctypes.c_int64(ld),
+                                       _dev_ptr(noise), _dev_ptr(states), _dev_ptr(states_out),
+                                       _dev_ptr(tokens_out), _dev_ptr(masked_out),
+                                       _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
+                                       _stream_ptr(stream)))
+
+
+def cstr_step_history(tables, logits, states_in, states_out, tokens_out, masked_out, ws: Workspace,
+                      **kw) -> None:
+    """``cstr_step`` with separate input and output state arrays (state history)."""
+    cstr_step(tables, logits, states_in, tokens_out, masked_out, ws, states_out=states_out, **kw)
+
+
+def cstr_accept_draft(draft_tokens, target_tokens, target_states, n_accepted, out_tokens, states,
+                      stream=None) -> None:
+    """Greedy verification + rewind.  CUDA int32 tensors: ``draft_tokens`` ``[B][k]``,
+    ``target_tokens`` / ``target_states`` / ``out_tokens`` ``[B][k+1]``, ``n_accepted`` / ``states`` ``[B]``."""
+    import torch
+    B, k1 = target_tokens.shape
+    k = k1 - 1
+    for name, t, shape in (("draft_tokens", draft_tokens, (B, k)), ("target_states", target_states, (B, k1)),
+                           ("out_tokens", out_tokens, (B, k1)), ("n_accepted", n_accepted, (B,)),
+                           ("states", states, (B,)), ("target_tokens", target_tokens, (B, k1))):
+        if t.dtype != torch.int32 or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous int32 tensor of shape %s" % (name, shape))
+    _check(lib().cstr_accept_draft(_dev_ptr(draft_tokens), _dev_ptr(target_tokens),
+                                   _dev_ptr(target_states), ctypes.c_int32(k), ctypes.c_int32(B),
+                                   _dev_ptr(n_accepted), _dev_ptr(out_tokens), _dev_ptr(states),
+                                   _stream_ptr(stream)))
 
 
 def cstr_step_static(tables, logits, states, tokens_out, masked_out, noise=None, row_table=None,
