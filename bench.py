@@ -443,6 +443,36 @@ def main():
     kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
     active_frac = float((dec.states >= 0).float().mean().item())
 
+    # ---- speculative verification: 64 sequences x (7 drafted + 1) positions --------
+    # one fused step over the state history (the 512 rows of the workload) + accept / rewind
+    spec = None
+    if rank == 0 and B % 8 == 0:
+        kk, seqs = 7, B // 8
+        hist = dec.states.clone()                      # stands for the draft's state history
+        t_st = torch.empty(B, dtype=torch.int32, device=dev)
+        t_tok = torch.empty(B, dtype=torch.int32, device=dev)
+        draft = torch.zeros((seqs, kk), dtype=torch.int32, device=dev)
+        n_acc = torch.empty(seqs, dtype=torch.int32, device=dev)
+        out_tok = torch.empty((seqs, kk + 1), dtype=torch.int32, device=dev)
+        new_st = torch.empty(seqs, dtype=torch.int32, device=dev)
+        sp = []
+        for i in range(12):
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record(stream)
+            cstr.cstr_step_history([table], dev_pool[i % POOL], hist, t_st, t_tok, out_bufs[i & 1],
+                                   dec.ws, stream=stream)
+            cstr.cstr_accept_draft(draft, t_tok.view(seqs, kk + 1), t_st.view(seqs, kk + 1), n_acc,
+                                   out_tok, new_st, stream=stream)
+            s1.record(stream)
+            s1.synchronize()
+            sp.append(s0.elapsed_time(s1))
+        spec_ms = float(np.mean(sp[2:]))
+        spec = {"sequences": seqs, "drafted_tokens": kk, "rows": B, "ms": spec_ms,
+                "logits_per_s": B * V / (spec_ms * 1e-3),
+                "frac_of_hbm_peak": B * V * BYTES_PER_LOGIT_F32_GREEDY / (spec_ms * 1e-3) / 1e9
+                / measured_hbm_peak()[0],
+                "kernels": "step_vec_kernel over the state history + accept_draft_kernel"}
+
     # ---- end to end: pinned host logits in, tokens + states out, every step ----
     staging = [torch.empty((B, V), dtype=torch.float32, device=dev) for _ in range(2)]
     h_tok = torch.empty(B, dtype=torch.int32).pin_memory()
@@ -573,6 +603,7 @@ def main():
                         if build_random else []),
         "table_build_e2e_ms": build_e2e_ms,
         "wildcard_table_build": wildcard,
+        "speculative_verify": spec,
         "other_workloads": others,
         "status_rows": {"bad_state": bad, "empty_mask": empty},
     }
