@@ -115,6 +115,20 @@ def test_mixed_tables_and_bad_table_index():
     assert ref["tokens"][3] == -1 and ref["tokens"][9] == -1 and ref["bad_state_rows"] == 2
 
 
+def test_wide_table_entries():
+    # more than 32,766 states: 32-bit table entries, decoded by the step's last-arriving CTA
+    rng = np.random.default_rng(12)
+    dfa = random_range_dfa(33000, seed=9)
+    vb, vo = random_vocab(rng, 300, max_len=3)
+    tables = gpu_tables([dfa], vb, vo)
+    V = vo.size - 1
+    states = np.array([0, 1, 32766, 32767, 32768, 32999, 33000, -1], dtype=np.int32)
+    for dtype in ("f32", "bf16"):
+        logits = rand_logits(rng, 8, V, (V + 7) // 8 * 8, dtype)
+        ref = run_step_both([dfa], tables, vb, vo, logits, states)
+        assert ref["bad_state_rows"] == 1 and (ref["tokens"][:6] >= 0).any()
+
+
 def test_error_codes_on_device_arguments():
     dfa = regex_to_dfa("a*")
     vb, vo = vocab_from_strings([b"a", b"b", b"aa"])
