@@ -381,9 +381,19 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     // States per lane: enough states per warp to amortise the per-token work,
     // without leaving most lanes idle on small automata.
     const int S = dfa->n_states;
-    int ns = S >= 4096 ? 8 : (S >= 1024 ? 4 : (S >= 256 ? 2 : 1));
-    if (ns == 8 && t->wide)
-        ns = 4;                        // a lane's unit of next is at most 16 bytes
+    // A warp's cost per token is mostly fixed (about 95 instructions) plus about
+    // 14 per state held by a lane, so take the NS with the fewest instructions
+    // over all state blocks.
+    int ns = 1;
+    long long best_cost = -1;
+    for (int cand = 1; cand <= (t->wide ? 4 : 8); cand *= 2) {   // a lane's unit of next is <= 16 bytes
+        const long long blocks = (S + 32 * cand - 1) / (32 * cand);
+        const long long cost = blocks * (95 + 14 * cand);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            ns = cand;
+        }
+    }
     const int per_warp = ns * 32;
     const int state_warps = (S + per_warp - 1) / per_warp;
 
