@@ -232,3 +232,35 @@ def test_two_calls_share_a_workspace_in_stream_order():
     # scratch is reset by the kernel itself: back-to-back steps on one stream need no host work
     dec = decode_and_check("api_1k", steps=4, pool=4, sample_rows=range(4), batch=64)
     assert dec.status()[0] == 0
+
+
+def test_repeated_runs_are_bit_identical():
+    # every kernel twice on the same inputs: any race or order dependence would show
+    name = "json_32k"
+    dfa = config_dfas(name)[0]
+    vb, vo = config_vocab(name)
+    V = vo.size - 1
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    h = cstr.cstr_load_dfa(*dfa)
+    S = dfa[0].shape[0]
+    t1 = cstr.cstr_table_create(vocab, S)
+    t2 = cstr.cstr_table_create(vocab, S)
+    cstr.cstr_table_build(t1, h)
+    cstr.cstr_table_build(t2, h)
+    cstr.cstr_table_build(t2, h)                     # rebuilding over itself changes nothing
+    a, b = cstr.cstr_table_download(t1), cstr.cstr_table_download(t2)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    B = 64
+    logits = to_dev_logits(normal_logits(3, 0, range(B), V, sigma=2.0, dtype="bf16"))
+    noise = torch.from_numpy(gumbel_noise(4, 0, range(B), V)).to(DEV)
+    ws = cstr.cstr_workspace_create(B)
+    outs = []
+    for rep in range(3):
+        st = torch.full((B,), int(dfa[2]), dtype=torch.int32, device=DEV)
+        tok = torch.empty(B, dtype=torch.int32, device=DEV)
+        masked = torch.empty_like(logits)
+        cstr.cstr_step([t1 if rep else t2], logits, st, tok, masked, ws, noise=noise)
+        torch.cuda.synchronize()
+        outs.append((tok.cpu().numpy(), st.cpu().numpy(), from_dev_logits(masked)))
+    for o in outs[1:]:
+        assert all(np.array_equal(x, y) for x, y in zip(outs[0], o))
