@@ -248,6 +248,18 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
             pairs.append((e0, e1))
     torch.cuda.synchronize()
     kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    # the same steps back to back between one pair of events (restart op included):
+    # for the small workloads this, not the per-launch bracket, is the sustained cost
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    loop_steps = 200
+    l0.record(stream)
+    for i in range(loop_steps):
+        dec.step(pool[i % pool_n], noise=None if noise is None else noise[i % len(noise)],
+                 masked_out=out[i & 1], stream=stream)
+        torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
+    l1.record(stream)
+    l1.synchronize()
+    loop_ms = l0.elapsed_time(l1) / loop_steps
     bytes_per_logit = 2 * esz + (4 if w.gumbel else 0) + 1.0 / 8.0
     step_bytes = B * V * bytes_per_logit
     gbs = step_bytes / (kernel_ms * 1e-3) / 1e9
@@ -258,7 +270,7 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
     return {
         "workload": name, "vocab": V, "batch": B, "dfa_states": [int(d[0].shape[0]) for d in dfas],
         "dtype": w.dtype, "sampler": "gumbel-max" if w.gumbel else "greedy",
-        "tables": len(tables), "step_kernel_ms": kernel_ms,
+        "tables": len(tables), "step_kernel_ms": kernel_ms, "step_loop_ms": loop_ms,
         "logits_per_s": B * V / (kernel_ms * 1e-3),
         "roofline": {"bound": "hbm" if hbm_honest else "launch latency (working set sits in L2)",
                      "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
