@@ -81,7 +81,7 @@ void cstr_free_dfa(cstr_dfa_t *dfa);
  *   n_labels     0..32; label t is bit t of the token sets given to
  *                cstr_vocab_set_token_sets
  * In the built table a state's terminal edges allow every token of their
- * labels' sets on top of the ordinary tokens ("applied en masse"); a selected
+ * labels' sets on top of the ordinary tokens (whole sets at once); a selected
  * token follows its ordinary edge if it has one, else the terminal edge of the
  * lowest label whose set holds it (the paper's precedence heuristic).
  */
@@ -96,8 +96,8 @@ int cstr_load_dfa_terminals(const int32_t *trans, const int32_t *term_trans, int
  * offsets[v+1]) (App. B.1: each token has one character sequence d(v); the
  * detokenization of a token sequence is the concatenation).  This is the
  * vocabulary-specific half of the method, prepared once per LM like the
- * detokenizing transducer T_V of Algorithm 1 (Section 2.4, "can easily be
- * pre-computed for each LM").
+ * detokenizing transducer T_V of Algorithm 1 (Section 2.4 notes that T_V
+ * depends only on the vocabulary and can be built ahead of time).
  *   vocab_bytes  HOST  uint8 [offsets[vocab_size]]
  *   offsets      HOST  int64 [vocab_size + 1], offsets[0] == 0, non-decreasing,
  *                total below 2^31
@@ -110,8 +110,8 @@ void cstr_free_vocab(cstr_vocab_t *vocab);
 
 /*
  * Attach the token sets of the terminal labels to a vocabulary (Section 2.5.1:
- * "terminal labels ... map to pre-computed masks of valid tokens", e.g. the
- * newline-free tokens for PARAGRAPH_TOKEN).  Prepared once per LM.
+ * every terminal label stands for a mask of tokens computed ahead of time,
+ * e.g. the newline-free tokens for PARAGRAPH_TOKEN).  Prepared once per LM.
  *   token_sets   HOST  uint32 [vocab_size]; bit t set iff the token belongs to
  *                the set of label t
  *   n_labels     1..32
@@ -217,15 +217,15 @@ int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t
 
 /*
  * cstr_step that leaves the input states untouched and writes the new ones to
- * states_out, so that a caller can keep "a full history of states instead of
- * just one" (Section 4, Speculative decoding: the constraint must be
- * rewindable because the target model may reject drafted tokens).
+ * states_out, so that a caller can keep the state after every drafted token
+ * (Section 4, Speculative decoding: the target model may reject drafted
+ * tokens, so the constraint has to be able to go back to an earlier state).
  *   states_in   DEVICE int32 [batch]
  *   states_out  DEVICE int32 [batch]; may equal states_in (then it is cstr_step)
  * Everything else as in cstr_step.  The same call, over batch x (k + 1) rows
  * whose states are the draft's history q_0 .. q_k of each sequence, penalises
  * the target model's logits at all drafted positions at once with the masks
- * the draft used ("sharing the penalties with the target model") and decodes
+ * the draft used (the penalties are computed once and serve both models) and decodes
  * the target's own token and next state at each position.
  */
 int cstr_step_history(const cstr_table_t *const *tables, int32_t n_tables,

@@ -17,11 +17,11 @@
  *   - Section 2.5.1, terminal labels: a state may also have edges labelled with
  *     terminal labels (symbols outside the byte alphabet), each label standing
  *     for a pre-computed set of tokens.  Such an edge allows every token of the
- *     label's set ("terminal masks are applied en masse"); when the selected
- *     token has no ordinary edge, the terminal edge of the first label (fixed
- *     precedence: ascending label index) whose set holds the token is taken
- *     ("prefer normal token edges when available, and otherwise follow a ...
- *     precedence ordering over terminal labels").
+ *     label's set at once (the whole set is OR-ed into the allowed tokens);
+ *     when the selected token has no ordinary edge, the terminal edge of the
+ *     first label (a fixed precedence: ascending label index) whose set holds
+ *     the token is taken - the paper's heuristic for the ambiguity: ordinary
+ *     token edges win, then a fixed order over the labels.
  *
  * Readings the paper leaves open (kept identical in the library under test):
  *   - a token of zero length never has an edge (Algorithm 1 emits the last
@@ -237,9 +237,9 @@ void oracle_step(const int32_t *const *trans, const uint8_t *const *accept,
 
 /*
  * Speculative decoding, greedy verification and rewind (Section 4): the target
- * model accepts a prefix of the drafted tokens; the constraint, which tracked
- * "a full history of states instead of just one", restarts from the state that
- * follows the last token kept.  With greedy selection the kept prefix is the
+ * model accepts a prefix of the drafted tokens; the constraint, which kept the
+ * state reached after every drafted token rather than only the latest one,
+ * restarts from the state that follows the last token kept.  With greedy selection the kept prefix is the
  * run of positions where the target's own (constrained) token equals the
  * drafted one, and the target's token at the first disagreement (or after the
  * last drafted position) is emitted as well.

@@ -4,8 +4,8 @@ Follows the paper's pipeline for the character-level automaton A_R
 (Algorithm 2, first lines; Section 2.1): a regular expression is turned into a
 non-deterministic FSA with epsilon edges by Thompson's construction
 (BuildRegexFSA), and that FSA is determinized by the subset construction
-(Section 2.1, "Surprisingly, non-deterministic and deterministic FSAs are
-equivalent"; Figure 2 shows it for a+|ab).  The alphabet is the 256 byte
+(Section 2.1 recalls that every FSA has an equivalent deterministic one;
+Figure 2 shows it for a+|ab).  The alphabet is the 256 byte
 values.  Matching is whole-string (the FSA accepts w iff a path from I to F
 spells w, Section 2.1).
 
