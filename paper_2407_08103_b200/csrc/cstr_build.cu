@@ -246,8 +246,10 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
 {
     __shared__ uint32_t tile[8][1024];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int w0 = blockIdx.x * 32;
-    const int sb0 = blockIdx.y * 8;
+    // x = group of 8 ballot words, y = group of 32 mask words: CTAs that read
+    // the four 32-byte quarters of the same maskT lines are launched together
+    const int sb0 = blockIdx.x * 8;
+    const int w0 = blockIdx.y * 32;
     for (int t = threadIdx.x; t < 1024; t += 256) {
         const long long tokid = (long long)w0 * 32 + t;
         uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
@@ -459,7 +461,9 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
                          cudaGetErrorString(e));
 
     const int ballot_words = ((S + per_warp - 1) / per_warp) * ns;
-    dim3 tgrid((unsigned)(t->ldw / 32), (unsigned)((ballot_words + 7) / 8));
+    dim3 tgrid((unsigned)((ballot_words + 7) / 8), (unsigned)(t->ldw / 32));
+    if (tgrid.y > 65535u)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: vocabulary too large for one launch");
     mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
                                                      ns);
     CSTR_CUDA_TRY(cudaGetLastError());

@@ -264,3 +264,15 @@ def test_repeated_runs_are_bit_identical():
         outs.append((tok.cpu().numpy(), st.cpu().numpy(), from_dev_logits(masked)))
     for o in outs[1:]:
         assert all(np.array_equal(x, y) for x, y in zip(outs[0], o))
+
+
+def test_many_rows_small_vocabulary():
+    # more rows than a grid dimension of 65,535 would hold: rows are linearised
+    rng = np.random.default_rng(21)
+    dfa = dense_random_dfa(rng, 20, live=0.5)
+    vb, vo = random_vocab(rng, 96, max_len=3)
+    tables = gpu_tables([dfa], vb, vo)
+    B, V = 70001, 96
+    logits = rng.standard_normal((B, V)).astype(np.float32)
+    states = rng.integers(-1, 20, size=B).astype(np.int32)
+    run_step_both([dfa], tables, vb, vo, logits, states)

@@ -130,3 +130,37 @@ def test_config_256k_sampled_states(name):
     live = (nxt >= 0).sum(axis=1)
     pop = np.unpackbits(mask.view(np.uint8), axis=1).sum(axis=1)
     assert np.array_equal(live, pop)
+
+
+def test_long_shared_prefixes_and_long_suffixes():
+    # Tokens that share far more than the 8 bytes the walk keeps on its stack,
+    # suffixes longer than the 8 bytes carried inline, exact duplicates, and a
+    # vocabulary order that is the reverse of the trie order.
+    rng = np.random.default_rng(77)
+    base = bytes(rng.integers(97, 100, size=60).astype(np.uint8))
+    toks = []
+    for _ in range(1500):
+        p = int(rng.integers(0, 60))
+        s = bytes(rng.integers(97, 100, size=int(rng.integers(0, 25))).astype(np.uint8))
+        toks.append(base[:p] + s)
+    toks += toks[:100]                                   # duplicates
+    toks = sorted(toks, reverse=True)
+    vb, vo = vocab_from_strings(toks)
+    S = 700
+    trans = rng.integers(0, S, size=(S, 256)).astype(np.int32)
+    trans[:, :97] = -1
+    trans[:, 100:] = -1
+    trans[rng.random((S, 256)) < 0.03] = -1              # long walks mostly survive
+    dfa = (trans, (rng.random(S) < 0.3).astype(np.uint8), 0)
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo)
+    # the same vocabulary against a counter-like chain (neighbouring states stay neighbours)
+    S = 300
+    chain = np.full((S, 256), -1, dtype=np.int32)
+    for q in range(S):
+        chain[q, 97] = (q + 1) % S
+        chain[q, 98] = q
+        chain[q, 99] = (q * 7 + 3) % S
+    dfa = (chain, np.ones(S, dtype=np.uint8), 5)
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo)
