@@ -62,7 +62,7 @@ typedef struct cstr_workspace cstr_workspace_t; /* per-stream scratch of cstr_st
  * symbol, so it is a table).  Sigma is the 256 byte values.
  *   trans        HOST  int32 [n_states][256], target state or -1 (no edge)
  *   accept       HOST  uint8 [n_states], non-zero = final state
- *   n_states     >= 1;  start_state in [0, n_states)
+ *   n_states     1 .. 4,000,000;  start_state in [0, n_states)
  * Validates every target, merges bytes that no state tells apart into
  * classes, and copies the class-major table to the device (16-bit entries up
  * to 32766 states, else 32-bit); returns the handle in *out.

@@ -12,13 +12,14 @@
 //
 //   - lane = state: every lane of a warp reads the same token, so there is no
 //     divergence on token length, and all control flow is warp-uniform;
-//   - the DFA is class-compressed and class-major (tt[class][state]) with a
-//     self-looping dead-sink column: a lookup is one indexed load, the first
-//     byte of a walk reads consecutive entries, and dead walks need no branch;
+//   - the DFA is class-compressed and class-major (tt[class][slot]) with a
+//     self-looping dead sink, and its entries are the byte offsets of the target
+//     slots: a lookup is one add and one load, and dead walks need no branch;
 //     it lives in shared memory when it fits, else it is gathered through L1/L2;
-//   - next-state entries leave as 64-byte state segments of the token's row;
-//     validity goes out as one ballot word per (token, 32-state block), which a
-//     second kernel bit-transposes into the state-major mask the step streams.
+//   - a lane holds NS consecutive states (NS = 1, 2, 4 or 8) and stores their
+//     next-state entries with one vector store into the token's row;
+//     validity goes out as NS ballot words per (token, warp), which a second
+//     kernel bit-transposes into the state-major mask the step streams.
 #include "cstr_internal.cuh"
 
 namespace {
@@ -44,9 +45,8 @@ struct BuildParams {
 };
 
 // NS consecutive table entries per lane travel as one aligned unit (one vector
-// load / store).  States are handled as unsigned values (entry types are read
-// as uint16 / uint32; "no edge" is all ones), which keeps every conversion a
-// plain bit operation.
+// load / store).  Entries are handled as unsigned values (uint16 / uint32),
+// which keeps packing and unpacking plain bit operations.
 template <int BYTES>
 struct Unit;
 template <> struct Unit<2> { typedef unsigned short type; };

@@ -56,6 +56,9 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     *out = nullptr;
     if (n_states < 1)
         return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: n_states = %d, need >= 1", n_states);
+    if (n_states > 4000000)       // row byte offsets of the class-major table are 32-bit
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: n_states = %d, at most 4,000,000 supported",
+                         n_states);
     if (start_state < 0 || start_state >= n_states)
         return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: start_state %d outside [0, %d)",
                          start_state, n_states);
