@@ -263,7 +263,7 @@ __device__ __forceinline__ void apply_one(const StepParams &p, const RowCtx &c, 
 // ---- vector kernel ----------------------------------------------------------
 
 template <bool BF16, bool NOISE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 step_vec_kernel(const __grid_constant__ StepParams p)
 {
     constexpr int VEC = BF16 ? 8 : 4;               // logits per 16-byte vector
