@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one full-size step launch (512 x 256,000 fp32),
 # from the ncu capture summarised in profiles/step_vec_kernel_fp32_full_size_traffic.md; set to
 # None whenever step_vec_kernel changes until the capture is repeated.
-STEP_TRAFFIC_BYTES = 993.9e6
+STEP_TRAFFIC_BYTES = 994.0e6
 
 
 def parse_args():
