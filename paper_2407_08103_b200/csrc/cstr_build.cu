@@ -291,31 +291,36 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
 // Terminal-label edges (wildcards matched by pre-computed token sets): for
 // every state that has some, every token without an ordinary edge takes the
 // terminal edge of the lowest label whose set holds it, and becomes allowed.
-// One CTA = 256 consecutive tokens of one such state; the mask words are
-// OR-ed by the warp that owns the 32 tokens (no other warp touches them).
+// One thread = one token, looping over the states with terminal edges (their
+// entries of the token's row share sectors when the states are neighbours);
+// the mask words are OR-ed by the warp that owns the 32 tokens, so no other
+// warp touches them.
 template <typename NT>
 __global__ void __launch_bounds__(256)
 apply_terminals_kernel(const int32_t *__restrict__ tstate, const uint32_t *__restrict__ tset,
-                       const uint32_t *__restrict__ ttarget, int n_labels,
+                       const uint32_t *__restrict__ ttarget, int n_term_states, int n_labels,
                        const uint32_t *__restrict__ tsets, const uint32_t *__restrict__ off, int V,
                        int eos_id, unsigned sink, NT *__restrict__ next, long long lds,
                        uint32_t *__restrict__ mask, long long ldw)
 {
     const int v = blockIdx.x * 256 + threadIdx.x;
-    const int i = blockIdx.y;
-    const int q = tstate[i];
-    bool fresh = false;
-    if (v < V) {
-        NT *slot = next + (long long)v * lds + q;
-        const uint32_t labels = tsets[v] & tset[i];
-        if ((unsigned)*slot == sink && labels != 0u && v != eos_id && off[v + 1] > off[v]) {
-            *slot = (NT)ttarget[(long long)i * n_labels + (__ffs((int)labels) - 1)];
+    const bool eligible = v < V && v != eos_id && off[min(v, V - 1) + 1] > off[min(v, V - 1)];
+    const uint32_t mine = eligible ? tsets[v] : 0u;
+    if (__ballot_sync(kFull, mine != 0u) == 0u)
+        return;                                          // no token of this warp is in any set
+    NT *row = next + (long long)min(v, V - 1) * lds;
+    for (int i = 0; i < n_term_states; ++i) {
+        const int q = tstate[i];
+        const uint32_t labels = mine & tset[i];
+        bool fresh = false;
+        if (labels != 0u && (unsigned)row[q] == sink) {
+            row[q] = (NT)ttarget[(long long)i * n_labels + (__ffs((int)labels) - 1)];
             fresh = true;
         }
+        const uint32_t word = __ballot_sync(kFull, fresh);
+        if ((threadIdx.x & 31) == 0 && word != 0u)
+            mask[(long long)q * ldw + (v >> 5)] |= word;
     }
-    const uint32_t word = __ballot_sync(kFull, fresh);
-    if ((threadIdx.x & 31) == 0 && word != 0u)
-        mask[(long long)q * ldw + (v >> 5)] |= word;
 }
 
 template <typename ST, typename NT, int NS, bool SMEM>
@@ -470,17 +475,16 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
 
     if (dfa->n_term_states > 0) {
         const unsigned sink = (unsigned)CSTR_PERM(S) << (dfa->wide ? 2 : 1);
-        dim3 agrid((unsigned)((t->V + 255) / 256), (unsigned)dfa->n_term_states);
-        if (agrid.y > 65535u)
-            return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: too many states with terminal edges");
+        const unsigned agrid = (unsigned)((t->V + 255) / 256);
         if (t->wide)
             apply_terminals_kernel<uint32_t><<<agrid, 256, 0, stream>>>(
-                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_labels, vc->tsets, vc->off, t->V,
-                t->eos_id, sink, (uint32_t *)t->next, t->lds, t->mask, t->ldw);
+                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
+                vc->off, t->V, t->eos_id, sink, (uint32_t *)t->next, t->lds, t->mask, t->ldw);
         else
             apply_terminals_kernel<uint16_t><<<agrid, 256, 0, stream>>>(
-                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_labels, vc->tsets, vc->off, t->V,
-                t->eos_id, sink & 0xffffu, (uint16_t *)t->next, t->lds, t->mask, t->ldw);
+                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
+                vc->off, t->V, t->eos_id, sink & 0xffffu, (uint16_t *)t->next, t->lds, t->mask,
+                t->ldw);
         CSTR_CUDA_TRY(cudaGetLastError());
     }
     return CSTR_OK;

@@ -35,6 +35,71 @@ static int check_device(int handle_device, const char *what)
 
 // ------------------------------------------------------------------ DFA
 
+namespace {
+
+// Two order-independent 64-bit hashes per byte column of the raw table
+// (thread = byte, a block sums a slab of rows, slabs combine with atomicAdd).
+__global__ void __launch_bounds__(256)
+dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_per_block,
+                       unsigned long long *__restrict__ hashes)
+{
+    const int b = threadIdx.x;
+    const int q0 = blockIdx.x * rows_per_block;
+    const int q1 = min(n_states, q0 + rows_per_block);
+    unsigned long long h1 = 0, h2 = 0;
+    for (int q = q0; q < q1; ++q) {
+        unsigned long long x = (unsigned long long)(unsigned)raw[(long long)q * 256 + b] +
+                               ((unsigned long long)(unsigned)q << 32) + 0x9e3779b97f4a7c15ull;
+        x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;        // splitmix64 finaliser: (q, value) -> 64 bits
+        x ^= x >> 27; x *= 0x94d049bb133111ebull;
+        x ^= x >> 31;
+        h1 += x;
+        h2 += (x ^ 0xc2b2ae3d27d4eb4full) * 0xff51afd7ed558ccdull;
+    }
+    atomicAdd(hashes + b, h1);
+    atomicAdd(hashes + 256 + b, h2);
+}
+
+// Class-major code table from the raw table, proving the proposed classes on
+// the way: tt[c][PERM(q)] = code(raw[q][rep[c]] or sink); every raw[q][b] must
+// equal raw[q][rep[cls[b]]], else *mismatch is set.  A block handles 8 states.
+__global__ void __launch_bounds__(256)
+dfa_build_table_kernel(const int32_t *__restrict__ raw, int n_states, int row, int n_classes,
+                       const uint8_t *__restrict__ cls, const uint8_t *__restrict__ rep, int wide,
+                       void *__restrict__ tt, unsigned long long *__restrict__ mismatch)
+{
+    __shared__ int32_t s_row[8][256];
+    const int b = threadIdx.x;
+    const int q0 = blockIdx.x * 8;
+    bool differs = false;
+    for (int i = 0; i < 8; ++i) {
+        const int q = q0 + i;
+        s_row[i][b] = (q < n_states) ? raw[(long long)q * 256 + b] : -1;
+    }
+    __syncthreads();
+    const int my_rep = rep[cls[b]];
+    for (int i = 0; i < 8; ++i)
+        differs |= s_row[i][b] != s_row[i][my_rep];
+    if (differs)
+        atomicOr(mismatch, 1ull);
+    for (int k = threadIdx.x; k < 8 * n_classes; k += 256) {
+        const int i = k & 7, c = k >> 3;
+        const int q = q0 + i;
+        if (q >= row)
+            continue;
+        const int32_t t = s_row[i][rep[c]];
+        const unsigned target = (unsigned)CSTR_PERM(t >= 0 ? t : n_states);
+        const long long at = (long long)c * row + CSTR_PERM(q);
+        if (wide)
+            ((uint32_t *)tt)[at] = target * 4u;
+        else
+            ((uint16_t *)tt)[at] = (uint16_t)(target * 2u);
+    }
+}
+
+}  // namespace
+
+
 extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
 {
     if (!dfa)
@@ -63,11 +128,16 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
         return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: start_state %d outside [0, %d)",
                          start_state, n_states);
     const int64_t n = (int64_t)n_states * 256;
-    for (int64_t i = 0; i < n; ++i) {
-        if (trans[i] < -1 || trans[i] >= n_states)
-            return cstr_fail(CSTR_ERR_DFA,
-                             "cstr_load_dfa: state %lld byte %lld has target %d outside [-1, %d)",
-                             (long long)(i / 256), (long long)(i % 256), trans[i], n_states);
+    int bad = 0;                   // branch-free so that the scan vectorises
+    for (int64_t i = 0; i < n; ++i)
+        bad |= (trans[i] < -1) | (trans[i] >= n_states);
+    if (bad) {
+        for (int64_t i = 0; i < n; ++i) {
+            if (trans[i] < -1 || trans[i] >= n_states)
+                return cstr_fail(CSTR_ERR_DFA,
+                                 "cstr_load_dfa: state %lld byte %lld has target %d outside [-1, %d)",
+                                 (long long)(i / 256), (long long)(i % 256), trans[i], n_states);
+        }
     }
     cstr_dfa *d = new (std::nothrow) cstr_dfa();
     if (!d)
@@ -79,77 +149,102 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     d->row = ((int64_t)n_states + 1 + 255) / 256 * 256;
     const size_t esz = d->wide ? 4 : 2;
 
-    // Byte classes: bytes whose columns are identical in every state.
-    std::vector<int32_t> col;      // column-major copy, col[b * S + q]
-    std::vector<int> order(256), cls_of(256), rep;
-    std::vector<uint8_t> cls8(256), flags;
-    std::vector<uint8_t> tt;
+    // The raw table goes to the device once; byte classes (bytes whose columns
+    // are identical in every state) and the class-major code table are made
+    // there: column hashes propose the classes, a second kernel proves them
+    // entry by entry while it writes the table, and only a hash collision (never
+    // seen) falls back to exact column comparisons on the host.
+    std::vector<uint8_t> flags;
     try {
-        col.resize((size_t)n);
-        for (int32_t q = 0; q < n_states; ++q)
-            for (int b = 0; b < 256; ++b)
-                col[(size_t)b * n_states + q] = trans[(size_t)q * 256 + b];
-        const size_t colbytes = (size_t)n_states * sizeof(int32_t);
-        for (int b = 0; b < 256; ++b)
-            order[b] = b;
-        std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
-            return memcmp(&col[(size_t)x * n_states], &col[(size_t)y * n_states], colbytes) < 0;
-        });
-        // classes numbered by their smallest byte
-        std::vector<int> group(256, -1);
-        int ngroups = 0;
-        for (int i = 0; i < 256; ++i) {
-            if (i > 0 && memcmp(&col[(size_t)order[i] * n_states],
-                                &col[(size_t)order[i - 1] * n_states], colbytes) == 0)
-                group[order[i]] = group[order[i - 1]];
-            else
-                group[order[i]] = ngroups++;
-        }
-        std::vector<int> renum(ngroups, -1);
-        for (int b = 0; b < 256; ++b) {
-            if (renum[group[b]] < 0) {
-                renum[group[b]] = (int)rep.size();
-                rep.push_back(b);
-            }
-            cls_of[b] = renum[group[b]];
-            cls8[b] = (uint8_t)cls_of[b];
-        }
-        d->n_classes = (int32_t)rep.size();
-        tt.assign((size_t)d->n_classes * (size_t)d->row * esz, 0);
-        const int32_t sink = n_states;
-        for (int c = 0; c < d->n_classes; ++c) {
-            const int32_t *src = &col[(size_t)rep[c] * n_states];
-            for (int64_t q = 0; q < d->row; ++q) {
-                const int32_t t = (q < n_states && src[q] >= 0) ? src[q] : sink;
-                const size_t at = (size_t)c * d->row + (size_t)CSTR_PERM(q);
-                // entries are codes: the byte offset of the target's slot in a row
-                if (d->wide)
-                    ((uint32_t *)tt.data())[at] = (uint32_t)CSTR_PERM(t) * 4u;
-                else
-                    ((uint16_t *)tt.data())[at] = (uint16_t)(CSTR_PERM(t) * 2);
-            }
-        }
         flags.resize(n_states);
-        for (int32_t q = 0; q < n_states; ++q)
-            flags[q] = accept[q] ? 1 : 0;
     } catch (const std::bad_alloc &) {
         delete d;
         return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
     }
+    for (int32_t q = 0; q < n_states; ++q)
+        flags[q] = accept[q] ? 1 : 0;
 
+    int32_t *raw = nullptr;
+    unsigned long long *hashes = nullptr;     // [2][256], then one mismatch flag
+    uint8_t *rep_dev = nullptr;
     cudaError_t e = cudaGetDevice(&d->device);
     if (e == cudaSuccess)
-        e = cudaMalloc(&d->tt, tt.size());
+        e = cudaMalloc((void **)&raw, (size_t)n * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&hashes, 513 * 8);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&rep_dev, 256);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&d->cls, 256);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&d->accept, (size_t)n_states);
     if (e == cudaSuccess)
-        e = cudaMemcpy(d->tt, tt.data(), tt.size(), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(d->cls, cls8.data(), 256, cudaMemcpyHostToDevice);
+        e = cudaMemcpy(raw, trans, (size_t)n * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(d->accept, flags.data(), (size_t)n_states, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemset(hashes, 0, 513 * 8);
+    unsigned long long host_hash[513];
+    if (e == cudaSuccess) {
+        const int rows_per_block = 64;
+        dfa_column_hash_kernel<<<(n_states + rows_per_block - 1) / rows_per_block, 256>>>(
+            raw, n_states, rows_per_block, hashes);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpy(host_hash, hashes, 512 * 8, cudaMemcpyDeviceToHost);
+
+    uint8_t cls8[256], rep8[256];
+    int n_classes = 0;
+    auto propose = [&](bool exact) {
+        n_classes = 0;
+        for (int b = 0; b < 256; ++b) {
+            int found = -1;
+            for (int c = 0; c < n_classes && found < 0; ++c) {
+                const int r = rep8[c];
+                bool same = host_hash[b] == host_hash[r] && host_hash[256 + b] == host_hash[256 + r];
+                if (exact) {
+                    same = true;
+                    for (int32_t q = 0; q < n_states && same; ++q)
+                        same = trans[(size_t)q * 256 + b] == trans[(size_t)q * 256 + r];
+                }
+                if (same)
+                    found = c;
+            }
+            if (found < 0) {                     // classes are numbered by their smallest byte
+                found = n_classes;
+                rep8[n_classes++] = (uint8_t)b;
+            }
+            cls8[b] = (uint8_t)found;
+        }
+    };
+    for (int attempt = 0; attempt < 2 && e == cudaSuccess; ++attempt) {
+        propose(attempt == 1);
+        d->n_classes = n_classes;
+        const size_t tt_bytes = (size_t)n_classes * (size_t)d->row * esz;
+        cudaFree(d->tt);
+        d->tt = nullptr;
+        e = cudaMalloc(&d->tt, tt_bytes);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->cls, cls8, 256, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(rep_dev, rep8, 256, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) {
+            dfa_build_table_kernel<<<(unsigned)((d->row + 7) / 8), 256>>>(
+                raw, n_states, (int)d->row, n_classes, d->cls, rep_dev, d->wide, d->tt,
+                hashes + 512);
+            e = cudaGetLastError();
+        }
+        unsigned long long mismatch = 0;
+        if (e == cudaSuccess)
+            e = cudaMemcpy(&mismatch, hashes + 512, 8, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess || mismatch == 0)
+            break;                               // proven (or failed): no second attempt
+        e = cudaMemset(hashes + 512, 0, 8);      // a collision: redo with exact classes
+    }
+    cudaFree(raw);
+    cudaFree(hashes);
+    cudaFree(rep_dev);
     if (e != cudaSuccess) {
         int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
                            "cstr_load_dfa: %s", cudaGetErrorString(e));
