@@ -36,7 +36,7 @@ struct BuildParams {
     const uint32_t *off;       // [V + 1]
     void *next;                // [V][lds]
     uint32_t *maskT;           // [V][ldb]
-    long long lds, ldb;
+    unsigned lds, ldb;         // row pitches of next (entries) and maskT (words)
     int row;                   // entries per class row of tt
     int n_states, n_classes, V, eos_id;
     int tokens_per_cta;
@@ -174,15 +174,14 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
             pk = s_stack[shared * 32];
             unpack_entries<ESZ, NS>(pk, cur);
         }
-        unsigned long long inl = ((unsigned long long)d.w << 32) | d.z;   // bytes shared .. shared+7
+#pragma unroll 1                         // 1.4 iterations on average: unrolling only adds dispatch code
         for (int k = shared; k < n; ++k) {
             unsigned b;
-            if (!first && k - shared < 8) {
-                b = (unsigned)inl & 0xffu;
-                inl >>= 8;
-            } else {
+            const unsigned r = (unsigned)(k - shared);
+            if (!first && r < 8u)
+                b = __byte_perm(d.z, d.w, r) & 0xffu;     // d.z / d.w hold bytes shared .. shared+7
+            else
                 b = __ldg(p.bytes + __ldg(p.off + tok) + k);
-            }
             const uint32_t ro = s_rowoff[b];
             if (SMEM) {
                 const unsigned char *rowp = s_tt + ro;
@@ -223,9 +222,9 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
         }
         prev_eos = is_eos;
         // lds is a multiple of 256 states: the whole unit is inside the token's row
-        *(NPack *)(next_lane + (size_t)tok * (size_t)p.lds) = outp;
+        *(NPack *)(next_lane + (unsigned long long)tok * p.lds) = outp;
         if (lane == 0) {                 // ballots are warp-uniform; (q0 >> 5) + NS <= lds / 32 < ldb
-            uint32_t *mrow = maskT_warp + (size_t)tok * (size_t)p.ldb;       // NS-word aligned
+            uint32_t *mrow = maskT_warp + (unsigned long long)tok * p.ldb;          // NS-word aligned
             if constexpr (NS == 1) *mrow = words[0];
             if constexpr (NS == 2) *(uint2 *)mrow = make_uint2(words[0], words[1]);
             if constexpr (NS >= 4) *(uint4 *)mrow = make_uint4(words[0], words[1], words[2], words[3]);
@@ -374,8 +373,8 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     p.next = t->next;
     p.maskT = t->maskT;
     p.row = (int)dfa->row;
-    p.lds = t->lds;
-    p.ldb = t->ldb;
+    p.lds = (unsigned)t->lds;      // at most 4,000,512 states
+    p.ldb = (unsigned)t->ldb;
     p.n_states = dfa->n_states;
     p.n_classes = dfa->n_classes;
     p.V = t->V;
@@ -388,14 +387,15 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     // States per lane: enough states per warp to amortise the per-token work,
     // without leaving most lanes idle on small automata.
     const int S = dfa->n_states;
-    // A warp's cost per token is mostly fixed (about 95 instructions) plus about
-    // 14 per state held by a lane, so take the NS with the fewest instructions
-    // over all state blocks.
+    // A warp's cost per token is mostly fixed (about 116 instructions measured)
+    // plus about 4.3 per state held by a lane, so take the NS with the fewest
+    // instructions over all state blocks.  (16 states per lane was tried: fewer
+    // instructions still, but too few resident warps to hide the latencies.)
     int ns = 1;
     long long best_cost = -1;
     for (int cand = 1; cand <= (t->wide ? 4 : 8); cand *= 2) {   // a lane's unit of next is <= 16 bytes
         const long long blocks = (S + 32 * cand - 1) / (32 * cand);
-        const long long cost = blocks * (95 + 14 * cand);
+        const long long cost = blocks * (1160 + 43 * cand);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             ns = cand;
