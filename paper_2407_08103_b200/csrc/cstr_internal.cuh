@@ -60,7 +60,7 @@ struct cstr_dfa {
 //               shared prefix (little endian in z, w) }
 // The shared prefix is clipped to CSTR_STACK_DEPTH.  Raw bytes / offsets serve
 // walks that start at the root and suffixes longer than 8 bytes.
-#define CSTR_STACK_DEPTH 8
+#define CSTR_STACK_DEPTH 4
 struct cstr_vocab {
     int device;
     int32_t V;
