@@ -7,9 +7,12 @@ A plain, slow CPU statement of the path the CUDA library implements:
 * ``token_table``   T[q][v] = delta*(q, bytes(v)) and the per-state allowed-token
                     bitmask (Algorithm 1 composed with the DFA, Theorem 2);
 * ``step``          mask, penalise with -inf, select, advance for a batch of
-                    rows (Algorithm 2, loop body).
+                    rows (Algorithm 2, loop body);
+* ``pda``           push-down constraints (Section 3): PDA acceptance, the
+                    token-level PDA's edges, Algorithm 3's allowed set and step.
 
-The last two are plain C (``cstr_oracle.c``), compiled with gcc on first use.
+All but the first are plain C (``cstr_oracle.c``, ``pda_oracle.c``), compiled
+with gcc on first use.
 Nothing here shares code with the CUDA path and the product never calls it:
 only tests, the smoke check and the benchmark's CPU-baseline leg do.
 """
@@ -22,7 +25,7 @@ import subprocess
 
 import numpy as np
 
-from . import regex_dfa  # noqa: F401
+from . import pda, regex_dfa  # noqa: F401
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cstr_oracle.c")
@@ -36,6 +39,7 @@ def build(force: bool = False) -> str:
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
                "-o", _LIB, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
+    pda.build(force)
     return _LIB
 
 
