@@ -43,6 +43,7 @@ extern "C" {
 #define CSTR_ERR_CUDA (-7)      /* a CUDA runtime call failed                         */
 #define CSTR_ERR_NOMEM (-8)     /* host or device allocation failed                   */
 #define CSTR_ERR_DEVICE (-9)    /* handle belongs to another CUDA device              */
+#define CSTR_ERR_PDA (-10)      /* byte PDA malformed, non-deterministic or over a limit */
 
 #define CSTR_F32 0              /* logits are IEEE fp32                               */
 #define CSTR_BF16 1             /* logits are bfloat16                                */
@@ -53,6 +54,9 @@ typedef struct cstr_dfa cstr_dfa_t;             /* device copy of a byte-level D
 typedef struct cstr_vocab cstr_vocab_t;         /* device copy of a vocabulary                */
 typedef struct cstr_table cstr_table_t;         /* device mask[S][W] + next[S][V]             */
 typedef struct cstr_workspace cstr_workspace_t; /* per-stream scratch of cstr_step            */
+typedef struct cstr_pda cstr_pda_t;             /* device copy of a byte-level PDA            */
+typedef struct cstr_pda_table cstr_pda_table_t; /* token-level PDA: masks per (state, top)    */
+typedef struct cstr_pda_workspace cstr_pda_workspace_t; /* per-stream scratch of cstr_pda_step */
 
 /* ------------------------------------------------------------------ DFA */
 
@@ -261,6 +265,110 @@ int cstr_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,
  */
 int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t *bad_state_rows,
                      int64_t *empty_mask_rows);
+
+/* ------------------------------------------------- push-down constraints */
+
+/*
+ * Load a deterministic byte-level push-down automaton (Section 3.1: a PDA
+ * (Sigma, Pi, S, Q, I, F, E) whose edges are tuples (source, input, pops,
+ * target, pushes); before an edge the stack must end with its pops, which it
+ * removes, then it appends its pushes).  Sigma is the 256 byte values, Pi the
+ * symbols 0 .. n_symbols-1; stacks are written bottom first (last = top).
+ *   edge_src, edge_byte, edge_tgt   HOST int32 [n_edges]
+ *   pop_off, push_off               HOST int32 [n_edges + 1], non-decreasing from 0
+ *   pops, pushes                    HOST int32: edge j pops pops[pop_off[j] .. pop_off[j+1])
+ *                                   (last entry = top) and appends pushes[push_off[j] ..
+ *                                   push_off[j+1]) in that order
+ *   accept                          HOST uint8 [n_states]; acceptance is by final state
+ * Limits (CSTR_ERR_PDA otherwise): every edge reads one byte (no epsilon
+ * input), pops at most one symbol and pushes at most CSTR_PDA_MAX_PUSH;
+ * n_symbols <= CSTR_PDA_MAX_SYMBOLS; the automaton is deterministic: for one
+ * (source, byte) either a single edge that pops nothing, or edges that pop
+ * pairwise different symbols (the paper's system likewise rejects
+ * non-deterministic grammars).  An edge that pops X and pushes X ... reads the
+ * top without removing it.  Synchronous; allocates device memory.
+ */
+#define CSTR_PDA_MAX_PUSH 3
+#define CSTR_PDA_MAX_SYMBOLS 254
+int cstr_load_pda(const int32_t *edge_src, const int32_t *edge_byte, const int32_t *edge_tgt,
+                  const int32_t *pop_off, const int32_t *pops, const int32_t *push_off,
+                  const int32_t *pushes, int32_t n_edges, const uint8_t *accept, int32_t n_states,
+                  int32_t n_symbols, int32_t start_state, cstr_pda_t **out);
+void cstr_free_pda(cstr_pda_t *pda);
+
+/*
+ * Build the token-level PDA P_{G o V} = P_G o T_V of Algorithm 3 (Section 3.2;
+ * Theorem 3: it accepts a token sequence iff the byte PDA accepts its
+ * detokenization).  An edge of P_{G o V} reads a token by chaining the byte
+ * edges of its characters, so it may pop and push several symbols.  Stored
+ * densely per situation (state q, top-of-stack symbol X or "empty stack"):
+ *     mask[q][X] bit v = token v has an edge from q that needs no more of the
+ *                        stack than its top symbol X
+ *     deep[q][X] bit v = whether v has an edge depends on symbols below X
+ *                        (cstr_pda_step decides those against the row's stack)
+ * If eos_id >= 0 that token is allowed exactly in accepting states.
+ * `pda` and `vocab` must outlive the table.  Tokens longer than
+ * 255 / (largest push of an edge) bytes are rejected with CSTR_ERR_SHAPE.
+ * Allocates the table; the build kernel is enqueued on cuda_stream.
+ */
+int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *vocab, int32_t eos_id,
+                         void *cuda_stream, cstr_pda_table_t **out);
+void cstr_free_pda_table(cstr_pda_table_t *table);
+
+/* Shape of a token-level PDA (any pointer may be NULL). */
+int cstr_pda_table_info(const cstr_pda_table_t *table, int32_t *n_states, int32_t *n_symbols,
+                        int32_t *vocab_size, int32_t *mask_words, int32_t *start_state);
+
+/*
+ * Copy one situation's rows to the host: state in [0, n_states), top a symbol
+ * or -1 for the empty stack.
+ *   mask_host, deep_host   HOST uint32 [W] or NULL
+ * Synchronises cuda_stream first.
+ */
+int cstr_pda_table_download(const cstr_pda_table_t *table, int32_t state, int32_t top,
+                            uint32_t *mask_host, uint32_t *deep_host, void *cuda_stream);
+
+/*
+ * Scratch for cstr_pda_step: the step's per-row cells plus one mask row per
+ * batch row (for rows whose allowed set depends on more than the top of their
+ * stack).  One workspace per stream.
+ */
+int cstr_pda_workspace_create(const cstr_pda_table_t *table, int32_t max_batch,
+                              cstr_pda_workspace_t **out);
+void cstr_free_pda_workspace(cstr_pda_workspace_t *ws);
+
+/*
+ * One decoding step of Algorithm 3 for `batch` independent rows:
+ *   A      = tokens with an edge of P_{G o V} that leaves the row's state q and
+ *            whose pops the row's stack s ends with
+ *   masked, token: as in cstr_step
+ *   the matching edge is traversed: q = its target, its pops leave s, its
+ *            pushes are appended
+ *   states  DEVICE int32 [batch], in/out (start: the PDA's start state)
+ *   stacks  DEVICE int32 [batch][stack_cap], in/out, bottom first
+ *   depths  DEVICE int32 [batch], in/out (Algorithm 3 starts from depth 0)
+ * logits, dtype, ld, noise, tokens_out, masked_out, accept_out: as in cstr_step.
+ * A row whose state is -1 or out of range, whose depth is outside
+ * [0, stack_cap] or whose stack holds a symbol outside [0, n_symbols) is
+ * inactive: token -1, state -1, all -infinity.  If the traversed edge would
+ * leave more than stack_cap symbols the token is still emitted and the row
+ * finishes (state -1).  Whenever the new state is -1 the row's stack and depth
+ * are left as they were.  Enqueues three kernels on cuda_stream; no
+ * allocation, no host synchronisation.
+ */
+int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dtype, int64_t ld,
+                  const float *noise, int32_t *states, int32_t *stacks, int32_t *depths,
+                  int32_t stack_cap, int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
+                  int32_t batch, cstr_pda_workspace_t *ws, void *cuda_stream);
+
+/*
+ * Rows since the last call that were inactive for another reason than state
+ * -1, active rows without a selectable token, and rows that finished because
+ * their stack outgrew stack_cap.  Synchronises cuda_stream, then resets the
+ * counters.  Any pointer may be NULL.
+ */
+int cstr_pda_step_status(cstr_pda_workspace_t *ws, void *cuda_stream, int64_t *bad_rows,
+                         int64_t *empty_mask_rows, int64_t *overflow_rows);
 
 /*
  * cstr_step without any allocation, for callers that cannot create a

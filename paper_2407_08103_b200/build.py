@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libcstr.so")
-SOURCES = ["cstr_host.cu", "cstr_build.cu", "cstr_step.cu"]
+SOURCES = ["cstr_host.cu", "cstr_build.cu", "cstr_step.cu", "cstr_pda.cu"]
 
 
 def _nvcc() -> str:

@@ -107,6 +107,51 @@ struct cstr_workspace {
     unsigned long long *counters;  // DEVICE [2] bad-state rows, empty-mask rows
 };
 
+// Byte-level PDA as the kernels read it.  act[(q * NT + t) * 256 + byte] is the
+// index of the edge taken from state q on `byte` when the top of the stack is
+// t, for t = a symbol, n_symbols ("stack empty") or n_symbols + 1 ("top not
+// known": only edges that pop nothing qualify; CSTR_PDA_NEEDCTX if the answer
+// depends on the symbol), or CSTR_PDA_NONE.
+// edge[j] = { target, push0 | push1 << 8 | push2 << 16 | npush << 24 | pop << 28 }.
+#define CSTR_PDA_NONE 0xffffffffu
+#define CSTR_PDA_NEEDCTX 0xfffffffeu
+struct cstr_pda {
+    int device;
+    int32_t n_states, n_symbols, start, n_edges;
+    int32_t NT;          // n_symbols + 2
+    int32_t max_push;    // largest number of symbols one edge pushes
+    uint32_t *act;       // DEVICE [n_states][NT][256]
+    int2 *edge;          // DEVICE [n_edges]
+    uint8_t *accept;     // DEVICE [n_states]
+};
+
+// Token-level PDA: one row of allowed-token words and one of "depends on deeper
+// symbols" words per situation cfg = q * (n_symbols + 1) + top (top = n_symbols
+// for the empty stack); ndeep[cfg] = number of bits set in deep[cfg].
+struct cstr_pda_table {
+    int device;
+    const cstr_pda *pda;
+    const cstr_vocab *vocab;
+    int32_t V, W;
+    int64_t ldw;         // words per row (W rounded up to 32), padding zero
+    int32_t n_cfg;
+    int32_t eos_id;
+    uint32_t *mask;      // DEVICE [n_cfg][ldw]
+    uint32_t *deep;      // DEVICE [n_cfg][ldw]
+    uint32_t *ndeep;     // DEVICE [n_cfg]
+};
+
+struct cstr_pda_workspace {
+    int device;
+    int32_t max_batch;
+    int64_t ldw;
+    unsigned long long *cell;      // DEVICE [max_batch]
+    unsigned int *ticket;          // DEVICE [max_batch]
+    unsigned long long *counters;  // DEVICE [4]: step's two (unused), then bad / empty / overflow
+    const uint32_t **row_mask;     // DEVICE [max_batch]
+    uint32_t *row_buf;             // DEVICE [max_batch][ldw]
+};
+
 // Kernel launchers (defined in cstr_build.cu / cstr_step.cu).
 int cstr_launch_build(cstr_table *table, const cstr_dfa *dfa, cudaStream_t stream);
 
@@ -129,6 +174,13 @@ struct cstr_step_args {
     unsigned int *ticket;          // DEVICE [batch]
     unsigned long long *counters;  // DEVICE [2]
     int device;
+    // Row-mask mode (push-down step): when row_mask is non-null the kernel takes
+    // row r's allowed-token words from row_mask[r] (null = inactive row), needs
+    // no tables, and only emits masked logits and tokens - states, accept flags
+    // and counters are the caller's business.
+    const uint32_t *const *row_mask;   // DEVICE [batch]
+    int32_t V;                         // vocabulary size  (row-mask mode only)
+    int64_t ldw;                       // words readable behind every row pointer
 };
 int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream);
 int cstr_launch_accept(const int32_t *draft, const int32_t *tgt_tok, const int32_t *tgt_state,

@@ -1,0 +1,681 @@
+// Push-down constraints (Section 3; Algorithm 3): the token-level PDA
+// P_{G o V} = P_G o T_V in a dense per-situation form, and the batched decoding
+// step that keeps a state and a stack per row.
+//
+// An edge of P_{G o V} reads a token by chaining the byte edges of its
+// characters, so what it pops depends on how far the chain reaches into the
+// stack it finds.  For all but a handful of tokens the top symbol is enough, so
+// the table keeps, per situation (state q, top symbol X or "empty"), one row of
+// allowed-token bits decided with X alone, and a second row flagging the tokens
+// whose fate depends on deeper symbols.  At decode time a row takes its
+// situation's mask row as is, or - if that situation has flagged tokens - a
+// private copy in which the flagged tokens have been walked against the row's
+// real stack.  The fused step kernel then streams the logits exactly as in the
+// finite-state case, and a small kernel traverses the selected token's edge:
+// it walks the token's bytes from (q, s), which yields the edge's target, pops
+// and pushes without storing variable-length stack edits per table entry.
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "cstr_internal.cuh"
+
+namespace {
+
+constexpr int kLocMax = 256;   // symbols one token may leave on top of the stack it found
+
+struct PdaView {
+    const uint32_t *act;
+    const int2 *edge;
+    int NT;
+    int n_symbols;
+};
+
+enum { WALK_DEAD = 0, WALK_OK = 1, WALK_DEEP = 2 };
+
+// Chain the byte edges of bytes[0..len) from state q.  The stack found is
+// ctx[0..cd) when ctx is non-null (all of it known), else the single symbol
+// known_top (cd = 1) or nothing (cd = 0) with `unknown_below` saying whether
+// unseen symbols lie underneath.  loc receives what the chain leaves on top.
+// WALK_DEEP: the chain reached a byte whose edge depends on an unseen symbol.
+__device__ __forceinline__ int pda_walk(const PdaView &P, int q, const int32_t *ctx, int known_top,
+                                        int cd, bool unknown_below, const uint8_t *bytes, int len,
+                                        uint8_t *loc, int &q_out, int &cd_out, int &nloc_out)
+{
+    int nloc = 0;
+    if (len <= 0)
+        return WALK_DEAD;                           // an empty token never has an edge
+    for (int k = 0; k < len; ++k) {
+        int t;
+        if (nloc > 0) {
+            t = loc[nloc - 1];
+        } else if (cd > 0) {
+            t = ctx ? ctx[cd - 1] : known_top;
+            if ((unsigned)t >= (unsigned)P.n_symbols)
+                return WALK_DEAD;
+        } else {
+            t = unknown_below ? P.n_symbols + 1 : P.n_symbols;
+        }
+        const uint32_t a = __ldg(P.act + ((long long)q * P.NT + t) * 256 + bytes[k]);
+        if (a == CSTR_PDA_NONE)
+            return WALK_DEAD;
+        if (a == CSTR_PDA_NEEDCTX)
+            return WALK_DEEP;
+        const int2 e = __ldg(P.edge + a);
+        const unsigned meta = (unsigned)e.y;
+        if (meta >> 28) {                           // pops the symbol it looked at
+            if (nloc > 0)
+                --nloc;
+            else
+                --cd;
+        }
+        const int npush = (meta >> 24) & 7;
+        if (nloc + npush > kLocMax)
+            return WALK_DEAD;                       // excluded by the build's length check
+        for (int i = 0; i < npush; ++i)
+            loc[nloc++] = (uint8_t)(meta >> (8 * i));
+        q = e.x;
+    }
+    q_out = q;
+    cd_out = cd;
+    nloc_out = nloc;
+    return WALK_OK;
+}
+
+// One warp per (situation, 32-token word): lane = token.
+__global__ void __launch_bounds__(256)
+pda_build_kernel(PdaView P, const uint8_t *__restrict__ accept, const uint8_t *__restrict__ vbytes,
+                 const uint32_t *__restrict__ voff, int V, int W, long long ldw, int eos_id,
+                 uint32_t *__restrict__ mask, uint32_t *__restrict__ deep,
+                 uint32_t *__restrict__ ndeep)
+{
+    const int lane = threadIdx.x & 31;
+    const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int cfg = blockIdx.y;
+    if (w >= W)
+        return;
+    const int q = cfg / (P.n_symbols + 1);
+    const int top = cfg - q * (P.n_symbols + 1);   // n_symbols = empty stack
+    const bool has_top = top < P.n_symbols;
+    const int v = w * 32 + lane;
+    int res = WALK_DEAD;
+    if (v < V) {
+        if (v == eos_id) {
+            res = accept[q] ? WALK_OK : WALK_DEAD;
+        } else {
+            uint8_t loc[kLocMax];
+            int q2, cd2, nloc2;
+            const uint32_t b = voff[v], e = voff[v + 1];
+            res = pda_walk(P, q, nullptr, top, has_top ? 1 : 0, has_top, vbytes + b, (int)(e - b),
+                           loc, q2, cd2, nloc2);
+        }
+    }
+    const unsigned ok = __ballot_sync(0xffffffffu, res == WALK_OK);
+    const unsigned dp = __ballot_sync(0xffffffffu, res == WALK_DEEP);
+    if (lane == 0) {
+        mask[(long long)cfg * ldw + w] = ok;
+        deep[(long long)cfg * ldw + w] = dp;
+        if (dp)
+            atomicAdd(ndeep + cfg, (uint32_t)__popc(dp));
+    }
+}
+
+struct PdaStepParams {
+    PdaView P;
+    const uint8_t *accept;
+    const uint8_t *vbytes;
+    const uint32_t *voff;
+    const uint32_t *mask, *deep, *ndeep;
+    long long ldw;
+    int n_states, V, eos_id;
+    int32_t *states, *stacks, *depths;
+    int cap, batch;
+    const int32_t *tokens;
+    uint8_t *accept_out;
+    const uint32_t **row_mask;
+    uint32_t *row_buf;
+    unsigned long long *counters;   // [0] bad, [1] empty, [2] overflow
+};
+
+// One warp per row: find the row's situation and point the step at its mask row,
+// or at a private copy in which the tokens that depend on deeper stack symbols
+// have been decided against the row's stack.
+__global__ void __launch_bounds__(128)
+pda_prepare_kernel(const __grid_constant__ PdaStepParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= p.batch)
+        return;
+    const int q = p.states[r];
+    const int d = p.depths[r];
+    const int32_t *s = p.stacks + (long long)r * p.cap;
+    bool ok = q >= 0 && q < p.n_states && d >= 0 && d <= p.cap;
+    if (ok) {
+        bool bad = false;
+        for (int i = lane; i < d; i += 32)
+            bad |= (unsigned)s[i] >= (unsigned)p.P.n_symbols;
+        ok = !__any_sync(0xffffffffu, bad);
+    }
+    if (!ok) {
+        if (lane == 0)
+            p.row_mask[r] = nullptr;
+        return;
+    }
+    const int top = d > 0 ? s[d - 1] : p.P.n_symbols;
+    const long long cfg = (long long)q * (p.P.n_symbols + 1) + top;
+    const uint32_t *mrow = p.mask + cfg * p.ldw;
+    if (p.ndeep[cfg] == 0) {
+        if (lane == 0)
+            p.row_mask[r] = mrow;
+        return;
+    }
+    const uint32_t *drow = p.deep + cfg * p.ldw;
+    uint32_t *out = p.row_buf + (long long)r * p.ldw;
+    for (long long w = lane; w < p.ldw; w += 32) {
+        uint32_t m = mrow[w];
+        uint32_t dw = drow[w];
+        while (dw) {
+            const int b = __ffs((int)dw) - 1;
+            dw &= dw - 1;
+            const int v = (int)w * 32 + b;
+            uint8_t loc[kLocMax];
+            int q2, cd2, nloc2;
+            const uint32_t b0 = p.voff[v], b1 = p.voff[v + 1];
+            if (pda_walk(p.P, q, s, 0, d, false, p.vbytes + b0, (int)(b1 - b0), loc, q2, cd2,
+                         nloc2) == WALK_OK)
+                m |= 1u << b;
+        }
+        out[w] = m;
+    }
+    if (lane == 0)
+        p.row_mask[r] = out;
+}
+
+// One thread per row: traverse the edge of the selected token.
+__global__ void __launch_bounds__(128)
+pda_advance_kernel(const __grid_constant__ PdaStepParams p)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= p.batch)
+        return;
+    const int q = p.states[r];
+    const int tok = p.tokens[r];
+    int q2 = CSTR_DEAD;
+    if (p.row_mask[r] == nullptr) {
+        if (q != -1)
+            atomicAdd(p.counters + 0, 1ull);
+    } else if (tok < 0) {
+        atomicAdd(p.counters + 1, 1ull);
+    } else if (tok != p.eos_id) {
+        const int d = p.depths[r];
+        int32_t *s = p.stacks + (long long)r * p.cap;
+        uint8_t loc[kLocMax];
+        int qn, cd, nloc;
+        const uint32_t b0 = p.voff[tok], b1 = p.voff[tok + 1];
+        if (pda_walk(p.P, q, s, 0, d, false, p.vbytes + b0, (int)(b1 - b0), loc, qn, cd, nloc) ==
+            WALK_OK) {
+            if (cd + nloc > p.cap) {
+                atomicAdd(p.counters + 2, 1ull);
+            } else {
+                for (int i = 0; i < nloc; ++i)
+                    s[cd + i] = loc[i];
+                p.depths[r] = cd + nloc;
+                q2 = qn;
+            }
+        }
+    }
+    p.states[r] = q2;
+    if (p.accept_out)
+        p.accept_out[r] = (q2 >= 0) ? (uint8_t)(p.accept[q2] != 0) : (uint8_t)0;
+}
+
+int check_device(int handle_device, const char *what)
+{
+    int cur = -1;
+    CSTR_CUDA_TRY(cudaGetDevice(&cur));
+    if (cur != handle_device)
+        return cstr_fail(CSTR_ERR_DEVICE, "%s was created on device %d but device %d is current",
+                         what, handle_device, cur);
+    return CSTR_OK;
+}
+
+int cuda_rc(cudaError_t e, const char *who)
+{
+    return cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA, "%s: %s", who,
+                     cudaGetErrorString(e));
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ PDA
+
+extern "C" void cstr_free_pda(cstr_pda_t *p)
+{
+    if (!p)
+        return;
+    cudaFree(p->act);
+    cudaFree(p->edge);
+    cudaFree(p->accept);
+    delete p;
+}
+
+extern "C" int cstr_load_pda(const int32_t *edge_src, const int32_t *edge_byte,
+                             const int32_t *edge_tgt, const int32_t *pop_off, const int32_t *pops,
+                             const int32_t *push_off, const int32_t *pushes, int32_t n_edges,
+                             const uint8_t *accept, int32_t n_states, int32_t n_symbols,
+                             int32_t start_state, cstr_pda_t **out)
+{
+    if (!out || !accept || !pop_off || !push_off ||
+        (n_edges > 0 && (!edge_src || !edge_byte || !edge_tgt)))
+        return cstr_fail(CSTR_ERR_NULL, "cstr_load_pda: null pointer");
+    *out = nullptr;
+    if (n_states < 1 || n_edges < 0)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_pda: n_states = %d, n_edges = %d", n_states,
+                         n_edges);
+    if (n_symbols < 0 || n_symbols > CSTR_PDA_MAX_SYMBOLS)
+        return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: n_symbols = %d, need 0..%d", n_symbols,
+                         CSTR_PDA_MAX_SYMBOLS);
+    if (start_state < 0 || start_state >= n_states)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_load_pda: start_state %d outside [0, %d)",
+                         start_state, n_states);
+    const int NT = n_symbols + 2;
+    const int64_t slots = (int64_t)n_states * NT * 256;
+    if (slots > ((int64_t)1 << 28))
+        return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: %d states x %d symbols exceed the lookup "
+                         "table limit of 2^28 entries", n_states, n_symbols);
+    if (pop_off[0] != 0 || push_off[0] != 0)
+        return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: pop_off[0] and push_off[0] must be 0");
+
+    std::vector<uint32_t> act;
+    std::vector<int2> edges;
+    std::vector<uint8_t> flags;
+    int max_push = 0;
+    try {
+        act.assign((size_t)slots, CSTR_PDA_NONE);
+        edges.resize((size_t)n_edges);
+        flags.resize((size_t)n_states);
+    } catch (const std::bad_alloc &) {
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_pda: out of host memory");
+    }
+    for (int32_t q = 0; q < n_states; ++q)
+        flags[q] = accept[q] ? 1 : 0;
+    for (int32_t j = 0; j < n_edges; ++j) {
+        const int32_t q = edge_src[j], b = edge_byte[j], t = edge_tgt[j];
+        if (q < 0 || q >= n_states || t < 0 || t >= n_states)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d joins states %d -> %d outside "
+                             "[0, %d)", j, q, t, n_states);
+        if (b < 0 || b > 255)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d reads %d; every edge must read "
+                             "one byte 0..255 (no epsilon input)", j, b);
+        const int32_t np = pop_off[j + 1] - pop_off[j], nu = push_off[j + 1] - push_off[j];
+        if (np < 0 || nu < 0)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: offsets decrease at edge %d", j);
+        if (np > 1)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d pops %d symbols, at most 1 "
+                             "supported", j, np);
+        if (nu > CSTR_PDA_MAX_PUSH)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d pushes %d symbols, at most %d "
+                             "supported", j, nu, CSTR_PDA_MAX_PUSH);
+        if ((np > 0 && !pops) || (nu > 0 && !pushes))
+            return cstr_fail(CSTR_ERR_NULL, "cstr_load_pda: null pops / pushes");
+        unsigned meta = (unsigned)nu << 24 | (unsigned)np << 28;
+        for (int32_t i = 0; i < nu; ++i) {
+            const int32_t y = pushes[push_off[j] + i];
+            if (y < 0 || y >= n_symbols)
+                return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d pushes symbol %d outside "
+                                 "[0, %d)", j, y, n_symbols);
+            meta |= (unsigned)y << (8 * i);
+        }
+        if (nu > max_push)
+            max_push = nu;
+        edges[j] = make_int2(t, (int)meta);
+        uint32_t *row = act.data() + (size_t)q * NT * 256 + b;   // row[t * 256]
+        bool clash = false;
+        if (np == 0) {
+            for (int tt = 0; tt < NT; ++tt) {
+                clash |= row[(size_t)tt * 256] != CSTR_PDA_NONE;
+                row[(size_t)tt * 256] = (uint32_t)j;
+            }
+        } else {
+            const int32_t x = pops[pop_off[j]];
+            if (x < 0 || x >= n_symbols)
+                return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: edge %d pops symbol %d outside "
+                                 "[0, %d)", j, x, n_symbols);
+            uint32_t &unknown = row[(size_t)(n_symbols + 1) * 256];
+            clash = row[(size_t)x * 256] != CSTR_PDA_NONE ||
+                    (unknown != CSTR_PDA_NONE && unknown != CSTR_PDA_NEEDCTX);
+            row[(size_t)x * 256] = (uint32_t)j;
+            unknown = CSTR_PDA_NEEDCTX;
+        }
+        if (clash)
+            return cstr_fail(CSTR_ERR_PDA, "cstr_load_pda: not deterministic: edge %d (state %d, "
+                             "byte %d) competes with an earlier edge", j, q, b);
+    }
+
+    cstr_pda *p = new (std::nothrow) cstr_pda();
+    if (!p)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_pda: out of host memory");
+    memset(p, 0, sizeof *p);
+    p->n_states = n_states;
+    p->n_symbols = n_symbols;
+    p->start = start_state;
+    p->n_edges = n_edges;
+    p->NT = NT;
+    p->max_push = max_push;
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&p->act, (size_t)slots * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&p->edge, ((size_t)n_edges + 1) * sizeof(int2));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&p->accept, (size_t)n_states);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->act, act.data(), (size_t)slots * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && n_edges > 0)
+        e = cudaMemcpy(p->edge, edges.data(), (size_t)n_edges * sizeof(int2),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->accept, flags.data(), (size_t)n_states, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        const int rc = cuda_rc(e, "cstr_load_pda");
+        cstr_free_pda(p);
+        return rc;
+    }
+    *out = p;
+    return CSTR_OK;
+}
+
+// ---------------------------------------------------------------- table
+
+extern "C" void cstr_free_pda_table(cstr_pda_table_t *t)
+{
+    if (!t)
+        return;
+    cudaFree(t->mask);
+    cudaFree(t->deep);
+    cudaFree(t->ndeep);
+    delete t;
+}
+
+extern "C" int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *vocab,
+                                    int32_t eos_id, void *cuda_stream, cstr_pda_table_t **out)
+{
+    if (!pda || !vocab || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_build_pda_table: null pointer");
+    *out = nullptr;
+    int rc = check_device(pda->device, "PDA");
+    if (rc)
+        return rc;
+    if (vocab->device != pda->device)
+        return cstr_fail(CSTR_ERR_DEVICE, "cstr_build_pda_table: PDA and vocabulary on different "
+                         "devices");
+    if (eos_id < -1 || eos_id >= vocab->V)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_build_pda_table: eos_id %d outside [-1, %d)", eos_id,
+                         vocab->V);
+    if ((int64_t)vocab->max_len * (pda->max_push > 0 ? pda->max_push : 1) > kLocMax - 1)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_build_pda_table: a token of %u bytes with edges "
+                         "that push up to %d symbols could leave more than %d symbols",
+                         vocab->max_len, pda->max_push, kLocMax - 1);
+    cstr_pda_table *t = new (std::nothrow) cstr_pda_table();
+    if (!t)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_build_pda_table: out of host memory");
+    memset(t, 0, sizeof *t);
+    t->device = pda->device;
+    t->pda = pda;
+    t->vocab = vocab;
+    t->V = vocab->V;
+    t->W = (vocab->V + 31) / 32;
+    t->ldw = ((int64_t)t->W + 31) / 32 * 32;
+    t->eos_id = eos_id;
+    const int64_t n_cfg = (int64_t)pda->n_states * (pda->n_symbols + 1);
+    if (n_cfg > 65535) {
+        delete t;
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_build_pda_table: %lld (state, top) situations, at "
+                         "most 65535 supported", (long long)n_cfg);
+    }
+    t->n_cfg = (int32_t)n_cfg;
+    const size_t row_bytes = (size_t)n_cfg * (size_t)t->ldw * 4;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMalloc((void **)&t->mask, row_bytes);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->deep, row_bytes);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->ndeep, (size_t)n_cfg * 4);
+    if (e == cudaSuccess)
+        e = cudaMemsetAsync(t->mask, 0, row_bytes, stream);
+    if (e == cudaSuccess)
+        e = cudaMemsetAsync(t->deep, 0, row_bytes, stream);
+    if (e == cudaSuccess)
+        e = cudaMemsetAsync(t->ndeep, 0, (size_t)n_cfg * 4, stream);
+    if (e == cudaSuccess) {
+        PdaView P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
+        const int warps = 8;
+        dim3 grid((unsigned)((t->W + warps - 1) / warps), (unsigned)n_cfg);
+        pda_build_kernel<<<grid, warps * 32, 0, stream>>>(P, pda->accept, vocab->bytes, vocab->off,
+                                                          t->V, t->W, t->ldw, eos_id, t->mask,
+                                                          t->deep, t->ndeep);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        rc = cuda_rc(e, "cstr_build_pda_table");
+        cstr_free_pda_table(t);
+        return rc;
+    }
+    *out = t;
+    return CSTR_OK;
+}
+
+extern "C" int cstr_pda_table_info(const cstr_pda_table_t *t, int32_t *n_states,
+                                   int32_t *n_symbols, int32_t *vocab_size, int32_t *mask_words,
+                                   int32_t *start_state)
+{
+    if (!t)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_table_info: null table");
+    if (n_states)
+        *n_states = t->pda->n_states;
+    if (n_symbols)
+        *n_symbols = t->pda->n_symbols;
+    if (vocab_size)
+        *vocab_size = t->V;
+    if (mask_words)
+        *mask_words = t->W;
+    if (start_state)
+        *start_state = t->pda->start;
+    return CSTR_OK;
+}
+
+extern "C" int cstr_pda_table_download(const cstr_pda_table_t *t, int32_t state, int32_t top,
+                                       uint32_t *mask_host, uint32_t *deep_host, void *cuda_stream)
+{
+    if (!t)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_table_download: null table");
+    int rc = check_device(t->device, "PDA table");
+    if (rc)
+        return rc;
+    if (state < 0 || state >= t->pda->n_states || top < -1 || top >= t->pda->n_symbols)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_table_download: (state %d, top %d) outside "
+                         "[0, %d) x [-1, %d)", state, top, t->pda->n_states, t->pda->n_symbols);
+    CSTR_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    const int64_t cfg = (int64_t)state * (t->pda->n_symbols + 1) + (top < 0 ? t->pda->n_symbols : top);
+    if (mask_host)
+        CSTR_CUDA_TRY(cudaMemcpy(mask_host, t->mask + cfg * t->ldw, (size_t)t->W * 4,
+                                 cudaMemcpyDeviceToHost));
+    if (deep_host)
+        CSTR_CUDA_TRY(cudaMemcpy(deep_host, t->deep + cfg * t->ldw, (size_t)t->W * 4,
+                                 cudaMemcpyDeviceToHost));
+    return CSTR_OK;
+}
+
+// ------------------------------------------------------------ workspace
+
+extern "C" void cstr_free_pda_workspace(cstr_pda_workspace_t *ws)
+{
+    if (!ws)
+        return;
+    cudaFree(ws->cell);
+    cudaFree(ws->ticket);
+    cudaFree(ws->counters);
+    cudaFree((void *)ws->row_mask);
+    cudaFree(ws->row_buf);
+    delete ws;
+}
+
+extern "C" int cstr_pda_workspace_create(const cstr_pda_table_t *table, int32_t max_batch,
+                                         cstr_pda_workspace_t **out)
+{
+    if (!table || !out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_workspace_create: null pointer");
+    *out = nullptr;
+    if (max_batch < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_workspace_create: max_batch = %d, need >= 1",
+                         max_batch);
+    int rc = check_device(table->device, "PDA table");
+    if (rc)
+        return rc;
+    cstr_pda_workspace *ws = new (std::nothrow) cstr_pda_workspace();
+    if (!ws)
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_pda_workspace_create: out of host memory");
+    memset(ws, 0, sizeof *ws);
+    ws->device = table->device;
+    ws->max_batch = max_batch;
+    ws->ldw = table->ldw;
+    const size_t buf_bytes = (size_t)max_batch * (size_t)ws->ldw * 4;
+    cudaError_t e = cudaMalloc((void **)&ws->cell, (size_t)max_batch * 8);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->ticket, (size_t)max_batch * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->counters, 5 * 8);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->row_mask, (size_t)max_batch * sizeof(void *));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&ws->row_buf, buf_bytes);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->cell, 0, (size_t)max_batch * 8);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->ticket, 0, (size_t)max_batch * 4);
+    if (e == cudaSuccess)
+        e = cudaMemset(ws->counters, 0, 5 * 8);
+    if (e == cudaSuccess)
+        e = cudaMemset((void *)ws->row_mask, 0, (size_t)max_batch * sizeof(void *));
+    if (e != cudaSuccess) {
+        rc = cuda_rc(e, "cstr_pda_workspace_create");
+        cstr_free_pda_workspace(ws);
+        return rc;
+    }
+    *out = ws;
+    return CSTR_OK;
+}
+
+// ----------------------------------------------------------------- step
+
+extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dtype,
+                             int64_t ld, const float *noise, int32_t *states, int32_t *stacks,
+                             int32_t *depths, int32_t stack_cap, int32_t *tokens_out,
+                             void *masked_out, uint8_t *accept_out, int32_t batch,
+                             cstr_pda_workspace_t *ws, void *cuda_stream)
+{
+    if (!table || !logits || !states || !stacks || !depths || !tokens_out || !masked_out || !ws)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_step: null pointer");
+    if (dtype != CSTR_F32 && dtype != CSTR_BF16)
+        return cstr_fail(CSTR_ERR_DTYPE, "cstr_pda_step: unknown dtype %d", dtype);
+    if (batch < 0 || stack_cap < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_step: batch = %d, stack_cap = %d", batch,
+                         stack_cap);
+    if (batch > ws->max_batch || ws->ldw != table->ldw)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_pda_step: workspace holds %d rows of %lld words, "
+                         "the call needs %d rows of %lld", ws->max_batch, (long long)ws->ldw, batch,
+                         (long long)table->ldw);
+    if (ld < table->V)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_pda_step: ld = %lld is below V = %d", (long long)ld,
+                         table->V);
+    int rc = check_device(ws->device, "PDA workspace");
+    if (rc)
+        return rc;
+    if (table->device != ws->device)
+        return cstr_fail(CSTR_ERR_DEVICE, "cstr_pda_step: table is on another device");
+    if (batch == 0)
+        return CSTR_OK;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const cstr_pda *pda = table->pda;
+
+    PdaStepParams p;
+    memset(&p, 0, sizeof p);
+    p.P.act = pda->act;
+    p.P.edge = pda->edge;
+    p.P.NT = pda->NT;
+    p.P.n_symbols = pda->n_symbols;
+    p.accept = pda->accept;
+    p.vbytes = table->vocab->bytes;
+    p.voff = table->vocab->off;
+    p.mask = table->mask;
+    p.deep = table->deep;
+    p.ndeep = table->ndeep;
+    p.ldw = table->ldw;
+    p.n_states = pda->n_states;
+    p.V = table->V;
+    p.eos_id = table->eos_id;
+    p.states = states;
+    p.stacks = stacks;
+    p.depths = depths;
+    p.cap = stack_cap;
+    p.batch = batch;
+    p.tokens = tokens_out;
+    p.accept_out = accept_out;
+    p.row_mask = ws->row_mask;
+    p.row_buf = ws->row_buf;
+    p.counters = ws->counters + 2;
+
+    pda_prepare_kernel<<<(batch + 3) / 4, 128, 0, stream>>>(p);
+    CSTR_CUDA_TRY(cudaGetLastError());
+
+    cstr_step_args a;
+    memset(&a, 0, sizeof a);
+    a.n_tables = 1;
+    a.logits = logits;
+    a.dtype = dtype;
+    a.ld = ld;
+    a.noise = noise;
+    a.states = states;
+    a.states_out = states;
+    a.tokens_out = tokens_out;
+    a.masked_out = masked_out;
+    a.batch = batch;
+    a.cell = ws->cell;
+    a.ticket = ws->ticket;
+    a.counters = ws->counters;
+    a.device = ws->device;
+    a.row_mask = ws->row_mask;
+    a.V = table->V;
+    a.ldw = table->ldw;
+    rc = cstr_launch_step(a, stream);
+    if (rc)
+        return rc;
+
+    pda_advance_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(p);
+    CSTR_CUDA_TRY(cudaGetLastError());
+    return CSTR_OK;
+}
+
+extern "C" int cstr_pda_step_status(cstr_pda_workspace_t *ws, void *cuda_stream, int64_t *bad_rows,
+                                    int64_t *empty_mask_rows, int64_t *overflow_rows)
+{
+    if (!ws)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_step_status: null workspace");
+    int rc = check_device(ws->device, "PDA workspace");
+    if (rc)
+        return rc;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long host[3] = {0, 0, 0};
+    CSTR_CUDA_TRY(cudaMemcpyAsync(host, ws->counters + 2, 24, cudaMemcpyDeviceToHost, stream));
+    CSTR_CUDA_TRY(cudaMemsetAsync(ws->counters + 2, 0, 24, stream));
+    CSTR_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (bad_rows)
+        *bad_rows = (int64_t)host[0];
+    if (empty_mask_rows)
+        *empty_mask_rows = (int64_t)host[1];
+    if (overflow_rows)
+        *overflow_rows = (int64_t)host[2];
+    return CSTR_OK;
+}

@@ -45,6 +45,7 @@ struct StepParams {
     unsigned long long *cell;
     unsigned int *ticket;
     unsigned long long *counters;
+    const uint32_t *const *row_mask;   // non-null: per-row mask pointers instead of tables
     long long ld;
     int V;
     int n_tables;
@@ -101,6 +102,13 @@ __device__ __forceinline__ RowCtx row_context(const StepParams &p)
     RowCtx c;
     c.r = blockIdx.x / p.nchunks;
     c.chunk = blockIdx.x - c.r * p.nchunks;
+    if (p.row_mask) {                               // the caller resolved the rows' masks
+        c.t = 0;
+        c.q = 0;
+        c.mrow = p.row_mask[c.r];
+        c.active = c.mrow != nullptr;
+        return c;
+    }
     c.t = p.row_table ? p.row_table[c.r] : 0;
     c.q = p.states[c.r];
     const bool table_ok = c.t >= 0 && c.t < p.n_tables;
@@ -142,6 +150,11 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     __threadfence();
     const unsigned long long key = atomicExch(p.cell + c.r, 0ull);
     p.ticket[c.r] = 0u;
+    if (p.row_mask) {                               // the caller advances its own automaton
+        p.tokens[c.r] = (c.active && key != 0ull)
+                            ? (int)(0xffffffffu - (unsigned)(key & 0xffffffffull)) : -1;
+        return;
+    }
     int tok = -1, q2 = CSTR_DEAD;
     const TableDesc &tb = p.tab[c.t];
     if (c.active && key != 0ull) {
@@ -430,7 +443,8 @@ int sm_count(int device)
 int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
 {
     StepParams p;
-    for (int i = 0; i < CSTR_MAX_TABLES; ++i) {
+    memset(&p, 0, sizeof p);
+    for (int i = 0; i < CSTR_MAX_TABLES && !a.row_mask; ++i) {
         const cstr_table *t = a.tables[i < a.n_tables ? i : 0];
         p.tab[i].mask = t->mask;
         p.tab[i].next = t->next;
@@ -441,7 +455,9 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         p.tab[i].wide = t->wide;
         p.tab[i].code_shift = t->code_shift;
     }
-    const cstr_table *t0 = a.tables[0];
+    if (a.row_mask)
+        p.tab[0].ldw = a.ldw;
+    p.row_mask = a.row_mask;
     p.row_table = a.row_table;
     p.logits = a.logits;
     p.noise = a.noise;
@@ -454,7 +470,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     p.ticket = a.ticket;
     p.counters = a.counters;
     p.ld = a.ld;
-    p.V = t0->V;
+    p.V = a.row_mask ? a.V : a.tables[0]->V;
     p.n_tables = a.n_tables;
 
     const bool bf16 = a.dtype == CSTR_BF16;

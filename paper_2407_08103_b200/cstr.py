@@ -27,6 +27,9 @@ EXPORTS = [
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
     "cstr_step", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
     "cstr_step_static", "cstr_last_error",
+    "cstr_load_pda", "cstr_free_pda", "cstr_build_pda_table", "cstr_free_pda_table",
+    "cstr_pda_table_info", "cstr_pda_table_download", "cstr_pda_workspace_create",
+    "cstr_free_pda_workspace", "cstr_pda_step", "cstr_pda_step_status",
 ]
 
 _lib = None
@@ -52,7 +55,8 @@ def lib():
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
         L.cstr_last_error.restype = ctypes.c_char_p
-        for name in ("cstr_free_dfa", "cstr_free_vocab", "cstr_free_table", "cstr_free_workspace"):
+        for name in ("cstr_free_dfa", "cstr_free_vocab", "cstr_free_table", "cstr_free_workspace",
+                     "cstr_free_pda", "cstr_free_pda_table", "cstr_free_pda_workspace"):
             getattr(L, name).restype = None
         _lib = L
     return _lib
@@ -111,6 +115,20 @@ class Table(_Handle):
 
 class Workspace(_Handle):
     _free = "cstr_free_workspace"
+
+
+class Pda(_Handle):
+    _free = "cstr_free_pda"
+
+
+class PdaTable(_Handle):
+    _free = "cstr_free_pda_table"
+    pda = None    # keep the handles the table refers to alive
+    vocab = None
+
+
+class PdaWorkspace(_Handle):
+    _free = "cstr_free_pda_workspace"
 
 
 def cstr_load_dfa(trans, accept, start_state=0) -> Dfa:
@@ -314,6 +332,102 @@ def cstr_step_status(ws: Workspace, stream=None):
     bad, empty = ctypes.c_int64(), ctypes.c_int64()
     _check(lib().cstr_step_status(ws.ptr, _stream_ptr(stream), ctypes.byref(bad), ctypes.byref(empty)))
     return int(bad.value), int(empty.value)
+
+
+def cstr_load_pda(edge_src, edge_byte, edge_tgt, pop_off, pops, push_off, pushes, accept,
+                  n_symbols: int, start_state: int = 0) -> Pda:
+    """Byte-level PDA from flat int32 edge arrays (see ``cstr_load_pda`` in cstr.h)."""
+    arrs = [np.ascontiguousarray(a, dtype=np.int32)
+            for a in (edge_src, edge_byte, edge_tgt, pop_off, pops, push_off, pushes)]
+    accept = np.ascontiguousarray(accept, dtype=np.uint8)
+    n_edges = arrs[0].size
+    if arrs[1].size != n_edges or arrs[2].size != n_edges or arrs[3].size != n_edges + 1 \
+            or arrs[5].size != n_edges + 1:
+        raise ValueError("edge arrays must have n_edges entries, offsets n_edges + 1")
+    if n_edges and (arrs[4].size < arrs[3][-1] or arrs[6].size < arrs[5][-1]):
+        raise ValueError("pops / pushes shorter than their offsets say")
+    out = ctypes.c_void_p()
+    _check(lib().cstr_load_pda(*[_np_ptr(a) for a in arrs], ctypes.c_int32(n_edges),
+                               _np_ptr(accept), ctypes.c_int32(accept.size),
+                               ctypes.c_int32(n_symbols), ctypes.c_int32(start_state),
+                               ctypes.byref(out)))
+    return Pda(out)
+
+
+def cstr_build_pda_table(pda: Pda, vocab: Vocab, eos_id: int = -1, stream=None) -> PdaTable:
+    out = ctypes.c_void_p()
+    _check(lib().cstr_build_pda_table(pda.ptr, vocab.ptr, ctypes.c_int32(eos_id),
+                                      _stream_ptr(stream), ctypes.byref(out)))
+    t = PdaTable(out)
+    t.pda, t.vocab = pda, vocab
+    return t
+
+
+def cstr_pda_table_info(table: PdaTable):
+    vals = [ctypes.c_int32() for _ in range(5)]
+    _check(lib().cstr_pda_table_info(table.ptr, *[ctypes.byref(v) for v in vals]))
+    keys = ("n_states", "n_symbols", "vocab_size", "mask_words", "start_state")
+    return {k: int(v.value) for k, v in zip(keys, vals)}
+
+
+def cstr_pda_table_download(table: PdaTable, state: int, top: int = -1, stream=None):
+    """(mask, deep) uint32 ``[W]`` rows of one situation; ``top`` = -1 for the empty stack."""
+    W = cstr_pda_table_info(table)["mask_words"]
+    mask = np.empty(W, dtype=np.uint32)
+    deep = np.empty(W, dtype=np.uint32)
+    _check(lib().cstr_pda_table_download(table.ptr, ctypes.c_int32(state), ctypes.c_int32(top),
+                                         _np_ptr(mask), _np_ptr(deep), _stream_ptr(stream)))
+    return mask, deep
+
+
+def cstr_pda_workspace_create(table: PdaTable, max_batch: int) -> PdaWorkspace:
+    out = ctypes.c_void_p()
+    _check(lib().cstr_pda_workspace_create(table.ptr, ctypes.c_int32(max_batch), ctypes.byref(out)))
+    return PdaWorkspace(out)
+
+
+def cstr_pda_step(table: PdaTable, logits, states, stacks, depths, tokens_out, masked_out,
+                  ws: PdaWorkspace, noise=None, accept_out=None, stream=None) -> None:
+    """Enqueue one step of Algorithm 3.  CUDA tensors: ``logits`` / ``masked_out`` /
+    ``noise`` as in ``cstr_step``; ``states`` / ``depths`` / ``tokens_out`` int32 ``[B]``;
+    ``stacks`` int32 ``[B][cap]`` (bottom first)."""
+    import torch
+    if logits.dtype == torch.float32:
+        dtype = CSTR_F32
+    elif logits.dtype == torch.bfloat16:
+        dtype = CSTR_BF16
+    else:
+        raise TypeError("logits must be float32 or bfloat16")
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [B][ld] with unit inner stride")
+    batch = logits.shape[0]
+    for name, t in (("masked_out", masked_out), ("noise", noise)):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0)
+                              or t.shape[0] != batch):
+            raise ValueError("%s must have the layout of logits" % name)
+    if masked_out.dtype != logits.dtype:
+        raise TypeError("masked_out must have the dtype of logits")
+    if noise is not None and noise.dtype != torch.float32:
+        raise TypeError("noise must be float32")
+    for name, t, dt in (("states", states, torch.int32), ("depths", depths, torch.int32),
+                        ("tokens_out", tokens_out, torch.int32),
+                        ("accept_out", accept_out, torch.uint8)):
+        if t is not None and (t.dtype != dt or t.numel() < batch or not t.is_contiguous()):
+            raise ValueError("%s must be a contiguous %s tensor with one entry per row" % (name, dt))
+    if stacks.dtype != torch.int32 or stacks.dim() != 2 or stacks.shape[0] < batch \
+            or not stacks.is_contiguous():
+        raise ValueError("stacks must be a contiguous int32 tensor [B][cap]")
+    _check(lib().cstr_pda_step(table.ptr, _dev_ptr(logits), ctypes.c_int32(dtype),
+                               ctypes.c_int64(logits.stride(0)), _dev_ptr(noise), _dev_ptr(states),
+                               _dev_ptr(stacks), _dev_ptr(depths), ctypes.c_int32(stacks.shape[1]),
+                               _dev_ptr(tokens_out), _dev_ptr(masked_out), _dev_ptr(accept_out),
+                               ctypes.c_int32(batch), ws.ptr, _stream_ptr(stream)))
+
+
+def cstr_pda_step_status(ws: PdaWorkspace, stream=None):
+    vals = [ctypes.c_int64() for _ in range(3)]
+    _check(lib().cstr_pda_step_status(ws.ptr, _stream_ptr(stream), *[ctypes.byref(v) for v in vals]))
+    return tuple(int(v.value) for v in vals)
 
 
 def cstr_last_error() -> str:

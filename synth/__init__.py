@@ -7,7 +7,8 @@ selecting, advancing) lives in this package, so both the CUDA library and the
 CPU oracle can be fed from it without sharing any code with each other.
 """
 
-from .vocab import make_vocab_api, make_vocab_geometric, vocab_from_strings  # noqa: F401
+from .vocab import (make_vocab_api, make_vocab_geometric, make_vocab_json,  # noqa: F401
+                    vocab_from_strings)
 from .constraints import (  # noqa: F401
     API_CALL_REGEX,
     FLAT_JSON_REGEX,

@@ -69,3 +69,26 @@ def make_vocab_geometric(vocab_size: int, seed: int = 0, p: float = 0.3, cap: in
     other = _OTHER_PRINTABLE[rng.integers(0, _OTHER_PRINTABLE.size, size=total)]
     chars = np.where(kind < 0.60, lower, np.where(kind < 0.75, np.uint8(0x20), other))
     return _pack(lengths, chars)
+
+
+# Multi-character structural tokens of the kind real LM vocabularies hold for
+# JSON-like text: they cross terminal boundaries and open or close several
+# nesting levels at once.
+_JSON_TOKENS = [
+    b"]]", b"]]]", b"]]]]", b"}}", b"}}}", b"}]", b"]}", b"}]}", b"]}]", b'"]', b'"}', b'"]]',
+    b'"}]', b'":', b'": ', b'":[', b'":{', b'": [', b'": {', b", ", b',"', b', "', b"[[", b"[[[",
+    b"[{", b'[{"', b'{"', b'[]', b"{}", b"[],", b"{},", b"[]]", b"{}]", b"{}}", b"[]}", b"],",
+    b"], ", b"},", b"}, ", b'},{"', b"],[", b"], [", b"true", b"false", b"null", b"true,",
+    b"false]", b"null}", b"tru", b"fal", b"nul", b"1]", b"1}", b"12", b"-1", b"0]", b"0}", b"0,",
+    b"10", b"100", b"01", b'""', b'"a"', b'"a":', b'a"]', b'a"}', b'\\"', b'\\\\', b"] ,", b"",
+]
+
+
+def make_vocab_json(vocab_size: int, seed: int = 0):
+    """``make_vocab_geometric`` with its first random strings replaced by a fixed
+    list of structural JSON tokens (brackets, quotes, literals and their
+    combinations); ids 0..255 stay the single bytes."""
+    base_bytes, base_off = make_vocab_geometric(vocab_size, seed=seed)
+    n = min(len(_JSON_TOKENS), vocab_size - 256)
+    toks = [bytes(base_bytes[base_off[v]:base_off[v + 1]]) for v in range(256 + n, vocab_size)]
+    return vocab_from_strings([bytes([c]) for c in range(256)] + _JSON_TOKENS[:n] + toks)

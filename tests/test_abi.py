@@ -69,7 +69,29 @@ def test_null_and_range_errors(lib):
     assert lib.cstr_step(None, 1, None, None, 0, 0, None, None, None, None, None, 1, None, None) == -1
     assert lib.cstr_step_status(None, None, None, None) == -1
     assert lib.cstr_table_info(None, None, None, None, None) == -1
+    # push-down entry points: validation that precedes every CUDA call
+    z = np.zeros(2, dtype=np.int32)
+    zp = z.ctypes.data_as(ctypes.c_void_p)
+    assert lib.cstr_load_pda(None, None, None, None, None, None, None, 0, None, 1, 0, 0,
+                             ctypes.byref(out)) == -1
+    assert lib.cstr_load_pda(zp, zp, zp, zp, zp, zp, zp, 0, ap, 0, 0, 0, ctypes.byref(out)) == -2
+    assert lib.cstr_load_pda(zp, zp, zp, zp, zp, zp, zp, 0, ap, 1, 255, 0, ctypes.byref(out)) == -10
+    assert lib.cstr_load_pda(zp, zp, zp, zp, zp, zp, zp, 0, ap, 2, 1, 2, ctypes.byref(out)) == -2
+    bad_byte = np.array([300], dtype=np.int32)
+    assert lib.cstr_load_pda(zp, bad_byte.ctypes.data_as(ctypes.c_void_p), zp, zp, zp, zp, zp, 1,
+                             ap, 2, 1, 0, ctypes.byref(out)) == -10
+    assert b"no epsilon input" in lib.cstr_last_error()
+    assert lib.cstr_build_pda_table(None, None, -1, None, ctypes.byref(out)) == -1
+    assert lib.cstr_pda_table_info(None, None, None, None, None, None) == -1
+    assert lib.cstr_pda_table_download(None, 0, 0, None, None, None) == -1
+    assert lib.cstr_pda_workspace_create(None, 4, ctypes.byref(out)) == -1
+    assert lib.cstr_pda_step(None, None, 0, 0, None, None, None, None, 4, None, None, None, 1,
+                             None, None) == -1
+    assert lib.cstr_pda_step_status(None, None, None, None, None) == -1
     # free functions accept NULL
+    lib.cstr_free_pda(None)
+    lib.cstr_free_pda_table(None)
+    lib.cstr_free_pda_workspace(None)
     lib.cstr_free_dfa(None)
     lib.cstr_free_vocab(None)
     lib.cstr_free_table(None)

@@ -1,0 +1,257 @@
+"""GPU parity of the push-down path (Section 3, Algorithm 3) with the oracle:
+the token-level PDA's per-situation masks and whole decoding loops, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_common import DEV, bits_equal, from_dev_logits, to_dev_logits
+from oracle import pda as op
+from paper_2407_08103_b200 import cstr
+from synth import (anbn_pda, dyck_pda, gumbel_noise, json_pda, make_vocab_json, normal_logits,
+                   stackless_pda, vocab_from_strings)
+from synth.configs import config_dfas, config_vocab
+
+pytestmark = pytest.mark.gpu
+THREADS = 16
+
+
+def load_pda(P):
+    return cstr.cstr_load_pda(P.src, P.inp, P.tgt, P.pop_off, P.pops, P.push_off, P.pushes,
+                              P.accept, P.n_symbols, P.start)
+
+
+def build(P, vb, vo, eos_id=-1):
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    table = cstr.cstr_build_pda_table(load_pda(P), vocab, eos_id)
+    torch.cuda.synchronize()
+    return table
+
+
+def check_table(table, P, vb, vo, eos_id=-1, states=None, deeper=3, seed=0):
+    """mask(q, X) is the allowed set of the one-symbol stack [X] (edges that pop at
+    most that symbol); with deeper stacks ending in X the allowed set grows only by
+    tokens flagged in deep(q, X)."""
+    info = cstr.cstr_pda_table_info(table)
+    V = vo.size - 1
+    assert info == dict(n_states=P.n_states, n_symbols=P.n_symbols, vocab_size=V,
+                        mask_words=(V + 31) // 32, start_state=P.start)
+    states = range(P.n_states) if states is None else states
+    rng = np.random.default_rng(seed)
+    qs, tops, stacks = [], [], []
+    for q in states:
+        for top in range(-1, P.n_symbols):
+            qs.append(q)
+            tops.append(top)
+            stacks.append([] if top < 0 else [top])
+    want = op.allowed(P, vb, vo, qs, stacks, eos_id=eos_id, threads=THREADS)
+    got = [cstr.cstr_pda_table_download(table, q, t) for q, t in zip(qs, tops)]
+    for i in range(len(qs)):
+        assert np.array_equal(got[i][0], want[i]), "mask of (state %d, top %d)" % (qs[i], tops[i])
+        assert not (got[i][0] & got[i][1]).any()
+        if tops[i] < 0:
+            assert not got[i][1].any()          # nothing lies below an empty stack
+    n_deep = 0
+    for _ in range(deeper if P.n_symbols else 0):
+        below = [list(rng.integers(0, P.n_symbols, size=int(rng.integers(1, 4)))) if t >= 0 else []
+                 for t in tops]
+        full = op.allowed(P, vb, vo, qs, [b + s for b, s in zip(below, stacks)], eos_id=eos_id,
+                          threads=THREADS)
+        for i in range(len(qs)):
+            assert not (want[i] & ~full[i]).any()
+            extra = full[i] & ~want[i]
+            assert not (extra & ~got[i][1]).any(), "token allowed by a deeper stack is not flagged"
+            n_deep += int(extra.any())
+    return n_deep
+
+
+def run_both(P, table, ws, vb, vo, logits, states, stacks, depth, noise=None, eos_id=-1,
+             in_place=False):
+    B = logits.shape[0]
+    V = vo.size - 1
+    d_logits = to_dev_logits(logits)
+    d_noise = None if noise is None else torch.from_numpy(noise).to(DEV)
+    d_states = torch.from_numpy(np.asarray(states, dtype=np.int32)).to(DEV)
+    d_stacks = torch.from_numpy(np.ascontiguousarray(stacks, dtype=np.int32)).to(DEV)
+    d_depth = torch.from_numpy(np.asarray(depth, dtype=np.int32)).to(DEV)
+    d_tokens = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+    d_acc = torch.full((B,), 9, dtype=torch.uint8, device=DEV)
+    d_out = d_logits if in_place else torch.full_like(d_logits, 123.0)
+    cstr.cstr_pda_step(table, d_logits, d_states, d_stacks, d_depth, d_tokens, d_out, ws,
+                       noise=d_noise, accept_out=d_acc)
+    torch.cuda.synchronize()
+    counters = cstr.cstr_pda_step_status(ws)
+    ref = op.step(P, vb, vo, logits, states, stacks, depth, noise=noise, eos_id=eos_id,
+                  vocab_size=V, threads=THREADS)
+    assert np.array_equal(d_tokens.cpu().numpy(), ref["tokens"])
+    assert np.array_equal(d_states.cpu().numpy(), ref["states"])
+    assert np.array_equal(d_depth.cpu().numpy(), ref["depth"])
+    g_stacks = d_stacks.cpu().numpy()
+    for r in range(B):
+        n = ref["depth"][r]
+        if 0 <= n <= g_stacks.shape[1]:
+            assert np.array_equal(g_stacks[r, :n], ref["stacks"][r, :n]), "stack of row %d" % r
+    got = from_dev_logits(d_out)
+    assert bits_equal(got[:, :V], ref["masked"][:, :V])
+    if not in_place and got.shape[1] > V:
+        pad = from_dev_logits(torch.full_like(d_logits, 123.0))[:, V:]
+        assert bits_equal(got[:, V:], pad)
+    assert np.array_equal(d_acc.cpu().numpy(), ref["accept"])
+    assert counters == (ref["bad_state_rows"], ref["empty_mask_rows"], ref["overflow_rows"])
+    ref["stacks_full"] = g_stacks
+    return ref
+
+
+# ------------------------------------------------------------------- tables
+
+def test_table_anbn_figure5_vocabulary():
+    P = anbn_pda()
+    vb, vo = vocab_from_strings([b"a", b"b", b"bb", b"aaab", b"", b"abb", b"bbb", b"ab"])
+    table = build(P, vb, vo)
+    assert check_table(table, P, vb, vo) > 0
+    st = {n: i for i, n in enumerate(P.state_names)}
+    A = P.symbol_names.index("A")
+    mask, deep = cstr.cstr_pda_table_download(table, st["bs"], A)
+    assert mask[0] == 0b00000010 and deep[0] == 0b01000100     # b | bb and bbb look deeper
+
+
+def test_table_dyck_and_eos():
+    P = dyck_pda((b"()", b"[]", b"{}", b"<>"), fillers=b"xy ")
+    vb, vo = make_vocab_json(1500, seed=3)
+    table = build(P, vb, vo, eos_id=77)
+    check_table(table, P, vb, vo, eos_id=77)
+
+
+def test_table_json_small_vocab_all_situations():
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(2051, seed=1)        # W = 65 words, ragged last word
+    table = build(P, vb, vo)
+    assert check_table(table, P, vb, vo) > 5
+
+
+def test_table_json_32k_sampled_situations():
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(32000, seed=0)
+    table = build(P, vb, vo)
+    st = {n: i for i, n in enumerate(P.state_names)}
+    check_table(table, P, vb, vo, deeper=1,
+                states=[st[n] for n in ("start", "after_value", "num_int", "str", "arr_first",
+                                        "colon", "done")])
+
+
+def test_stackless_pda_matches_the_finite_state_table():
+    dfa = config_dfas("api_1k")[0]
+    vb, vo = config_vocab("api_1k")
+    P = stackless_pda(*dfa)
+    table = build(P, vb, vo)
+    check_table(table, P, vb, vo)
+
+
+# -------------------------------------------------------------------- steps
+
+@pytest.mark.parametrize("dtype,gumbel,vocab_size,pad", [
+    ("f32", False, 2051, 0), ("bf16", False, 4096, 8), ("f32", True, 3000, 4),
+])
+def test_decode_loop_json(dtype, gumbel, vocab_size, pad):
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(vocab_size, seed=2)
+    V = vo.size - 1
+    toks = [bytes(vb[vo[v]:vo[v + 1]]) for v in range(V)]
+    table = build(P, vb, vo)
+    B, cap, steps = 48, 5, 40
+    ws = cstr.cstr_pda_workspace_create(table, B)
+    states = np.full(B, P.start, dtype=np.int32)
+    stacks = np.zeros((B, cap), dtype=np.int32)
+    depth = np.zeros(B, dtype=np.int32)
+    sigma = 2.0 if dtype == "bf16" else 1.0
+    seen_depth, overflow, deep_rows = 0, 0, 0
+    for t in range(steps):
+        logits = normal_logits(31, t, range(B), V, ld=V + pad, sigma=sigma, dtype="f32")
+        # most rows favour structure over string bodies, some dig for the overflow path
+        for name, bonus in ((b"[", 5.0), (b"[[", 5.0), (b"]]", 6.0), (b"]]]", 6.0), (b"]", 4.0),
+                            (b'"', 4.0), (b"}", 4.0), (b"{", 3.0), (b"1]", 5.0), (b", ", 4.0),
+                            (b"1", 4.0), (b'":', 5.0)):
+            logits[: B - 8, toks.index(name)] += np.float32(bonus)
+        for name in (b"[", b"[[", b"[{"):
+            logits[B - 8:, toks.index(name)] += np.float32(7.0)
+        if dtype == "bf16":
+            from synth import f32_to_bf16_bits
+            logits = f32_to_bf16_bits(logits)
+        noise = gumbel_noise(1, t, range(B), V, ld=V + pad) if gumbel else None
+        ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth, noise=noise)
+        deep_rows += int(((depth >= 2) & (states >= 0)).sum())
+        states, depth = ref["states"], ref["depth"]
+        stacks = ref["stacks_full"]
+        seen_depth = max(seen_depth, int(depth.max()))
+        overflow += ref["overflow_rows"]
+        if t == 20:                                 # restart the finished rows
+            done = states < 0
+            states = np.where(done, P.start, states).astype(np.int32)
+            depth = np.where(done, 0, depth).astype(np.int32)
+    assert seen_depth >= 4 and overflow > 0 and deep_rows > 50
+
+
+def test_decode_loop_anbn_deep_pops():
+    # every b-run token reaches below the top of the stack
+    P = anbn_pda()
+    vb, vo = vocab_from_strings([b"a", b"b", b"bb", b"aaab", b"bbbb", b"aa", b"ab", b"<e>", b"bbb"])
+    V = vo.size - 1
+    table = build(P, vb, vo, eos_id=7)
+    B, cap = 64, 12
+    ws = cstr.cstr_pda_workspace_create(table, B)
+    states = np.full(B, P.start, dtype=np.int32)
+    stacks = np.zeros((B, cap), dtype=np.int32)
+    depth = np.zeros(B, dtype=np.int32)
+    finished = 0
+    for t in range(14):
+        logits = normal_logits(41, t, range(B), V, ld=12)
+        if t < 3:
+            logits[:, [0, 5]] += np.float32(3.0)        # grow first
+        ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth, eos_id=7,
+                       in_place=(t % 2 == 1))
+        finished += int(((ref["tokens"] == 7)).sum())
+        states, depth, stacks = ref["states"], ref["depth"], ref["stacks_full"]
+    assert finished > 10                                 # rows reached "done" and took EOS
+
+
+def test_inactive_rows_bad_stacks_and_overflow():
+    P = anbn_pda()
+    vb, vo = vocab_from_strings([b"a", b"b", b"bb", b"aaab", b"<eos>"])
+    st = {n: i for i, n in enumerate(P.state_names)}
+    Z, A = P.symbol_names.index("Z"), P.symbol_names.index("A")
+    table = build(P, vb, vo, eos_id=4)
+    ws = cstr.cstr_pda_workspace_create(table, 16)
+    logits = np.array([[0.0, 1.0, 2.0, 3.0, 0.5]] * 9, dtype=np.float32)
+    states = np.array([st["start"], st["as"], st["bs"], -1, 9, st["as"], st["done"], st["as"],
+                       st["bs"]], np.int32)
+    stacks = np.array([[0, 0, 0], [Z, A, 0], [Z, A, 0], [0, 0, 0], [0, 0, 0], [Z, 7, 0],
+                       [0, 0, 0], [Z, A, A], [-1, A, 0]], np.int32)
+    depth = np.array([0, 2, 2, 0, 0, 2, 0, 4, 2], np.int32)
+    ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth, eos_id=4)
+    assert list(ref["tokens"]) == [3, 3, 2, -1, -1, -1, 4, -1, -1]
+    assert (ref["bad_state_rows"], ref["empty_mask_rows"], ref["overflow_rows"]) == (4, 0, 1)
+
+
+def test_load_pda_rejects_what_it_cannot_run():
+    P = anbn_pda()
+
+    def load(**kw):
+        d = dict(src=P.src, inp=P.inp, tgt=P.tgt, pop_off=P.pop_off, pops=P.pops,
+                 push_off=P.push_off, pushes=P.pushes, accept=P.accept, n_symbols=P.n_symbols,
+                 start=P.start)
+        d.update(kw)
+        return cstr.cstr_load_pda(d["src"], d["inp"], d["tgt"], d["pop_off"], d["pops"],
+                                  d["push_off"], d["pushes"], d["accept"], d["n_symbols"],
+                                  d["start"])
+
+    load()
+    with pytest.raises(cstr.CstrError) as e:
+        load(inp=np.where(np.arange(P.n_edges) == 1, -1, P.inp))     # an epsilon edge
+    assert e.value.code == -10
+    with pytest.raises(cstr.CstrError) as e:                          # two edges, same situation
+        load(src=np.append(P.src, P.src[0]), inp=np.append(P.inp, P.inp[0]),
+             tgt=np.append(P.tgt, P.tgt[0]), pop_off=np.append(P.pop_off, P.pop_off[-1]),
+             push_off=np.append(P.push_off, P.push_off[-1]))
+    assert e.value.code == -10 and "deterministic" in str(e.value)
+    with pytest.raises(cstr.CstrError) as e:                          # a two-symbol pop
+        load(pop_off=np.append(P.pop_off[:-1], P.pop_off[-1] + 1), pops=np.append(P.pops, 0))
+    assert e.value.code == -10
