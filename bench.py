@@ -339,6 +339,60 @@ def time_wildcard_build(torch, cstr, vocab, vb, vo, stream, peak):
             "frac_of_hbm_peak": S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9 / peak}
 
 
+def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=512, steps=48):
+    """Push-down step (Algorithm 3) on a nested-JSON PDA over a 256,000-token
+    vocabulary with structural multi-bracket tokens, batch 512, fp32, greedy:
+    table build (allocation + kernel) and the two-kernel step (situation
+    lookup; fused penalise / select / edge traversal), events around each call;
+    finished rows are restarted."""
+    from synth import json_pda, make_vocab_json
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(V, seed=0)
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    h = cstr.cstr_load_pda(P.src, P.inp, P.tgt, P.pop_off, P.pops, P.push_off, P.pushes, P.accept,
+                           P.n_symbols, P.start)
+    build_ms = []
+    table = None
+    for _ in range(3):
+        del table
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        table = cstr.cstr_build_pda_table(h, vocab, -1, stream)
+        torch.cuda.synchronize()
+        build_ms.append((time.perf_counter() - t0) * 1e3)
+    n_cfg = P.n_states * (P.n_symbols + 1)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(17)
+    pool = [torch.randn((B, V), generator=gen, device=dev) for _ in range(3)]
+    out = [torch.empty((B, V), device=dev) for _ in range(2)]
+    dec = PushdownDecoder(table, B, stack_cap=64, device=dev)
+    pairs, depth_sum, depth_max = [], 0.0, 0
+    for i in range(steps + 4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        dec.step(pool[i % 3], masked_out=out[i & 1], stream=stream)
+        e1.record(stream)
+        dec.restart_finished()
+        if i >= 4:
+            pairs.append((e0, e1))
+            depth_sum += float(dec.depths.float().mean().item())
+            depth_max = max(depth_max, int(dec.depths.max().item()))
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    bad, empty, overflow = dec.status()
+    gbs = B * V * BYTES_PER_LOGIT_F32_GREEDY / (ms * 1e-3) / 1e9
+    return {"workload": "nested JSON PDA (%d states, %d stack symbols, %d situations) x vocab %d, "
+                        "batch %d, fp32 greedy" % (P.n_states, P.n_symbols, n_cfg, V, B),
+            "table_build_ms": float(min(build_ms)),
+            "table_transitions_per_s": n_cfg * V / (min(build_ms) * 1e-3),
+            "step_ms": ms, "logits_per_s": B * V / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                         "frac": gbs / peak, "traffic": None,
+                         "note": "two kernels per step (situation lookup, fused step); 8.125 algorithmic bytes per logit"},
+            "mean_stack_depth": depth_sum / max(len(pairs), 1), "max_stack_depth": depth_max,
+            "status_rows": {"bad": bad, "empty_mask": empty, "overflow": overflow}}
+
+
 def time_small_batches(torch, cstr, table, V, dev, stream, batches=(1, 8, 64)):
     """Step latency for small batches at the full vocabulary (fp32, greedy): 64
     steps captured in one CUDA graph, logits rotating through a pool larger than
@@ -439,7 +493,7 @@ def main():
 
     from paper_2407_08103_b200 import build as libbuild
     from paper_2407_08103_b200 import cstr
-    from paper_2407_08103_b200.decode import ConstrainedDecoder
+    from paper_2407_08103_b200.decode import ConstrainedDecoder, PushdownDecoder
     from synth import normal_logits
     libbuild.build_library()
 
@@ -617,11 +671,13 @@ def main():
         wildcard = time_wildcard_build(torch, cstr, vocab, vb, vo, stream, measured_hbm_peak()[0])
 
     # ---- the other four workloads (single-GPU runs only) --------------------
-    others = None
+    others, pushdown = None, None
     if rank == 0 and world == 1 and not args.skip_other_workloads and args.case == "full":
         del dev_pool, staging, out_bufs
         torch.cuda.empty_cache()
         peak_now, _ = measured_hbm_peak()
+        pushdown = time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak_now)
+        torch.cuda.empty_cache()
         others = []
         for name in ("api_1k", "json_32k", "schema40_128k", "random10k_256k"):
             others.append(time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream,
@@ -694,6 +750,7 @@ def main():
         "dfa_load_ms": dfa_load_ms,
         "wildcard_table_build": wildcard,
         "speculative_verify": spec,
+        "pushdown_step": pushdown,
         "small_batch_step_latency": small,
         "other_workloads": others,
         "status_rows": {"bad_state": bad, "empty_mask": empty},

@@ -353,7 +353,7 @@ void cstr_free_pda_workspace(cstr_pda_workspace_t *ws);
  * inactive: token -1, state -1, all -infinity.  If the traversed edge would
  * leave more than stack_cap symbols the token is still emitted and the row
  * finishes (state -1).  Whenever the new state is -1 the row's stack and depth
- * are left as they were.  Enqueues three kernels on cuda_stream; no
+ * are left as they were.  Enqueues two kernels on cuda_stream; no
  * allocation, no host synchronisation.
  */
 int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dtype, int64_t ld,

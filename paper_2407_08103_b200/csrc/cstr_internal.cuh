@@ -115,6 +115,25 @@ struct cstr_workspace {
 // edge[j] = { target, push0 | push1 << 8 | push2 << 16 | npush << 24 | pop << 28 }.
 #define CSTR_PDA_NONE 0xffffffffu
 #define CSTR_PDA_NEEDCTX 0xfffffffeu
+struct cstr_pda_view {
+    const uint32_t *act;
+    const int2 *edge;
+    int NT;
+    int n_symbols;
+};
+
+// What the step kernel needs to traverse an edge of the token-level PDA.
+struct cstr_pda_advance {
+    cstr_pda_view P;
+    const uint8_t *accept;         // DEVICE [n_states]
+    const uint8_t *vbytes;         // DEVICE vocabulary bytes
+    const uint32_t *voff;          // DEVICE [V + 1]
+    int32_t n_states, eos_id, cap;
+    int32_t *states, *stacks, *depths;   // DEVICE [batch], [batch][cap], [batch]
+    uint8_t *accept_out;           // DEVICE [batch] or null
+    unsigned long long *counters;  // DEVICE [3]: bad rows, rows without a token, overflows
+};
+
 struct cstr_pda {
     int device;
     int32_t n_states, n_symbols, start, n_edges;
@@ -174,13 +193,14 @@ struct cstr_step_args {
     unsigned int *ticket;          // DEVICE [batch]
     unsigned long long *counters;  // DEVICE [2]
     int device;
-    // Row-mask mode (push-down step): when row_mask is non-null the kernel takes
-    // row r's allowed-token words from row_mask[r] (null = inactive row), needs
-    // no tables, and only emits masked logits and tokens - states, accept flags
-    // and counters are the caller's business.
-    const uint32_t *const *row_mask;   // DEVICE [batch]
-    int32_t V;                         // vocabulary size  (row-mask mode only)
-    int64_t ldw;                       // words readable behind every row pointer
+    // Push-down mode: when pda is non-null the kernel takes row r's allowed-token
+    // words from row_mask[r] (null = inactive row), needs no tables, and the last
+    // CTA of a row traverses the selected token's edge of the token-level PDA
+    // (state, stack, depth, accept flag, counters: see cstr_pda_advance).
+    const struct cstr_pda_advance *pda;   // HOST
+    const uint32_t *const *row_mask;      // DEVICE [batch]
+    int32_t V;                            // vocabulary size  (push-down mode only)
+    int64_t ldw;                          // words readable behind every row pointer
 };
 int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream);
 int cstr_launch_accept(const int32_t *draft, const int32_t *tgt_tok, const int32_t *tgt_state,

@@ -11,81 +11,25 @@
 // situation's mask row as is, or - if that situation has flagged tokens - a
 // private copy in which the flagged tokens have been walked against the row's
 // real stack.  The fused step kernel then streams the logits exactly as in the
-// finite-state case, and a small kernel traverses the selected token's edge:
-// it walks the token's bytes from (q, s), which yields the edge's target, pops
-// and pushes without storing variable-length stack edits per table entry.
+// finite-state case, and the last CTA of each row traverses the selected
+// token's edge: it walks the token's bytes from (q, s), which yields the edge's
+// target, pops and pushes without storing variable-length stack edits per
+// table entry.
 #include <string.h>
 
 #include <new>
 #include <vector>
 
 #include "cstr_internal.cuh"
+#include "cstr_pda_walk.cuh"
 
 namespace {
 
-constexpr int kLocMax = 256;   // symbols one token may leave on top of the stack it found
-
-struct PdaView {
-    const uint32_t *act;
-    const int2 *edge;
-    int NT;
-    int n_symbols;
-};
-
-enum { WALK_DEAD = 0, WALK_OK = 1, WALK_DEEP = 2 };
-
-// Chain the byte edges of bytes[0..len) from state q.  The stack found is
-// ctx[0..cd) when ctx is non-null (all of it known), else the single symbol
-// known_top (cd = 1) or nothing (cd = 0) with `unknown_below` saying whether
-// unseen symbols lie underneath.  loc receives what the chain leaves on top.
-// WALK_DEEP: the chain reached a byte whose edge depends on an unseen symbol.
-__device__ __forceinline__ int pda_walk(const PdaView &P, int q, const int32_t *ctx, int known_top,
-                                        int cd, bool unknown_below, const uint8_t *bytes, int len,
-                                        uint8_t *loc, int &q_out, int &cd_out, int &nloc_out)
-{
-    int nloc = 0;
-    if (len <= 0)
-        return WALK_DEAD;                           // an empty token never has an edge
-    for (int k = 0; k < len; ++k) {
-        int t;
-        if (nloc > 0) {
-            t = loc[nloc - 1];
-        } else if (cd > 0) {
-            t = ctx ? ctx[cd - 1] : known_top;
-            if ((unsigned)t >= (unsigned)P.n_symbols)
-                return WALK_DEAD;
-        } else {
-            t = unknown_below ? P.n_symbols + 1 : P.n_symbols;
-        }
-        const uint32_t a = __ldg(P.act + ((long long)q * P.NT + t) * 256 + bytes[k]);
-        if (a == CSTR_PDA_NONE)
-            return WALK_DEAD;
-        if (a == CSTR_PDA_NEEDCTX)
-            return WALK_DEEP;
-        const int2 e = __ldg(P.edge + a);
-        const unsigned meta = (unsigned)e.y;
-        if (meta >> 28) {                           // pops the symbol it looked at
-            if (nloc > 0)
-                --nloc;
-            else
-                --cd;
-        }
-        const int npush = (meta >> 24) & 7;
-        if (nloc + npush > kLocMax)
-            return WALK_DEAD;                       // excluded by the build's length check
-        for (int i = 0; i < npush; ++i)
-            loc[nloc++] = (uint8_t)(meta >> (8 * i));
-        q = e.x;
-    }
-    q_out = q;
-    cd_out = cd;
-    nloc_out = nloc;
-    return WALK_OK;
-}
+using namespace cstr_pda_dev;
 
 // One warp per (situation, 32-token word): lane = token.
 __global__ void __launch_bounds__(256)
-pda_build_kernel(PdaView P, const uint8_t *__restrict__ accept, const uint8_t *__restrict__ vbytes,
+pda_build_kernel(cstr_pda_view P, const uint8_t *__restrict__ accept, const uint8_t *__restrict__ vbytes,
                  const uint32_t *__restrict__ voff, int V, int W, long long ldw, int eos_id,
                  uint32_t *__restrict__ mask, uint32_t *__restrict__ deep,
                  uint32_t *__restrict__ ndeep)
@@ -121,45 +65,46 @@ pda_build_kernel(PdaView P, const uint8_t *__restrict__ accept, const uint8_t *_
     }
 }
 
-struct PdaStepParams {
-    PdaView P;
-    const uint8_t *accept;
+// What the prepare kernel reads: the rows' situations and the table.
+struct PdaPrepParams {
+    cstr_pda_view P;
     const uint8_t *vbytes;
     const uint32_t *voff;
     const uint32_t *mask, *deep, *ndeep;
     long long ldw;
-    int n_states, V, eos_id;
-    int32_t *states, *stacks, *depths;
-    int cap, batch;
-    const int32_t *tokens;
-    uint8_t *accept_out;
+    int n_states;
+    const int32_t *states, *stacks, *depths;
+    int cap;
     const uint32_t **row_mask;
     uint32_t *row_buf;
-    unsigned long long *counters;   // [0] bad, [1] empty, [2] overflow
 };
 
-// One warp per row: find the row's situation and point the step at its mask row,
-// or at a private copy in which the tokens that depend on deeper stack symbols
-// have been decided against the row's stack.
-__global__ void __launch_bounds__(128)
-pda_prepare_kernel(const __grid_constant__ PdaStepParams p)
+// Find each row's situation and point the step at its mask row, or - when the
+// situation has tokens that depend on deeper stack symbols - at a private copy
+// in which those tokens have been walked against the row's real stack.
+// blockIdx.x = row, blockIdx.y = slice of kPrepWords mask words; every block of
+// a row re-derives the (cheap) row checks.  Spreading a row over several blocks
+// matters: each flagged token costs a chain of dependent loads, and a row's
+// tokens are walked by different threads in parallel.
+constexpr int kPrepThreads = 256;
+constexpr int kPrepWords = 1024;
+
+__global__ void __launch_bounds__(kPrepThreads)
+pda_prepare_kernel(const __grid_constant__ PdaPrepParams p)
 {
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (r >= p.batch)
-        return;
+    const int r = blockIdx.x;
+    const int slice = blockIdx.y;
     const int q = p.states[r];
     const int d = p.depths[r];
     const int32_t *s = p.stacks + (long long)r * p.cap;
-    bool ok = q >= 0 && q < p.n_states && d >= 0 && d <= p.cap;
-    if (ok) {
-        bool bad = false;
-        for (int i = lane; i < d; i += 32)
+    const bool shape_ok = q >= 0 && q < p.n_states && d >= 0 && d <= p.cap;   // block-uniform
+    bool bad = false;
+    if (shape_ok)
+        for (int i = threadIdx.x; i < d; i += kPrepThreads)
             bad |= (unsigned)s[i] >= (unsigned)p.P.n_symbols;
-        ok = !__any_sync(0xffffffffu, bad);
-    }
+    const bool ok = shape_ok && !__syncthreads_or(bad);
     if (!ok) {
-        if (lane == 0)
+        if (slice == 0 && threadIdx.x == 0)
             p.row_mask[r] = nullptr;
         return;
     }
@@ -167,15 +112,17 @@ pda_prepare_kernel(const __grid_constant__ PdaStepParams p)
     const long long cfg = (long long)q * (p.P.n_symbols + 1) + top;
     const uint32_t *mrow = p.mask + cfg * p.ldw;
     if (p.ndeep[cfg] == 0) {
-        if (lane == 0)
+        if (slice == 0 && threadIdx.x == 0)
             p.row_mask[r] = mrow;
         return;
     }
     const uint32_t *drow = p.deep + cfg * p.ldw;
     uint32_t *out = p.row_buf + (long long)r * p.ldw;
-    for (long long w = lane; w < p.ldw; w += 32) {
-        uint32_t m = mrow[w];
-        uint32_t dw = drow[w];
+    const long long w_end = min(p.ldw, (long long)(slice + 1) * kPrepWords);
+    for (long long w = (long long)slice * kPrepWords + threadIdx.x; w < w_end;
+         w += kPrepThreads) {
+        uint32_t m = __ldg(mrow + w);
+        uint32_t dw = __ldg(drow + w);
         while (dw) {
             const int b = __ffs((int)dw) - 1;
             dw &= dw - 1;
@@ -189,46 +136,8 @@ pda_prepare_kernel(const __grid_constant__ PdaStepParams p)
         }
         out[w] = m;
     }
-    if (lane == 0)
+    if (slice == 0 && threadIdx.x == 0)
         p.row_mask[r] = out;
-}
-
-// One thread per row: traverse the edge of the selected token.
-__global__ void __launch_bounds__(128)
-pda_advance_kernel(const __grid_constant__ PdaStepParams p)
-{
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= p.batch)
-        return;
-    const int q = p.states[r];
-    const int tok = p.tokens[r];
-    int q2 = CSTR_DEAD;
-    if (p.row_mask[r] == nullptr) {
-        if (q != -1)
-            atomicAdd(p.counters + 0, 1ull);
-    } else if (tok < 0) {
-        atomicAdd(p.counters + 1, 1ull);
-    } else if (tok != p.eos_id) {
-        const int d = p.depths[r];
-        int32_t *s = p.stacks + (long long)r * p.cap;
-        uint8_t loc[kLocMax];
-        int qn, cd, nloc;
-        const uint32_t b0 = p.voff[tok], b1 = p.voff[tok + 1];
-        if (pda_walk(p.P, q, s, 0, d, false, p.vbytes + b0, (int)(b1 - b0), loc, qn, cd, nloc) ==
-            WALK_OK) {
-            if (cd + nloc > p.cap) {
-                atomicAdd(p.counters + 2, 1ull);
-            } else {
-                for (int i = 0; i < nloc; ++i)
-                    s[cd + i] = loc[i];
-                p.depths[r] = cd + nloc;
-                q2 = qn;
-            }
-        }
-    }
-    p.states[r] = q2;
-    if (p.accept_out)
-        p.accept_out[r] = (q2 >= 0) ? (uint8_t)(p.accept[q2] != 0) : (uint8_t)0;
 }
 
 int check_device(int handle_device, const char *what)
@@ -450,7 +359,7 @@ extern "C" int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *v
     if (e == cudaSuccess)
         e = cudaMemsetAsync(t->ndeep, 0, (size_t)n_cfg * 4, stream);
     if (e == cudaSuccess) {
-        PdaView P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
+        cstr_pda_view P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
         const int warps = 8;
         dim3 grid((unsigned)((t->W + warps - 1) / warps), (unsigned)n_cfg);
         pda_build_kernel<<<grid, warps * 32, 0, stream>>>(P, pda->accept, vocab->bytes, vocab->off,
@@ -600,13 +509,12 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const cstr_pda *pda = table->pda;
 
-    PdaStepParams p;
+    PdaPrepParams p;
     memset(&p, 0, sizeof p);
     p.P.act = pda->act;
     p.P.edge = pda->edge;
     p.P.NT = pda->NT;
     p.P.n_symbols = pda->n_symbols;
-    p.accept = pda->accept;
     p.vbytes = table->vocab->bytes;
     p.voff = table->vocab->off;
     p.mask = table->mask;
@@ -614,20 +522,17 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     p.ndeep = table->ndeep;
     p.ldw = table->ldw;
     p.n_states = pda->n_states;
-    p.V = table->V;
-    p.eos_id = table->eos_id;
     p.states = states;
     p.stacks = stacks;
     p.depths = depths;
     p.cap = stack_cap;
-    p.batch = batch;
-    p.tokens = tokens_out;
-    p.accept_out = accept_out;
     p.row_mask = ws->row_mask;
     p.row_buf = ws->row_buf;
-    p.counters = ws->counters + 2;
 
-    pda_prepare_kernel<<<(batch + 3) / 4, 128, 0, stream>>>(p);
+    const long long slices = (table->ldw + kPrepWords - 1) / kPrepWords;
+    if (slices > 65535)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_pda_step: vocabulary too large");
+    pda_prepare_kernel<<<dim3((unsigned)batch, (unsigned)slices), kPrepThreads, 0, stream>>>(p);
     CSTR_CUDA_TRY(cudaGetLastError());
 
     cstr_step_args a;
@@ -646,16 +551,25 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     a.ticket = ws->ticket;
     a.counters = ws->counters;
     a.device = ws->device;
+    cstr_pda_advance adv;
+    memset(&adv, 0, sizeof adv);
+    adv.P = p.P;
+    adv.accept = pda->accept;
+    adv.vbytes = p.vbytes;
+    adv.voff = p.voff;
+    adv.n_states = pda->n_states;
+    adv.eos_id = table->eos_id;
+    adv.cap = stack_cap;
+    adv.states = states;
+    adv.stacks = stacks;
+    adv.depths = depths;
+    adv.accept_out = accept_out;
+    adv.counters = ws->counters + 2;
+    a.pda = &adv;
     a.row_mask = ws->row_mask;
     a.V = table->V;
     a.ldw = table->ldw;
-    rc = cstr_launch_step(a, stream);
-    if (rc)
-        return rc;
-
-    pda_advance_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(p);
-    CSTR_CUDA_TRY(cudaGetLastError());
-    return CSTR_OK;
+    return cstr_launch_step(a, stream);
 }
 
 extern "C" int cstr_pda_step_status(cstr_pda_workspace_t *ws, void *cuda_stream, int64_t *bad_rows,

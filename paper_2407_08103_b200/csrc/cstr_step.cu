@@ -18,6 +18,7 @@
 #include <mutex>
 
 #include "cstr_internal.cuh"
+#include "cstr_pda_walk.cuh"
 
 namespace {
 
@@ -45,7 +46,8 @@ struct StepParams {
     unsigned long long *cell;
     unsigned int *ticket;
     unsigned long long *counters;
-    const uint32_t *const *row_mask;   // non-null: per-row mask pointers instead of tables
+    const uint32_t *const *row_mask;   // push-down kernels: per-row mask pointers, no tables
+    cstr_pda_advance pda;              // push-down kernels: what the edge traversal needs
     long long ld;
     int V;
     int n_tables;
@@ -97,12 +99,13 @@ struct RowCtx {
     const uint32_t *mrow;
 };
 
+template <bool PDA>
 __device__ __forceinline__ RowCtx row_context(const StepParams &p)
 {
     RowCtx c;
     c.r = blockIdx.x / p.nchunks;
     c.chunk = blockIdx.x - c.r * p.nchunks;
-    if (p.row_mask) {                               // the caller resolved the rows' masks
+    if (PDA) {                                      // the rows' masks were resolved beforehand
         c.t = 0;
         c.q = 0;
         c.mrow = p.row_mask[c.r];
@@ -120,6 +123,7 @@ __device__ __forceinline__ RowCtx row_context(const StepParams &p)
 }
 
 // CTA-level reduction, cross-CTA fold, and the last arriver's finalisation.
+template <bool PDA>
 __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c, Best b)
 {
     __shared__ float s_v[32];
@@ -150,9 +154,11 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     __threadfence();
     const unsigned long long key = atomicExch(p.cell + c.r, 0ull);
     p.ticket[c.r] = 0u;
-    if (p.row_mask) {                               // the caller advances its own automaton
-        p.tokens[c.r] = (c.active && key != 0ull)
-                            ? (int)(0xffffffffu - (unsigned)(key & 0xffffffffull)) : -1;
+    if (PDA) {                                      // Algorithm 3: traverse the token's edge
+        const int t = (c.active && key != 0ull)
+                          ? (int)(0xffffffffu - (unsigned)(key & 0xffffffffull)) : -1;
+        p.tokens[c.r] = t;
+        cstr_pda_dev::pda_traverse(p.pda, c.r, c.active, t);
         return;
     }
     int tok = -1, q2 = CSTR_DEAD;
@@ -275,7 +281,7 @@ __device__ __forceinline__ void apply_one(const StepParams &p, const RowCtx &c, 
 
 // ---- vector kernel ----------------------------------------------------------
 
-template <bool BF16, bool NOISE>
+template <bool BF16, bool NOISE, bool PDA>
 __global__ void __launch_bounds__(256, 4)
 step_vec_kernel(const __grid_constant__ StepParams p)
 {
@@ -286,7 +292,7 @@ step_vec_kernel(const __grid_constant__ StepParams p)
     constexpr int WPL = WORDS >= 32 ? WORDS / 32 : 1;   // mask words per lane per tile
     constexpr int LANES_PER_WORD = 32 / VEC;
 
-    const RowCtx c = row_context(p);
+    const RowCtx c = row_context<PDA>(p);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const long long row_off = (long long)c.r * p.ld;
     const uint4 *in = (const uint4 *)((const char *)p.logits + row_off * (BF16 ? 2 : 4));
@@ -404,23 +410,23 @@ step_vec_kernel(const __grid_constant__ StepParams p)
         merge(b, tb.v, tb.i);
     }
 
-    finish_row(p, c, b);
+    finish_row<PDA>(p, c, b);
 }
 
 // ---- scalar kernel: any alignment / stride ----------------------------------
 
-template <bool BF16>
+template <bool BF16, bool PDA>
 __global__ void __launch_bounds__(256)
 step_scalar_kernel(const __grid_constant__ StepParams p)
 {
-    const RowCtx c = row_context(p);
+    const RowCtx c = row_context<PDA>(p);
     const long long row_off = (long long)c.r * p.ld;
     const long long begin = (long long)c.chunk * p.tiles_per_cta * p.tile_tokens;
     const int end = (int)min((long long)p.V, begin + (long long)p.tiles_per_cta * p.tile_tokens);
     Best b = {-CUDART_INF_F, -1};
     for (int i = (int)begin + threadIdx.x; i < end; i += blockDim.x)
         apply_one<BF16>(p, c, row_off, i, b);
-    finish_row(p, c, b);
+    finish_row<PDA>(p, c, b);
 }
 
 int g_sm_count[64] = {0};
@@ -444,7 +450,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
 {
     StepParams p;
     memset(&p, 0, sizeof p);
-    for (int i = 0; i < CSTR_MAX_TABLES && !a.row_mask; ++i) {
+    for (int i = 0; i < CSTR_MAX_TABLES && !a.pda; ++i) {
         const cstr_table *t = a.tables[i < a.n_tables ? i : 0];
         p.tab[i].mask = t->mask;
         p.tab[i].next = t->next;
@@ -455,8 +461,10 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         p.tab[i].wide = t->wide;
         p.tab[i].code_shift = t->code_shift;
     }
-    if (a.row_mask)
+    if (a.pda) {
         p.tab[0].ldw = a.ldw;
+        p.pda = *a.pda;
+    }
     p.row_mask = a.row_mask;
     p.row_table = a.row_table;
     p.logits = a.logits;
@@ -470,7 +478,7 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     p.ticket = a.ticket;
     p.counters = a.counters;
     p.ld = a.ld;
-    p.V = a.row_mask ? a.V : a.tables[0]->V;
+    p.V = a.pda ? a.V : a.tables[0]->V;
     p.n_tables = a.n_tables;
 
     const bool bf16 = a.dtype == CSTR_BF16;
@@ -499,24 +507,22 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
                         (a.ld * esz) % 16 == 0 &&
                         (!a.noise || (aligned16(a.noise) && (a.ld * 4) % 16 == 0));
     const unsigned grid = (unsigned)ctas;
-    if (vec_ok) {
-        if (bf16) {
-            if (a.noise)
-                step_vec_kernel<true, true><<<grid, threads, 0, stream>>>(p);
-            else
-                step_vec_kernel<true, false><<<grid, threads, 0, stream>>>(p);
-        } else {
-            if (a.noise)
-                step_vec_kernel<false, true><<<grid, threads, 0, stream>>>(p);
-            else
-                step_vec_kernel<false, false><<<grid, threads, 0, stream>>>(p);
-        }
-    } else {
-        if (bf16)
-            step_scalar_kernel<true><<<grid, threads, 0, stream>>>(p);
-        else
-            step_scalar_kernel<false><<<grid, threads, 0, stream>>>(p);
+    const int variant = (vec_ok ? 4 : 0) | (bf16 ? 2 : 0) | (a.noise ? 1 : 0);
+#define CSTR_LAUNCH_STEP(PDA)                                                              \
+    switch (variant) {                                                                     \
+    case 7: step_vec_kernel<true, true, PDA><<<grid, threads, 0, stream>>>(p); break;      \
+    case 6: step_vec_kernel<true, false, PDA><<<grid, threads, 0, stream>>>(p); break;     \
+    case 5: step_vec_kernel<false, true, PDA><<<grid, threads, 0, stream>>>(p); break;     \
+    case 4: step_vec_kernel<false, false, PDA><<<grid, threads, 0, stream>>>(p); break;    \
+    case 3: case 2: step_scalar_kernel<true, PDA><<<grid, threads, 0, stream>>>(p); break; \
+    default: step_scalar_kernel<false, PDA><<<grid, threads, 0, stream>>>(p); break;       \
     }
+    if (a.pda) {
+        CSTR_LAUNCH_STEP(true)
+    } else {
+        CSTR_LAUNCH_STEP(false)
+    }
+#undef CSTR_LAUNCH_STEP
     CSTR_CUDA_TRY(cudaGetLastError());
     return CSTR_OK;
 }

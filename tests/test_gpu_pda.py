@@ -255,3 +255,38 @@ def test_load_pda_rejects_what_it_cannot_run():
     with pytest.raises(cstr.CstrError) as e:                          # a two-symbol pop
         load(pop_off=np.append(P.pop_off[:-1], P.pop_off[-1] + 1), pops=np.append(P.pops, 0))
     assert e.value.code == -10
+
+
+def test_full_size_json_256k_sampled_rows():
+    # vocabulary 256,000 x batch 512 as bench.py times it; the oracle replays the whole
+    # trajectory of a few rows (each row depends only on its own logits, state and stack)
+    from paper_2407_08103_b200.decode import PushdownDecoder
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(256000, seed=0)
+    V = vo.size - 1
+    toks = {bytes(vb[vo[v]:vo[v + 1]]): v for v in range(V - 1, -1, -1)}
+    table = build(P, vb, vo)
+    B, cap, steps = 512, 64, 10
+    rows = [0, 3, 77, 300, 511]
+    dec = PushdownDecoder(table, B, stack_cap=cap)
+    o_states = np.full(len(rows), P.start, dtype=np.int32)
+    o_stacks = np.zeros((len(rows), cap), dtype=np.int32)
+    o_depth = np.zeros(len(rows), dtype=np.int32)
+    deepest = 0
+    for t in range(steps):
+        logits = normal_logits(51, t, range(B), V)
+        for name, bonus in ((b"[", 6.0), (b"[[", 6.0), (b"]]", 7.0), (b"]]]", 7.0), (b"1]", 6.0),
+                            (b"{", 4.0), (b"}]", 6.0), (b'"', 5.0), (b", ", 5.0), (b"1", 5.0)):
+            logits[:, toks[name]] += np.float32(bonus)
+        tokens, masked = dec.step(to_dev_logits(logits))
+        ref = op.step(P, vb, vo, logits[rows], o_states, o_stacks, o_depth, threads=THREADS)
+        assert np.array_equal(tokens.cpu().numpy()[rows], ref["tokens"]), "step %d tokens" % t
+        assert np.array_equal(dec.states.cpu().numpy()[rows], ref["states"])
+        assert np.array_equal(dec.depths.cpu().numpy()[rows], ref["depth"])
+        g_stacks = dec.stacks.cpu().numpy()[rows]
+        for i in range(len(rows)):
+            assert np.array_equal(g_stacks[i, :ref["depth"][i]], ref["stacks"][i, :ref["depth"][i]])
+        assert bits_equal(from_dev_logits(masked[rows]), ref["masked"])
+        o_states, o_stacks, o_depth = ref["states"], ref["stacks"], ref["depth"]
+        deepest = max(deepest, int(o_depth.max()))
+    assert deepest >= 3 and (o_states >= 0).any()
