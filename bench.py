@@ -58,6 +58,9 @@ def parse_args():
     ap.add_argument("--skip-other-workloads", action="store_true",
                     help="do not time the four other workloads (reported under 'other_workloads')")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--pushdown-only", action="store_true",
+                    help="time only the push-down step leg (batch 128 with --case small) and print "
+                         "its entry; for profiler captures, not a bench line")
     return ap.parse_args()
 
 
@@ -366,8 +369,8 @@ def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=5
     pool = [torch.randn((B, V), generator=gen, device=dev) for _ in range(3)]
     out = [torch.empty((B, V), device=dev) for _ in range(2)]
     dec = PushdownDecoder(table, B, stack_cap=64, device=dev)
-    pairs, depth_sum, depth_max = [], 0.0, 0
-    for i in range(steps + 4):
+    pairs = []
+    for i in range(steps + 4):                      # no host synchronisation inside the loop
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         dec.step(pool[i % 3], masked_out=out[i & 1], stream=stream)
@@ -375,10 +378,14 @@ def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=5
         dec.restart_finished()
         if i >= 4:
             pairs.append((e0, e1))
-            depth_sum += float(dec.depths.float().mean().item())
-            depth_max = max(depth_max, int(dec.depths.max().item()))
     torch.cuda.synchronize()
     ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+    depth_sum, depth_max, probes = 0.0, 0, 8        # stack statistics, outside the timing
+    for i in range(probes):
+        dec.step(pool[i % 3], masked_out=out[i & 1], stream=stream)
+        dec.restart_finished()
+        depth_sum += float(dec.depths.float().mean().item())
+        depth_max = max(depth_max, int(dec.depths.max().item()))
     bad, empty, overflow = dec.status()
     gbs = B * V * BYTES_PER_LOGIT_F32_GREEDY / (ms * 1e-3) / 1e9
     return {"workload": "nested JSON PDA (%d states, %d stack symbols, %d situations) x vocab %d, "
@@ -389,7 +396,7 @@ def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=5
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
                          "frac": gbs / peak, "traffic": None,
                          "note": "two kernels per step (situation lookup, fused step); 8.125 algorithmic bytes per logit"},
-            "mean_stack_depth": depth_sum / max(len(pairs), 1), "max_stack_depth": depth_max,
+            "mean_stack_depth": depth_sum / probes, "max_stack_depth": depth_max,
             "status_rows": {"bad": bad, "empty_mask": empty, "overflow": overflow}}
 
 
@@ -496,6 +503,13 @@ def main():
     from paper_2407_08103_b200.decode import ConstrainedDecoder, PushdownDecoder
     from synth import normal_logits
     libbuild.build_library()
+
+    if args.pushdown_only:
+        entry = time_pushdown(torch, cstr, PushdownDecoder, dev, torch.cuda.current_stream(),
+                              measured_hbm_peak()[0], B=128 if args.case == "small" else 512,
+                              steps=max(args.steps, 1) if args.steps < 100 else 48)
+        print(json.dumps({"pushdown_step": entry}))
+        return
 
     w, dfa, vb, vo = workload_inputs(args.case)
     V = vo.size - 1

@@ -83,9 +83,7 @@ struct PdaPrepParams {
 // situation has tokens that depend on deeper stack symbols - at a private copy
 // in which those tokens have been walked against the row's real stack.
 // blockIdx.x = row, blockIdx.y = slice of kPrepWords mask words; every block of
-// a row re-derives the (cheap) row checks.  Spreading a row over several blocks
-// matters: each flagged token costs a chain of dependent loads, and a row's
-// tokens are walked by different threads in parallel.
+// a row re-derives the (cheap) row checks.
 constexpr int kPrepThreads = 256;
 constexpr int kPrepWords = 1024;
 
@@ -118,23 +116,50 @@ pda_prepare_kernel(const __grid_constant__ PdaPrepParams p)
     }
     const uint32_t *drow = p.deep + cfg * p.ldw;
     uint32_t *out = p.row_buf + (long long)r * p.ldw;
-    const long long w_end = min(p.ldw, (long long)(slice + 1) * kPrepWords);
-    for (long long w = (long long)slice * kPrepWords + threadIdx.x; w < w_end;
-         w += kPrepThreads) {
-        uint32_t m = __ldg(mrow + w);
-        uint32_t dw = __ldg(drow + w);
-        while (dw) {
-            const int b = __ffs((int)dw) - 1;
-            dw &= dw - 1;
-            const int v = (int)w * 32 + b;
+    // Pass 1: copy the words without flagged tokens, queue the others.
+    __shared__ int s_queue[kPrepWords];
+    __shared__ int s_count;
+    if (threadIdx.x == 0)
+        s_count = 0;
+    __syncthreads();
+    constexpr int kPer = kPrepWords / kPrepThreads;
+    const long long w0 = (long long)slice * kPrepWords + threadIdx.x;
+    uint32_t mw[kPer], dw[kPer];
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+        const long long w = w0 + (long long)j * kPrepThreads;
+        mw[j] = w < p.ldw ? __ldg(mrow + w) : 0u;
+        dw[j] = w < p.ldw ? __ldg(drow + w) : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+        const long long w = w0 + (long long)j * kPrepThreads;
+        if (w >= p.ldw)
+            continue;
+        if (dw[j] == 0u)
+            out[w] = mw[j];
+        else
+            s_queue[atomicAdd(&s_count, 1)] = (int)w;
+    }
+    __syncthreads();
+    // Pass 2: one warp per queued word, one lane per flagged token - each walk is
+    // a chain of dependent loads, so the tokens of a word are walked side by side.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = warp; i < s_count; i += kPrepThreads / 32) {
+        const long long w = s_queue[i];
+        const uint32_t flagged = __ldg(drow + w);
+        bool allowed = false;
+        if ((flagged >> lane) & 1u) {
+            const int v = (int)w * 32 + lane;
             uint8_t loc[kLocMax];
             int q2, cd2, nloc2;
             const uint32_t b0 = p.voff[v], b1 = p.voff[v + 1];
-            if (pda_walk(p.P, q, s, 0, d, false, p.vbytes + b0, (int)(b1 - b0), loc, q2, cd2,
-                         nloc2) == WALK_OK)
-                m |= 1u << b;
+            allowed = pda_walk(p.P, q, s, 0, d, false, p.vbytes + b0, (int)(b1 - b0), loc, q2, cd2,
+                               nloc2) == WALK_OK;
         }
-        out[w] = m;
+        const uint32_t extra = __ballot_sync(0xffffffffu, allowed);
+        if (lane == 0)
+            out[w] = __ldg(mrow + w) | extra;
     }
     if (slice == 0 && threadIdx.x == 0)
         p.row_mask[r] = out;
