@@ -11,7 +11,7 @@ from synth.configs import config_dfas, config_vocab
 from synth.regex_frontend import regex_to_dfa
 from helpers import read_records, split_tokens
 
-RECORDS = [r for r in read_records("paper_examples.txt") if "tokens" in r]
+RECORDS = [r for r in read_records("paper_examples.txt") if "tokens" in r and "regex" in r]
 
 
 def bits(mask_row, V):
