@@ -26,6 +26,9 @@ namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kDepth = CSTR_STACK_DEPTH;
+constexpr int kDedupMaxClasses = 16;    // duplicate-column pass: automata with at most this many
+constexpr int kDedupMinTokens = 8192;   // byte classes, vocabularies of at least this many tokens
+constexpr int kDedupMinStates = 2048;   // and enough states for the walk to outweigh the extra passes
 
 struct BuildParams {
     const void *tt;            // [n_classes][row]
@@ -42,6 +45,10 @@ struct BuildParams {
     int tokens_per_cta;
     int warps_s;               // warps of a CTA that split its states ...
     int warps_t;               // ... times warps that split its token chunk
+    // duplicate-column pass: desc lists one representative per class string and
+    // its length is only known on the device
+    const int32_t *count_dev;  // null: desc holds all V tokens
+    const uint32_t *reptok;    // [V] representative token id per token id, or null
 };
 
 // NS consecutive table entries per lane travel as one aligned unit (one vector
@@ -147,8 +154,13 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     s_stack[0] = pk;
     __syncwarp();
 
-    const int c_begin = blockIdx.y * p.tokens_per_cta;
-    const int c_end = min(p.V, c_begin + p.tokens_per_cta);
+    int n_tokens = p.V, tokens_per_cta = p.tokens_per_cta;
+    if (p.count_dev) {                                   // representatives only: equal shares
+        n_tokens = *p.count_dev;
+        tokens_per_cta = (n_tokens + (int)gridDim.y - 1) / (int)gridDim.y;
+    }
+    const int c_begin = blockIdx.y * tokens_per_cta;
+    const int c_end = min(n_tokens, c_begin + tokens_per_cta);
     const int per_t = (c_end - c_begin + p.warps_t - 1) / p.warps_t;
     const int t_begin = c_begin + warp_t * per_t;
     const int t_end = min(c_end, t_begin + per_t);
@@ -241,7 +253,8 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
 // NS l + k of the block in bit l.
 __global__ void __launch_bounds__(256)
 mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
-                      long long ldw, int n_states, int V, int ns)
+                      long long ldw, int n_states, int V, int ns,
+                      const uint32_t *__restrict__ reptok)
 {
     __shared__ uint32_t tile[8][1024];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -253,7 +266,9 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
         const long long tokid = (long long)w0 * 32 + t;
         uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
         if (tokid < V) {
-            const uint4 *src = (const uint4 *)(maskT + tokid * ldb + sb0);   // ldb, sb0 multiples of 8
+            // after a duplicate-column pass only the representatives' rows were written
+            const long long rowid = reptok ? (long long)__ldg(reptok + tokid) : tokid;
+            const uint4 *src = (const uint4 *)(maskT + rowid * ldb + sb0);   // ldb, sb0 multiples of 8
             a = __ldg(src);
             b = __ldg(src + 1);
         }
@@ -322,6 +337,221 @@ apply_terminals_kernel(const int32_t *__restrict__ tstate, const uint32_t *__res
     }
 }
 
+// ---- duplicate columns -------------------------------------------------------
+//
+// Two tokens that read as the same string of byte classes have the same column
+// of the table in every state.  For automata with few byte classes (a quoted
+// string tells apart quote, backslash and "anything else") a natural vocabulary
+// collapses to a few hundred class strings, so the walk runs for one
+// representative per class string and the other columns are copies.
+// Grouping is by a 64-bit hash in an open-addressing table, then proven by an
+// exact comparison: a token whose class string differs from its group's
+// representative (a hash collision) simply stays its own representative.
+
+__device__ __forceinline__ unsigned long long class_string_hash(const uint8_t *__restrict__ cls,
+                                                                const uint8_t *__restrict__ b,
+                                                                unsigned n)
+{
+    unsigned long long h = 0x9e3779b97f4a7c15ull ^ (unsigned long long)n;
+    for (unsigned k = 0; k < n; ++k) {
+        h = (h ^ (unsigned long long)cls[b[k]]) * 0x100000001b3ull;
+        h ^= h >> 29;
+    }
+    h ^= h >> 32;
+    h *= 0xd6e8feb86659fd93ull;
+    h ^= h >> 32;
+    return h | 1ull;                                     // 0 marks an empty slot
+}
+
+// Each group's slot ends up holding the smallest sorted index of the group.
+__global__ void __launch_bounds__(256)
+group_insert_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
+                    const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int V,
+                    int eos_id, unsigned long long *key, uint32_t *minv, uint32_t slots)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= V)
+        return;
+    const unsigned tok = desc[i].x;
+    if ((int)tok == eos_id)
+        return;                                          // the EOS column is special: never shared
+    const uint32_t b0 = off[tok], b1 = off[tok + 1];
+    const unsigned long long h = class_string_hash(cls, bytes + b0, b1 - b0);
+    uint32_t slot = (uint32_t)(h >> 20) & (slots - 1);
+    for (uint32_t probe = 0; probe < slots; ++probe) {   // slots >= 4 V: an empty slot exists
+        unsigned long long seen = *(volatile unsigned long long *)(key + slot);
+        if (seen == 0ull)
+            seen = atomicCAS(key + slot, 0ull, h);       // returns 0 if this thread claimed it
+        if (seen == 0ull || seen == h) {
+            // the minimum only ever falls, so a value already at or below i needs no atomic:
+            // thousands of tokens share a few popular class strings
+            if (*(volatile uint32_t *)(minv + slot) > (uint32_t)i)
+                atomicMin(minv + slot, (uint32_t)i);
+            return;
+        }
+        slot = (slot + 1) & (slots - 1);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+group_resolve_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
+                     const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int V,
+                     int eos_id, const unsigned long long *__restrict__ key,
+                     const uint32_t *__restrict__ minv, uint32_t slots, uint32_t *__restrict__ rep,
+                     uint32_t *__restrict__ reptok)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= V)
+        return;
+    const unsigned tok = desc[i].x;
+    uint32_t r = (uint32_t)i;
+    unsigned rtok = tok;
+    if ((int)tok != eos_id) {
+        const uint32_t b0 = off[tok], n = off[tok + 1] - b0;
+        const unsigned long long h = class_string_hash(cls, bytes + b0, n);
+        uint32_t slot = (uint32_t)(h >> 20) & (slots - 1);
+        for (uint32_t probe = 0; probe < slots; ++probe) {
+            const unsigned long long k = key[slot];
+            if (k == h) {
+                r = minv[slot];
+                break;
+            }
+            if (k == 0ull)
+                break;                                   // cannot happen after the insert pass
+            slot = (slot + 1) & (slots - 1);
+        }
+        if (r != (uint32_t)i) {                          // prove it: same length, same classes
+            rtok = desc[r].x;
+            const uint32_t c0 = off[rtok], m = off[rtok + 1] - c0;
+            bool same = m == n && (int)rtok != eos_id;
+            for (uint32_t k = 0; same && k < n; ++k)
+                same = cls[bytes[b0 + k]] == cls[bytes[c0 + k]];
+            if (!same) {
+                r = (uint32_t)i;
+                rtok = tok;
+            }
+        }
+    }
+    rep[i] = r;
+    reptok[tok] = rtok;
+}
+
+// Representatives in sorted order: a count per block of 1,024 sorted tokens, an
+// exclusive scan of the counts, and a scatter by rank.
+__global__ void __launch_bounds__(1024)
+group_count_kernel(const uint32_t *__restrict__ rep, int V, int32_t *__restrict__ blk)
+{
+    const int i = blockIdx.x * 1024 + threadIdx.x;
+    const int n = __syncthreads_count(i < V && rep[i] == (uint32_t)i);
+    if (threadIdx.x == 0)
+        blk[blockIdx.x] = n;
+}
+
+__global__ void __launch_bounds__(1024)
+group_scan_kernel(int32_t *__restrict__ blk, int n_blocks, int32_t *__restrict__ count)
+{
+    __shared__ int s_sum[1024];
+    const int t = threadIdx.x;
+    const int per = (n_blocks + 1023) / 1024;
+    const int lo = min(n_blocks, t * per), hi = min(n_blocks, lo + per);
+    int sum = 0;
+    for (int k = lo; k < hi; ++k)
+        sum += blk[k];
+    s_sum[t] = sum;
+    __syncthreads();
+    if (t == 0) {                                        // 1,024 partial sums: a serial scan is enough
+        int acc = 0;
+        for (int k = 0; k < 1024; ++k) {
+            const int c = s_sum[k];
+            s_sum[k] = acc;
+            acc += c;
+        }
+        *count = acc;
+    }
+    __syncthreads();
+    int acc = s_sum[t];
+    for (int k = lo; k < hi; ++k) {
+        const int c = blk[k];
+        blk[k] = acc;                                    // exclusive prefix
+        acc += c;
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+group_scatter_kernel(const uint32_t *__restrict__ rep, int V, const int32_t *__restrict__ blk,
+                     uint32_t *__restrict__ uniq)
+{
+    __shared__ int s_warp[32];
+    const int i = blockIdx.x * 1024 + threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool flag = i < V && rep[i] == (uint32_t)i;
+    const unsigned bal = __ballot_sync(kFull, flag);
+    if (lane == 0)
+        s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+        int v = s_warp[lane], incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o)
+                incl += y;
+        }
+        s_warp[lane] = incl - v;
+    }
+    __syncthreads();
+    if (flag)
+        uniq[blk[blockIdx.x] + s_warp[warp] + __popc(bal & ((1u << lane) - 1u))] = (uint32_t)i;
+}
+
+// Trie descriptors of the representatives' own sorted list: entry k = { token id,
+// length | shared prefix with representative k-1 (clipped to the walk's stack
+// depth) << 24, first 8 bytes after that prefix }.
+__global__ void __launch_bounds__(256)
+group_desc_kernel(const uint4 *__restrict__ desc, const uint32_t *__restrict__ uniq,
+                  const int32_t *__restrict__ count, const uint8_t *__restrict__ bytes,
+                  const uint32_t *__restrict__ off, uint4 *__restrict__ udesc)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= *count)
+        return;
+    const unsigned tok = desc[uniq[k]].x;
+    const uint32_t b0 = off[tok], len = off[tok + 1] - b0;
+    uint32_t shared = 0;
+    if (k > 0) {
+        const unsigned ptok = desc[uniq[k - 1]].x;
+        const uint32_t p0 = off[ptok], plen = off[ptok + 1] - p0;
+        const uint32_t m = min(min(len, plen), (uint32_t)kDepth);
+        while (shared < m && bytes[b0 + shared] == bytes[p0 + shared])
+            ++shared;
+    }
+    uint32_t lo8 = 0, hi8 = 0;
+    for (uint32_t j = 0; j < 8 && shared + j < len; ++j) {
+        const uint32_t byte = bytes[b0 + shared + j];
+        if (j < 4)
+            lo8 |= byte << (8 * j);
+        else
+            hi8 |= byte << (8 * (j - 4));
+    }
+    udesc[k] = make_uint4(tok, len | (shared << 24), lo8, hi8);
+}
+
+// One CTA per token: a token that is not its own representative takes the
+// representative's row of next (token-major: contiguous).
+__global__ void __launch_bounds__(256)
+expand_rows_kernel(const uint32_t *__restrict__ reptok, unsigned char *__restrict__ next,
+                   unsigned long long next_pitch, int next_n16)
+{
+    const uint32_t v = blockIdx.x;
+    const uint32_t r = reptok[v];
+    if (r == v)
+        return;
+    const uint4 *src = (const uint4 *)(next + r * next_pitch);
+    uint4 *dst = (uint4 *)(next + v * next_pitch);
+    for (int k = threadIdx.x; k < next_n16; k += blockDim.x)
+        __stcs(dst + k, __ldg(src + k));
+}
+
 template <typename ST, typename NT, int NS, bool SMEM>
 cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
                         cudaStream_t stream)
@@ -383,6 +613,36 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     if (dfa->wide && !t->wide)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
     const size_t st = dfa->wide ? 4 : 2;
+
+    // Duplicate-column pass for large automata with few byte classes over a large
+    // vocabulary (elsewhere class strings rarely repeat, or the walk is too short
+    // for the extra passes to pay).
+    const bool dedup = dfa->n_classes <= kDedupMaxClasses && t->V >= kDedupMinTokens &&
+                       dfa->n_states >= kDedupMinStates;
+    p.count_dev = nullptr;
+    p.reptok = nullptr;
+    if (dedup) {
+        CSTR_CUDA_TRY(cudaMemsetAsync(t->group_key, 0, (size_t)t->group_slots * 8, stream));
+        CSTR_CUDA_TRY(cudaMemsetAsync(t->group_min, 0xff, (size_t)t->group_slots * 4, stream));
+        const unsigned g = (unsigned)((t->V + 255) / 256);
+        group_insert_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
+                                                   t->eos_id, t->group_key, t->group_min,
+                                                   t->group_slots);
+        group_resolve_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
+                                                    t->eos_id, t->group_key, t->group_min,
+                                                    t->group_slots, t->group_rep, t->group_reptok);
+        const int n_blk = (t->V + 1023) / 1024;
+        group_count_kernel<<<n_blk, 1024, 0, stream>>>(t->group_rep, t->V, t->group_blk);
+        group_scan_kernel<<<1, 1024, 0, stream>>>(t->group_blk, n_blk, t->group_count);
+        group_scatter_kernel<<<n_blk, 1024, 0, stream>>>(t->group_rep, t->V, t->group_blk,
+                                                         t->group_uniq);
+        group_desc_kernel<<<g, 256, 0, stream>>>(vc->desc, t->group_uniq, t->group_count, vc->bytes,
+                                                 vc->off, t->group_desc);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        p.desc = t->group_desc;
+        p.count_dev = t->group_count;
+        p.reptok = t->group_reptok;
+    }
 
     // States per lane: enough states per warp to amortise the per-token work,
     // without leaving most lanes idle on small automata.
@@ -466,11 +726,21 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
                          cudaGetErrorString(e));
 
     const int ballot_words = ((S + per_warp - 1) / per_warp) * ns;
+    if (dedup) {
+        const size_t nt = t->wide ? 4 : 2;
+        long long used = (long long)state_warps * per_warp;          // entries the walk wrote
+        if (used > t->lds)
+            used = t->lds;
+        expand_rows_kernel<<<(unsigned)t->V, 256, 0, stream>>>(
+            t->group_reptok, (unsigned char *)t->next, (unsigned long long)t->lds * nt,
+            (int)(used * nt / 16));
+        CSTR_CUDA_TRY(cudaGetLastError());
+    }
     dim3 tgrid((unsigned)((ballot_words + 7) / 8), (unsigned)(t->ldw / 32));
     if (tgrid.y > 65535u)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: vocabulary too large for one launch");
     mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
-                                                     ns);
+                                                     ns, p.reptok);
     CSTR_CUDA_TRY(cudaGetLastError());
 
     if (dfa->n_term_states > 0) {

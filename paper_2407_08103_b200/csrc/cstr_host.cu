@@ -488,6 +488,14 @@ extern "C" void cstr_free_table(cstr_table_t *t)
     cudaFree(t->mask);
     cudaFree(t->maskT);
     cudaFree(t->accept);
+    cudaFree(t->group_key);
+    cudaFree(t->group_min);
+    cudaFree(t->group_rep);
+    cudaFree(t->group_reptok);
+    cudaFree(t->group_desc);
+    cudaFree(t->group_count);
+    cudaFree(t->group_uniq);
+    cudaFree(t->group_blk);
     cstr_free_vocab(t->owned_vocab);
     delete t;
 }
@@ -527,6 +535,25 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
         e = cudaMalloc((void **)&t->maskT, maskT_bytes);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->accept, (size_t)max_states);
+    t->group_slots = 1024;
+    while (t->group_slots < 4ull * (unsigned)t->V && t->group_slots < (1u << 30))
+        t->group_slots <<= 1;
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_key, (size_t)t->group_slots * 8);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_min, (size_t)t->group_slots * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_rep, (size_t)t->V * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_reptok, (size_t)t->V * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_desc, (size_t)t->V * sizeof(uint4));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_count, 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_uniq, (size_t)t->V * 4);
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->group_blk, ((size_t)t->V / 1024 + 1) * 4);
     if (e == cudaSuccess)
         e = cudaMemset(t->mask, 0, mask_bytes);   // padding words stay zero for good
     if (e == cudaSuccess)

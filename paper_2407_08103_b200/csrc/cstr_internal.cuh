@@ -97,6 +97,19 @@ struct cstr_table {
     int32_t start;
     int32_t eos_id;
     int32_t code_shift; // next entries are CSTR_PERM(state) << code_shift (1: 16-bit DFA, 2: 32-bit)
+    // Scratch of the builder's duplicate-column pass (tokens that read as the same
+    // string of byte classes share one walk): an open-addressing table keyed by a
+    // 64-bit hash of the class string, each sorted token's representative, the
+    // representatives' own trie-ordered descriptor list and its length.
+    uint32_t group_slots;          // power of two >= 4 V
+    unsigned long long *group_key; // DEVICE [group_slots]
+    uint32_t *group_min;           // DEVICE [group_slots] smallest sorted index of the group
+    uint32_t *group_rep;           // DEVICE [V] representative's sorted index, per sorted index
+    uint32_t *group_reptok;        // DEVICE [V] representative's token id, per token id
+    uint4 *group_desc;             // DEVICE [V] descriptors of the representatives, in order
+    int32_t *group_count;          // DEVICE [1] number of representatives
+    uint32_t *group_uniq;          // DEVICE [V] sorted indices of the representatives, in order
+    int32_t *group_blk;            // DEVICE [ceil(V / 1024)] representatives per 1,024 sorted tokens
 };
 
 struct cstr_workspace {

@@ -164,3 +164,41 @@ def test_long_shared_prefixes_and_long_suffixes():
     dfa = (chain, np.ones(S, dtype=np.uint8), 5)
     (table,) = gpu_tables([dfa], vb, vo)
     check_table(table, dfa, vb, vo)
+
+
+@pytest.mark.parametrize("case", ["string", "two_classes", "one_class", "eos_and_terminals"])
+def test_few_byte_classes_take_the_duplicate_column_pass(case):
+    # Automata of >= 2,048 states with at most 16 byte classes over >= 8,192 tokens share
+    # one walk per class string; every column must still be the oracle's, copies included.
+    from synth import make_vocab_geometric
+    rng = np.random.default_rng(11)
+    vb, vo = make_vocab_geometric(9000 if case != "string" else 20000, seed=5)
+    V = vo.size - 1
+    eos, term, sets = -1, None, None
+    if case == "string":
+        dfa = regex_to_dfa(r'"([^"\\]|\\.){0,1100}"')        # 3 classes, 2,203 states
+    elif case == "two_classes":
+        dfa = regex_to_dfa(r"([a-z ]{3}[^a-z ]){0,600}")
+    elif case == "one_class":
+        dfa = regex_to_dfa(r".{0,2100}")
+    else:
+        full = regex_to_dfa(r'x(?P<WORD>)+"[^"]{0,2050}"', ["WORD"])
+        dfa = (np.ascontiguousarray(full[0][:, :256]), full[1], full[2])
+        term = [np.ascontiguousarray(full[0][:, 256:])]
+        sets = (rng.random(V) < 0.3).astype(np.uint32)
+        eos = 4242                                             # a token equal to many others
+    toks = [bytes(vb[vo[v]:vo[v + 1]]) for v in range(V)]
+    assert len(set(toks)) < V                                  # the vocabulary repeats strings
+    (table,) = gpu_tables([dfa], vb, vo, eos_id=eos, term_trans=term, token_sets=sets)
+    S = dfa[0].shape[0]
+    assert S >= 2048
+    sample = sorted(set([0, 1, 2, 255, 256, 257, S - 3, S - 2, S - 1] + rng.integers(0, S, 40).tolist()))
+    check_table(table, dfa, vb, vo, eos_id=eos, states=sample,
+                term_trans=None if term is None else term[0], token_sets=sets)
+    # rebuilding into the same table reuses the grouping scratch
+    h = (cstr.cstr_load_dfa_terminals(dfa[0], term[0], dfa[1], dfa[2]) if term is not None
+         else cstr.cstr_load_dfa(*dfa))
+    cstr.cstr_table_build(table, h, eos)
+    torch.cuda.synchronize()
+    check_table(table, dfa, vb, vo, eos_id=eos, states=[0, dfa[0].shape[0] - 1],
+                term_trans=None if term is None else term[0], token_sets=sets)
