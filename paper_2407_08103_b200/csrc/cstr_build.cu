@@ -247,16 +247,19 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
 
 // mask[q][w] bit t = validity of token 32 w + t in state q, gathered from the
 // per-token ballot words: 32 x 32 bit-matrix transposes.  A CTA takes 1,024
-// tokens (32 mask words) x 8 ballot words; warp j transposes the 32 tiles of
-// ballot word sb0 + j and each lane writes the 32 consecutive words of its
-// state row (128 bytes).  Ballot word k of a block of 32 NS states holds state
-// NS l + k of the block in bit l.
+// tokens (32 mask words) x 8 ballot words.  Warp j handles ballot word sb0 + j;
+// lane l takes the 32 tokens of mask word w0 + l into registers, transposes the
+// 32 x 32 bit block in registers (no shuffles), and for each of the 32 states
+// the warp stores 32 consecutive mask words of that state's row (128 bytes).
+// Ballot word k of a block of 32 NS states holds state NS l + k of the block
+// in bit l.
 __global__ void __launch_bounds__(256)
 mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
                       long long ldw, int n_states, int V, int ns,
                       const uint32_t *__restrict__ reptok)
 {
-    __shared__ uint32_t tile[8][1024];
+    // one padding word per 32 tokens: lane l then reads word 33 l + r, free of bank conflicts
+    __shared__ uint32_t tile[8][1024 + 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // x = group of 8 ballot words, y = group of 32 mask words: CTAs that read
     // the four 32-byte quarters of the same maskT lines are launched together
@@ -272,34 +275,38 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
             a = __ldg(src);
             b = __ldg(src + 1);
         }
-        tile[0][t] = a.x; tile[1][t] = a.y; tile[2][t] = a.z; tile[3][t] = a.w;
-        tile[4][t] = b.x; tile[5][t] = b.y; tile[6][t] = b.z; tile[7][t] = b.w;
+        const int at = t + (t >> 5);
+        tile[0][at] = a.x; tile[1][at] = a.y; tile[2][at] = a.z; tile[3][at] = a.w;
+        tile[4][at] = b.x; tile[5][at] = b.y; tile[6][at] = b.z; tile[7][at] = b.w;
     }
     __syncthreads();
     const int sbw = sb0 + warp;
     const int first_state = (sbw / ns) * (ns * 32) + (sbw % ns);
     if (first_state >= n_states)
         return;
-    const int q = first_state + ns * lane;
-    uint32_t outw[32];
+    uint32_t x[32];                                      // x[r]: token 32 (w0 + lane) + r, bit = state slot
 #pragma unroll
-    for (int wi = 0; wi < 32; ++wi) {
-        uint32_t x = tile[warp][wi * 32 + lane];         // row = token, bit = state slot
-        uint32_t m = 0x0000ffffu;
+    for (int r = 0; r < 32; ++r)
+        x[r] = tile[warp][33 * lane + r];
+    uint32_t m = 0x0000ffffu;
 #pragma unroll
-        for (int j = 16; j >= 1; j >>= 1) {
-            const uint32_t y = __shfl_xor_sync(kFull, x, j);
-            x = (lane & j) ? ((x & ~m) | ((y >> j) & m)) : ((x & m) | ((y << j) & ~m));
-            m ^= m << (j >> 1);
+    for (int j = 16; j >= 1; j >>= 1) {
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            if ((k & j) == 0) {
+                const uint32_t t = ((x[k] >> j) ^ x[k + j]) & m;
+                x[k] ^= t << j;
+                x[k + j] ^= t;
+            }
         }
-        outw[wi] = x;                                    // row = state slot, bit = token
+        m ^= m << (j >> 1);
     }
-    if (q < n_states) {
-        uint4 *dst = (uint4 *)(mask + (long long)q * ldw + w0);              // ldw multiple of 32
+    // now x[s]: state slot s, bit = token: mask word w0 + lane of state first_state + ns s
+    uint32_t *dst = mask + (long long)first_state * ldw + w0 + lane;         // ldw multiple of 32
 #pragma unroll
-        for (int g = 0; g < 8; ++g)
-            dst[g] = make_uint4(outw[4 * g], outw[4 * g + 1], outw[4 * g + 2], outw[4 * g + 3]);
-    }
+    for (int sl = 0; sl < 32; ++sl)
+        if (first_state + ns * sl < n_states)            // warp-uniform
+            dst[(long long)ns * sl * ldw] = x[sl];
 }
 
 // Terminal-label edges (wildcards matched by pre-computed token sets): for
