@@ -58,6 +58,10 @@ def parse_args():
     ap.add_argument("--skip-other-workloads", action="store_true",
                     help="do not time the four other workloads (reported under 'other_workloads')")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--build-only", default=None, metavar="WORKLOAD",
+                    help="time only the token-table build of one workload (with --case small: the "
+                         "4,099-state string DFA / a 4,096-state random DFA) and print its entry; "
+                         "for profiler captures, not a bench line")
     ap.add_argument("--pushdown-only", action="store_true",
                     help="time only the push-down step leg (batch 128 with --case small) and print "
                          "its entry; for profiler captures, not a bench line")
@@ -400,6 +404,39 @@ def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=5
             "status_rows": {"bad": bad, "empty_mask": empty, "overflow": overflow}}
 
 
+def time_build_only(torch, cstr, name, case, stream, repeats=4):
+    """Token-table build of one workload's (first) DFA over its vocabulary."""
+    from synth import random_range_dfa
+    from synth.configs import CONFIGS, config_dfas, config_vocab
+    from synth.regex_frontend import regex_to_dfa
+    w = CONFIGS[name]
+    vb, vo = config_vocab(name)
+    if case == "small" and name == "string_256k":
+        dfa = regex_to_dfa(w.regex.replace("{0,4096}", "{0,2048}"))
+    elif case == "small" and name == "random10k_256k":
+        dfa = random_range_dfa(4096, seed=2)
+    else:
+        dfa = config_dfas(name)[0]
+    V, S = vo.size - 1, int(dfa[0].shape[0])
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    h = cstr.cstr_load_dfa(*dfa)
+    table = cstr.cstr_table_create(vocab, S)
+    ms = []
+    for _ in range(repeats):
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        cstr.cstr_table_build(table, h, -1, stream)
+        a1.record(stream)
+        a1.synchronize()
+        ms.append(a0.elapsed_time(a1))
+    best = float(np.mean(ms[1:]))
+    peak, kind = measured_hbm_peak()
+    gbs = S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9
+    return {"workload": name + (" (small case)" if case == "small" else ""), "dfa_states": S,
+            "vocab": V, "ms": best, "transitions_per_s": S * V / (best * 1e-3), "store_gbs": gbs,
+            "frac_of_hbm_peak": gbs / peak, "peak_kind": "of %s" % kind}
+
+
 def time_small_batches(torch, cstr, table, V, dev, stream, batches=(1, 8, 64)):
     """Step latency for small batches at the full vocabulary (fp32, greedy): 64
     steps captured in one CUDA graph, logits rotating through a pool larger than
@@ -504,6 +541,10 @@ def main():
     from synth import normal_logits
     libbuild.build_library()
 
+    if args.build_only:
+        print(json.dumps({"table_build": time_build_only(torch, cstr, args.build_only, args.case,
+                                                         torch.cuda.current_stream())}))
+        return
     if args.pushdown_only:
         entry = time_pushdown(torch, cstr, PushdownDecoder, dev, torch.cuda.current_stream(),
                               measured_hbm_peak()[0], B=128 if args.case == "small" else 512,

@@ -373,11 +373,11 @@ __device__ __forceinline__ unsigned long long class_string_hash(const uint8_t *_
 // Each group's slot ends up holding the smallest sorted index of the group.
 __global__ void __launch_bounds__(256)
 group_insert_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
-                    const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int V,
-                    int eos_id, unsigned long long *key, uint32_t *minv, uint32_t slots)
+                    const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int i_begin,
+                    int i_end, int eos_id, unsigned long long *key, uint32_t *minv, uint32_t slots)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= V)
+    const int i = i_begin + blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= i_end)
         return;
     const unsigned tok = desc[i].x;
     if ((int)tok == eos_id)
@@ -632,9 +632,16 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_key, 0, (size_t)t->group_slots * 8, stream));
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_min, 0xff, (size_t)t->group_slots * 4, stream));
         const unsigned g = (unsigned)((t->V + 255) / 256);
-        group_insert_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
-                                                   t->eos_id, t->group_key, t->group_min,
-                                                   t->group_slots);
+        // A small first launch seeds the table: thousands of tokens share a few
+        // popular class strings, and once a group's minimum is in place the bulk
+        // of the tokens finds it with plain loads instead of same-address atomics.
+        const int seed = 4096;
+        group_insert_kernel<<<seed / 256, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, 0,
+                                                            seed, t->eos_id, t->group_key,
+                                                            t->group_min, t->group_slots);
+        group_insert_kernel<<<(unsigned)((t->V - seed + 255) / 256), 256, 0, stream>>>(
+            vc->desc, vc->bytes, vc->off, dfa->cls, seed, t->V, t->eos_id, t->group_key,
+            t->group_min, t->group_slots);
         group_resolve_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
                                                     t->eos_id, t->group_key, t->group_min,
                                                     t->group_slots, t->group_rep, t->group_reptok);
