@@ -3,7 +3,7 @@
 A plain, slow CPU statement of the path the CUDA library implements:
 
 * ``regex_dfa``     regex -> Thompson NFA -> subset construction -> trim
-                    (Algorithm 2, first lines; Section 2.1);
+                    (Algorithm 2, automaton construction; Section 2.1);
 * ``token_table``   T[q][v] = delta*(q, bytes(v)) and the per-state allowed-token
                     bitmask (Algorithm 1 composed with the DFA, Theorem 2);
 * ``step``          mask, penalise with -inf, select, advance for a batch of

@@ -1,7 +1,7 @@
 """ORACLE (test infrastructure, not product code): regex -> NFA -> DFA.
 
 Follows the paper's pipeline for the character-level automaton A_R
-(Algorithm 2, first lines; Section 2.1): a regular expression is turned into a
+(Algorithm 2, automaton construction; Section 2.1): a regular expression is turned into a
 non-deterministic FSA with epsilon edges by Thompson's construction
 (BuildRegexFSA), and that FSA is determinized by the subset construction
 (Section 2.1 recalls that every FSA has an equivalent deterministic one;

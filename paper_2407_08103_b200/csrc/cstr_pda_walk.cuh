@@ -60,7 +60,7 @@ __device__ __forceinline__ int pda_walk(const cstr_pda_view &P, int q, const int
     return WALK_OK;
 }
 
-// Traverse the edge of token `tok` for row r (Algorithm 3, last line): walk the
+// Traverse the edge of token `tok` for row r (Algorithm 3, edge traversal): walk the
 // token's bytes from the row's state and stack, which yields the edge's target
 // and stack edit.  `active` = the row had a usable state and stack.
 __device__ __forceinline__ void pda_traverse(const cstr_pda_advance &a, int r, bool active, int tok)
