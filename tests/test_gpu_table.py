@@ -202,3 +202,30 @@ def test_few_byte_classes_take_the_duplicate_column_pass(case):
     torch.cuda.synchronize()
     check_table(table, dfa, vb, vo, eos_id=eos, states=[0, dfa[0].shape[0] - 1],
                 term_trans=None if term is None else term[0], token_sets=sets)
+
+
+def test_duplicate_column_pass_wide_entries_and_table_reuse():
+    # 32-bit next entries (more than 32,766 states) through the duplicate-column pass, then the
+    # same table rebuilt for automata that take the plain walk (many byte classes; few states).
+    from synth import make_vocab_geometric
+    vb, vo = make_vocab_geometric(8200, seed=9)
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    wide = regex_to_dfa(r"[a-z ]{0,33000}")
+    S = wide[0].shape[0]
+    assert S > 32767
+    table = cstr.cstr_table_create(vocab, S)
+    cstr.cstr_table_build(table, cstr.cstr_load_dfa(*wide))
+    torch.cuda.synchronize()
+    check_table(table, wide, vb, vo, states=[0, 1, 255, 256, 12345, 32766, 32767, 32768, S - 2, S - 1])
+    rng = np.random.default_rng(4)
+    many = dense_random_dfa(rng, 300, live=0.6)                      # 256 byte classes
+    cstr.cstr_table_build(table, cstr.cstr_load_dfa(*many))
+    torch.cuda.synchronize()
+    check_table(table, many, vb, vo, states=[0, 1, 150, 299])
+    small = regex_to_dfa(r'"[^"]{0,40}"')                            # few classes, few states
+    cstr.cstr_table_build(table, cstr.cstr_load_dfa(*small))
+    torch.cuda.synchronize()
+    check_table(table, small, vb, vo)
+    cstr.cstr_table_build(table, cstr.cstr_load_dfa(*wide), 300)      # and back, with an EOS token
+    torch.cuda.synchronize()
+    check_table(table, wide, vb, vo, eos_id=300, states=[0, 77, S - 1])
