@@ -150,6 +150,7 @@ def test_stackless_pda_matches_the_finite_state_table():
 
 @pytest.mark.parametrize("dtype,gumbel,vocab_size,pad", [
     ("f32", False, 2051, 0), ("bf16", False, 4096, 8), ("f32", True, 3000, 4),
+    ("bf16", True, 2048, 0),
 ])
 def test_decode_loop_json(dtype, gumbel, vocab_size, pad):
     P = json_pda(space=True)
