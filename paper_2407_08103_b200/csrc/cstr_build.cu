@@ -104,7 +104,7 @@ __device__ __forceinline__ void unpack_entries(typename Unit<ESZ * NS>::type u, 
 // it is stored as word (q0 / 32 + j) of the token's maskT row and un-permuted
 // by the transpose kernel.
 template <typename ST, typename NT, int NS, bool SMEM>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(NS == 8 ? 1024 : 512)
 build_trie_kernel(const __grid_constant__ BuildParams p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -687,11 +687,17 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     const bool in_smem = 1024 + 4 * stack_per_warp + table_bytes <= cta_max;
     const size_t fixed = 1024 + (in_smem ? table_bytes : 0);
     size_t budget = in_smem ? cta_half : 48 * 1024;
-    if (fixed + 8 * stack_per_warp > budget)
-        budget = cta_max;
+    int warp_cap = 16;
+    bool one_cta_per_sm = false;
+    if (fixed + 8 * stack_per_warp > budget) {
+        budget = cta_max;            // one CTA per SM: let it hold all the warps the register
+        one_cta_per_sm = true;       // file allows (the 8-states-per-lane kernels fit 1,024 threads)
+        if (ns == 8)
+            warp_cap = 32;
+    }
     int max_warps = (int)((budget - fixed) / stack_per_warp);
-    if (max_warps > 16)
-        max_warps = 16;
+    if (max_warps > warp_cap)
+        max_warps = warp_cap;
     if (max_warps < 1)
         max_warps = 1;
     int state_groups = (state_warps + max_warps - 1) / max_warps;
@@ -720,6 +726,14 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     if (tokens_per_cta < min_tokens)
         tokens_per_cta = min_tokens;
     chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
+    if (one_cta_per_sm && state_groups * chunks < dev_sms) {
+        // fewer CTAs than SMs and only one fits an SM: shorter chunks (at least
+        // 32 tokens per warp) so that every SM gets one
+        const long long fill = (dev_sms + state_groups - 1) / state_groups;
+        const long long per = (t->V + fill - 1) / fill;
+        tokens_per_cta = per > 32LL * warps_t ? per : 32LL * warps_t;
+        chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
+    }
     if (chunks > 65535) {
         chunks = 65535;
         tokens_per_cta = (t->V + chunks - 1) / chunks;
