@@ -162,7 +162,7 @@ static int ends_with(const int32_t *s, int32_t depth, const tok_edge *e)
     return 1;
 }
 
-#define EDGE_CAP 64
+#define EDGE_CAP 512
 
 /* The edge Algorithm 3 traverses for token v from (q, s), or NULL if v is not in A. */
 static const tok_edge *matching_edge(const pda_view *P, int32_t q, const int32_t *s, int32_t depth,

@@ -19,4 +19,5 @@ from .constraints import (  # noqa: F401
 from .logits import normal_logits, gumbel_noise, f32_to_bf16_bits, bf16_bits_to_f32  # noqa: F401
 from .regex_frontend import regex_to_dfa  # noqa: F401
 from .configs import CONFIGS, get_config  # noqa: F401
-from .pda import Pda, PdaBuilder, anbn_pda, dyck_pda, json_pda, stackless_pda  # noqa: F401
+from .pda import (Pda, PdaBuilder, anbn_pda, dyck_pda, json_pda, random_pda,  # noqa: F401
+                  stackless_pda)

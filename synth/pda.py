@@ -217,3 +217,38 @@ def stackless_pda(trans: np.ndarray, accept: np.ndarray, start: int) -> Pda:
                np.asarray(trans)[src, inp].astype(np.int32), zeros, np.zeros(0, dtype=np.int32),
                zeros.copy(), np.zeros(0, dtype=np.int32),
                np.ascontiguousarray(accept, dtype=np.uint8))
+
+
+def random_pda(seed: int, n_states: int = 6, n_symbols: int = 3, alphabet: bytes = b"abcd",
+               max_push: int = 3) -> Pda:
+    """A random deterministic real-time PDA over a small alphabet: per (state,
+    byte) either no edge, one edge that pops nothing, or edges popping pairwise
+    different symbols; every edge pushes 0..max_push random symbols (an edge
+    may push back the symbol it popped).  About a third of the states accept."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    b = PdaBuilder()
+    states = ["q%d" % i for i in range(n_states)]
+    syms = ["s%d" % i for i in range(n_symbols)]
+    for q in states:
+        b.state(q)
+    for y in syms:
+        b.symbol(y)
+
+    def pushes():
+        return tuple(syms[int(k)] for k in rng.integers(0, n_symbols, size=int(rng.integers(0, max_push + 1))))
+
+    for q in states:
+        for byte in alphabet:
+            kind = rng.random()
+            if kind < 0.25 or n_symbols == 0 and kind < 0.5:
+                continue
+            if kind < 0.6 or n_symbols == 0:
+                b.edge(q, byte, states[int(rng.integers(n_states))], pushes=pushes() if n_symbols else ())
+            else:
+                for y in syms:
+                    if rng.random() < 0.7:
+                        b.edge(q, byte, states[int(rng.integers(n_states))], pops=(y,), pushes=pushes())
+    for q in states:
+        if rng.random() < 0.35:
+            b.final.add(q)
+    return b.build(states[0])

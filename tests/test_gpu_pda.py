@@ -8,7 +8,7 @@ from gpu_common import DEV, bits_equal, from_dev_logits, to_dev_logits
 from oracle import pda as op
 from paper_2407_08103_b200 import cstr
 from synth import (anbn_pda, dyck_pda, gumbel_noise, json_pda, make_vocab_json, normal_logits,
-                   stackless_pda, vocab_from_strings)
+                   random_pda, stackless_pda, vocab_from_strings)
 from synth.configs import config_dfas, config_vocab
 
 pytestmark = pytest.mark.gpu
@@ -291,3 +291,35 @@ def test_full_size_json_256k_sampled_rows():
         o_states, o_stacks, o_depth = ref["states"], ref["stacks"], ref["depth"]
         deepest = max(deepest, int(o_depth.max()))
     assert deepest >= 3 and (o_states >= 0).any()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_pdas_table_and_decode_loop(seed):
+    # random deterministic PDAs (pops, multi-symbol pushes, edges that push back what they
+    # popped) over all short strings of a small alphabet as the vocabulary
+    import itertools
+    rng = np.random.default_rng(seed)
+    n_symbols = int(rng.choice([1, 2, 3]))
+    P = random_pda(seed, n_states=int(rng.choice([2, 5, 9])), n_symbols=n_symbols)
+    toks = [bytes(t) for n in range(0, 5) for t in itertools.product(b"abcd", repeat=n)]
+    toks = [toks[i] for i in rng.permutation(len(toks))][:300] + [b"e", b"ae"]
+    vb, vo = vocab_from_strings(toks)
+    V = vo.size - 1
+    eos = int(rng.integers(V)) if seed % 2 else -1
+    table = build(P, vb, vo, eos_id=eos)
+    check_table(table, P, vb, vo, eos_id=eos, seed=seed)
+    B, cap = 40, 12
+    ws = cstr.cstr_pda_workspace_create(table, B)
+    states = rng.integers(0, P.n_states, size=B).astype(np.int32)
+    depth = rng.integers(0, 8, size=B).astype(np.int32)
+    stacks = rng.integers(0, n_symbols, size=(B, cap)).astype(np.int32)
+    emitted = 0
+    for t in range(12):
+        logits = normal_logits(61 + seed, t, range(B), V)
+        ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth, eos_id=eos)
+        emitted += int((ref["tokens"] >= 0).sum())
+        states, depth, stacks = ref["states"], ref["depth"], ref["stacks_full"]
+        if t % 4 == 3:                                  # revive finished rows somewhere else
+            done = states < 0
+            states = np.where(done, rng.integers(0, P.n_states, size=B), states).astype(np.int32)
+    assert emitted > 20
