@@ -359,3 +359,40 @@ def test_inactive_rows_overflow_and_eos_by_hand():
     assert list(np.isneginf(m[2])) == [True, False, False, True, True]
     assert list(np.isneginf(m[6])) == [True, True, True, True, False]   # only EOS in "done"
     assert list(res["accept"]) == [0, 0, 1, 0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_pdas_allowed_set_and_traversal_against_direct_walk(seed):
+    # multi-symbol pushes, edges that push back what they popped, pops reaching several
+    # symbols down: the composed edges must agree with running the bytes one by one
+    from synth import random_pda
+    rng = np.random.default_rng(100 + seed)
+    P = random_pda(seed, n_states=int(rng.choice([3, 6])), n_symbols=int(rng.choice([1, 2, 3])))
+    toks = [bytes(t) for n in range(0, 5) for t in itertools.product(b"abcd", repeat=n)]
+    toks = [toks[i] for i in rng.permutation(len(toks))][:120]
+    vb, vo = vocab_from_strings(toks)
+    V = vo.size - 1
+    edges = edge_index(P)
+    states = rng.integers(0, P.n_states, size=10)
+    stacks = [list(rng.integers(0, P.n_symbols, size=int(rng.integers(0, 6)))) for _ in range(10)]
+    got = op.allowed(P, vb, vo, states, stacks)
+    for i in range(10):
+        want = py_allowed(P, vb, vo, int(states[i]), [int(x) for x in stacks[i]])
+        assert np.array_equal(bits(got[i], V), want)
+    cap = 16
+    sk = np.zeros((10, cap), dtype=np.int32)
+    dp = np.array([len(s) for s in stacks], dtype=np.int32)
+    for i, s in enumerate(stacks):
+        sk[i, :len(s)] = s
+    logits = normal_logits(5, seed, range(10), V)
+    res = op.step(P, vb, vo, logits, states.astype(np.int32), sk, dp)
+    for i in range(10):
+        tok = int(res["tokens"][i])
+        if tok < 0:
+            assert not bits(got[i], V).any()
+            continue
+        q2, s2 = py_walk(P, edges, int(states[i]), [int(x) for x in stacks[i]], toks[tok])
+        if len(s2) > cap:
+            assert res["states"][i] == -1
+        else:
+            assert res["states"][i] == q2 and list(res["stacks"][i, :res["depth"][i]]) == s2
