@@ -21,3 +21,4 @@ from .regex_frontend import regex_to_dfa  # noqa: F401
 from .configs import CONFIGS, get_config  # noqa: F401
 from .pda import (Pda, PdaBuilder, anbn_pda, dyck_pda, json_pda, random_pda,  # noqa: F401
                   stackless_pda)
+from .grammar import GrammarError, anbn_grammar_pda, grammar_to_pda, json_grammar_pda  # noqa: F401

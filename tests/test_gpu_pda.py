@@ -323,3 +323,28 @@ def test_random_pdas_table_and_decode_loop(seed):
             done = states < 0
             states = np.where(done, rng.integers(0, P.n_states, size=B), states).astype(np.int32)
     assert emitted > 20
+
+
+def test_grammar_built_json_pda():
+    # the bracketed-grammar front-end's nested-JSON PDA (one stack symbol per call site)
+    from synth import json_grammar_pda
+    P = json_grammar_pda()
+    vb, vo = make_vocab_json(3000, seed=4)
+    V = vo.size - 1
+    toks = [bytes(vb[vo[v]:vo[v + 1]]) for v in range(V)]
+    table = build(P, vb, vo)
+    rng = np.random.default_rng(2)
+    assert check_table(table, P, vb, vo, states=rng.choice(P.n_states, size=12, replace=False)) > 0
+    B, cap = 32, 6
+    ws = cstr.cstr_pda_workspace_create(table, B)
+    states = np.full(B, P.start, dtype=np.int32)
+    stacks = np.zeros((B, cap), dtype=np.int32)
+    depth = np.zeros(B, dtype=np.int32)
+    for t in range(24):
+        logits = normal_logits(71, t, range(B), V)
+        for name, bonus in ((b"[", 5.0), (b"[[", 5.0), (b"]]", 6.0), (b"]", 4.0), (b'"', 4.0),
+                            (b"}", 4.0), (b"{", 3.0), (b"1]", 5.0), (b", ", 4.0), (b"1", 4.0)):
+            logits[:, toks.index(name)] += np.float32(bonus)
+        ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth)
+        states, depth, stacks = ref["states"], ref["depth"], ref["stacks_full"]
+    assert depth.max() >= 2

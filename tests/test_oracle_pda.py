@@ -396,3 +396,47 @@ def test_random_pdas_allowed_set_and_traversal_against_direct_walk(seed):
             assert res["states"][i] == -1
         else:
             assert res["states"][i] == q2 and list(res["stacks"][i, :res["depth"][i]]) == s2
+
+
+# ------------------------------------------------ grammar front-end (input generator)
+
+def test_bracketed_grammar_front_end():
+    # The PDAs it builds are inputs of both sides; here they are checked as languages:
+    # Figure 4's grammar against the closed form, nested JSON against the json module and
+    # against the hand-built PDA, and ambiguous grammars are refused.
+    from synth import GrammarError, anbn_grammar_pda, grammar_to_pda, json_grammar_pda
+    P = anbn_grammar_pda()
+    words = list(all_words(b"abc", 9))
+    assert np.array_equal(op.accepts(P, words, threads=4),
+                          np.array([is_anbn(w) for w in words], dtype=np.uint8))
+    assert all(P.pop_off[j + 1] - P.pop_off[j] <= 1 and P.push_off[j + 1] - P.push_off[j] <= 1
+               for j in range(P.n_edges))
+
+    def deterministic(A):          # at most one edge per (state, byte, popped symbol or none)
+        keys = [(int(A.src[j]), int(A.inp[j]), tuple(A.pops[A.pop_off[j]:A.pop_off[j + 1]]))
+                for j in range(A.n_edges)]
+        plain = {k[:2] for k in keys if not k[2]}
+        return len(set(keys)) == len(keys) and not any(k[:2] in plain for k in keys if k[2])
+    assert deterministic(P) and deterministic(json_grammar_pda())
+    J, H = json_grammar_pda(), json_pda(space=True)
+    words = list(all_words(b'[]{}"a:, 1', 6)) + list(all_words(b"[]-01,tru", 6))
+    got = op.accepts(J, words, threads=8)
+    assert np.array_equal(got, op.accepts(H, words, threads=8))
+
+    def valid(w):
+        if w[:1] not in (b"[", b"{"):
+            return False
+        try:
+            json.loads(w.decode("ascii"))
+            return b" " not in w        # blanks are only allowed after ':' and ',' here
+        except ValueError:
+            return False
+    no_blank = [i for i, w in enumerate(words) if b" " not in w]
+    assert all(bool(got[i]) == valid(words[i]) for i in no_blank)
+    assert got.sum() > 100
+    with pytest.raises(GrammarError):            # a byte edge and a call start with the same byte
+        grammar_to_pda(r"<B>|\(x", {}, {"B": ("(", "y", ")")})
+    with pytest.raises(GrammarError):            # the body may read its own closing byte
+        grammar_to_pda(r"<B>", {}, {"B": ("(", r"[a)]*", ")")})
+    with pytest.raises(GrammarError):            # recursion outside a bracket
+        grammar_to_pda(r"<m>", {"m": "a<m>?"}, {})
