@@ -315,6 +315,15 @@ int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *vocab, int32
                          void *cuda_stream, cstr_pda_table_t **out);
 void cstr_free_pda_table(cstr_pda_table_t *table);
 
+/*
+ * Build the same token-level PDA again into the table's existing storage, with
+ * a (possibly different) end-of-sequence token: the compile step of Algorithm 3
+ * without any allocation or host synchronisation, only kernels enqueued on
+ * cuda_stream.  The table must not be in use by a cstr_pda_step that has not
+ * completed.
+ */
+int cstr_pda_table_rebuild(cstr_pda_table_t *table, int32_t eos_id, void *cuda_stream);
+
 /* Shape of a token-level PDA (any pointer may be NULL). */
 int cstr_pda_table_info(const cstr_pda_table_t *table, int32_t *n_states, int32_t *n_symbols,
                         int32_t *vocab_size, int32_t *mask_words, int32_t *start_state);

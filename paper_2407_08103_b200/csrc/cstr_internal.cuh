@@ -171,6 +171,10 @@ struct cstr_pda_table {
     uint32_t *mask;      // DEVICE [n_cfg][ldw]
     uint32_t *deep;      // DEVICE [n_cfg][ldw]
     uint32_t *ndeep;     // DEVICE [n_cfg]
+    // builder scratch, per state: tokens allowed whatever the stack holds, and
+    // tokens whose walk looks at the top of the stack
+    uint32_t *base;      // DEVICE [n_states][ldw]
+    uint32_t *need;      // DEVICE [n_states][ldw]
 };
 
 struct cstr_pda_workspace {

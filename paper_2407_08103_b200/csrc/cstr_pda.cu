@@ -27,21 +27,23 @@ namespace {
 
 using namespace cstr_pda_dev;
 
-// One warp per (situation, 32-token word): lane = token.
+// The table is built in two passes.  Most walks never look at the stack, so a
+// first pass decides every (state, token) pair with the top of the stack
+// unknown: allowed whatever the stack holds, dead, or "looks at the top".  The
+// second pass fills the rows of the situations (state, top): it copies the
+// state's stack-independent bits and walks only the tokens of the third kind,
+// now with the top known.  One warp per 32-token word, lane = token.
 __global__ void __launch_bounds__(256)
-pda_build_kernel(cstr_pda_view P, const uint8_t *__restrict__ accept, const uint8_t *__restrict__ vbytes,
-                 const uint32_t *__restrict__ voff, int V, int W, long long ldw, int eos_id,
-                 uint32_t *__restrict__ mask, uint32_t *__restrict__ deep,
-                 uint32_t *__restrict__ ndeep)
+pda_state_pass_kernel(cstr_pda_view P, const uint8_t *__restrict__ accept,
+                      const uint8_t *__restrict__ vbytes, const uint32_t *__restrict__ voff, int V,
+                      int W, long long ldw, int eos_id, uint32_t *__restrict__ base,
+                      uint32_t *__restrict__ need)
 {
     const int lane = threadIdx.x & 31;
     const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int cfg = blockIdx.y;
+    const int q = blockIdx.y;
     if (w >= W)
         return;
-    const int q = cfg / (P.n_symbols + 1);
-    const int top = cfg - q * (P.n_symbols + 1);   // n_symbols = empty stack
-    const bool has_top = top < P.n_symbols;
     const int v = w * 32 + lane;
     int res = WALK_DEAD;
     if (v < V) {
@@ -51,18 +53,64 @@ pda_build_kernel(cstr_pda_view P, const uint8_t *__restrict__ accept, const uint
             uint8_t loc[kLocMax];
             int q2, cd2, nloc2;
             const uint32_t b = voff[v], e = voff[v + 1];
-            res = pda_walk(P, q, nullptr, top, has_top ? 1 : 0, has_top, vbytes + b, (int)(e - b),
-                           loc, q2, cd2, nloc2);
+            res = pda_walk(P, q, nullptr, 0, 0, true, vbytes + b, (int)(e - b), loc, q2, cd2, nloc2);
         }
     }
     const unsigned ok = __ballot_sync(0xffffffffu, res == WALK_OK);
-    const unsigned dp = __ballot_sync(0xffffffffu, res == WALK_DEEP);
+    const unsigned nd = __ballot_sync(0xffffffffu, res == WALK_DEEP);
     if (lane == 0) {
-        mask[(long long)cfg * ldw + w] = ok;
-        deep[(long long)cfg * ldw + w] = dp;
-        if (dp)
-            atomicAdd(ndeep + cfg, (uint32_t)__popc(dp));
+        base[(long long)q * ldw + w] = ok;
+        need[(long long)q * ldw + w] = nd;
     }
+}
+
+// One warp per 32 consecutive words of a situation's rows: lane = word for the
+// (coalesced) copy; for the few words that hold top-dependent tokens the whole
+// warp walks that word's tokens, lane = token.
+__global__ void __launch_bounds__(256)
+pda_situation_pass_kernel(cstr_pda_view P, const uint8_t *__restrict__ vbytes,
+                          const uint32_t *__restrict__ voff, long long ldw,
+                          const uint32_t *__restrict__ base, const uint32_t *__restrict__ need,
+                          uint32_t *__restrict__ mask, uint32_t *__restrict__ deep,
+                          uint32_t *__restrict__ ndeep)
+{
+    const int lane = threadIdx.x & 31;
+    const long long w0 = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32;
+    const int cfg = blockIdx.y;
+    if (w0 >= ldw)
+        return;                                     // ldw is a multiple of 32: whole groups
+    const int q = cfg / (P.n_symbols + 1);
+    const int top = cfg - q * (P.n_symbols + 1);    // n_symbols = empty stack
+    const bool has_top = top < P.n_symbols;
+    unsigned ok = base[(long long)q * ldw + w0 + lane];
+    const unsigned nd = need[(long long)q * ldw + w0 + lane];
+    unsigned dp = 0u;
+    unsigned pending = __ballot_sync(0xffffffffu, nd != 0u);
+    while (pending) {                               // warp-uniform
+        const int src = __ffs((int)pending) - 1;
+        pending &= pending - 1;
+        const unsigned word_nd = __shfl_sync(0xffffffffu, nd, src);
+        int res = WALK_DEAD;
+        if ((word_nd >> lane) & 1u) {
+            const int v = (int)(w0 + src) * 32 + lane;
+            uint8_t loc[kLocMax];
+            int q2, cd2, nloc2;
+            const uint32_t b = voff[v], e = voff[v + 1];
+            res = pda_walk(P, q, nullptr, top, has_top ? 1 : 0, has_top, vbytes + b, (int)(e - b),
+                           loc, q2, cd2, nloc2);
+        }
+        const unsigned got_ok = __ballot_sync(0xffffffffu, res == WALK_OK);
+        const unsigned got_dp = __ballot_sync(0xffffffffu, res == WALK_DEEP);
+        if (lane == src) {
+            ok |= got_ok;
+            dp = got_dp;
+        }
+    }
+    mask[(long long)cfg * ldw + w0 + lane] = ok;
+    deep[(long long)cfg * ldw + w0 + lane] = dp;
+    const unsigned total = __reduce_add_sync(0xffffffffu, (unsigned)__popc(dp));
+    if (lane == 0 && total)
+        atomicAdd(ndeep + cfg, total);
 }
 
 // What the prepare kernel reads: the rows' situations and the table.
@@ -330,7 +378,46 @@ extern "C" void cstr_free_pda_table(cstr_pda_table_t *t)
     cudaFree(t->mask);
     cudaFree(t->deep);
     cudaFree(t->ndeep);
+    cudaFree(t->base);
+    cudaFree(t->need);
     delete t;
+}
+
+// The two build passes into a table's existing storage (every word of the
+// situation rows is rewritten; only the per-situation counts need clearing).
+static cudaError_t enqueue_pda_build(cstr_pda_table *t, cudaStream_t stream)
+{
+    const cstr_pda *pda = t->pda;
+    const cstr_vocab *vocab = t->vocab;
+    cudaError_t e = cudaMemsetAsync(t->ndeep, 0, (size_t)t->n_cfg * 4, stream);
+    if (e != cudaSuccess)
+        return e;
+    cstr_pda_view P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
+    const int warps = 8;
+    const unsigned gx = (unsigned)((t->W + warps - 1) / warps);
+    pda_state_pass_kernel<<<dim3(gx, (unsigned)pda->n_states), warps * 32, 0, stream>>>(
+        P, pda->accept, vocab->bytes, vocab->off, t->V, t->W, t->ldw, t->eos_id, t->base, t->need);
+    const unsigned gx2 = (unsigned)((t->ldw / 32 + warps - 1) / warps);
+    pda_situation_pass_kernel<<<dim3(gx2, (unsigned)t->n_cfg), warps * 32, 0, stream>>>(
+        P, vocab->bytes, vocab->off, t->ldw, t->base, t->need, t->mask, t->deep, t->ndeep);
+    return cudaGetLastError();
+}
+
+extern "C" int cstr_pda_table_rebuild(cstr_pda_table_t *t, int32_t eos_id, void *cuda_stream)
+{
+    if (!t)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_table_rebuild: null table");
+    int rc = check_device(t->device, "PDA table");
+    if (rc)
+        return rc;
+    if (eos_id < -1 || eos_id >= t->V)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_table_rebuild: eos_id %d outside [-1, %d)", eos_id,
+                         t->V);
+    t->eos_id = eos_id;
+    const cudaError_t e = enqueue_pda_build(t, (cudaStream_t)cuda_stream);
+    if (e != cudaSuccess)
+        return cuda_rc(e, "cstr_pda_table_rebuild");
+    return CSTR_OK;
 }
 
 extern "C" int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *vocab,
@@ -377,21 +464,17 @@ extern "C" int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *v
         e = cudaMalloc((void **)&t->deep, row_bytes);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->ndeep, (size_t)n_cfg * 4);
+    const size_t state_bytes = (size_t)pda->n_states * (size_t)t->ldw * 4;
     if (e == cudaSuccess)
-        e = cudaMemsetAsync(t->mask, 0, row_bytes, stream);
+        e = cudaMalloc((void **)&t->base, state_bytes);
     if (e == cudaSuccess)
-        e = cudaMemsetAsync(t->deep, 0, row_bytes, stream);
+        e = cudaMalloc((void **)&t->need, state_bytes);
     if (e == cudaSuccess)
-        e = cudaMemsetAsync(t->ndeep, 0, (size_t)n_cfg * 4, stream);
-    if (e == cudaSuccess) {
-        cstr_pda_view P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
-        const int warps = 8;
-        dim3 grid((unsigned)((t->W + warps - 1) / warps), (unsigned)n_cfg);
-        pda_build_kernel<<<grid, warps * 32, 0, stream>>>(P, pda->accept, vocab->bytes, vocab->off,
-                                                          t->V, t->W, t->ldw, eos_id, t->mask,
-                                                          t->deep, t->ndeep);
-        e = cudaGetLastError();
-    }
+        e = cudaMemsetAsync(t->base, 0, state_bytes, stream);   // padding words stay zero
+    if (e == cudaSuccess)
+        e = cudaMemsetAsync(t->need, 0, state_bytes, stream);
+    if (e == cudaSuccess)
+        e = enqueue_pda_build(t, stream);
     if (e != cudaSuccess) {
         rc = cuda_rc(e, "cstr_build_pda_table");
         cstr_free_pda_table(t);

@@ -28,7 +28,8 @@ EXPORTS = [
     "cstr_step", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
     "cstr_step_static", "cstr_last_error",
     "cstr_load_pda", "cstr_free_pda", "cstr_build_pda_table", "cstr_free_pda_table",
-    "cstr_pda_table_info", "cstr_pda_table_download", "cstr_pda_workspace_create",
+    "cstr_pda_table_rebuild", "cstr_pda_table_info", "cstr_pda_table_download",
+    "cstr_pda_workspace_create",
     "cstr_free_pda_workspace", "cstr_pda_step", "cstr_pda_step_status",
 ]
 
@@ -361,6 +362,10 @@ def cstr_build_pda_table(pda: Pda, vocab: Vocab, eos_id: int = -1, stream=None) 
     t = PdaTable(out)
     t.pda, t.vocab = pda, vocab
     return t
+
+
+def cstr_pda_table_rebuild(table: PdaTable, eos_id: int = -1, stream=None) -> None:
+    _check(lib().cstr_pda_table_rebuild(table.ptr, ctypes.c_int32(eos_id), _stream_ptr(stream)))
 
 
 def cstr_pda_table_info(table: PdaTable):

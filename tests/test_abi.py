@@ -83,6 +83,7 @@ def test_null_and_range_errors(lib):
     assert b"no epsilon input" in lib.cstr_last_error()
     assert lib.cstr_build_pda_table(None, None, -1, None, ctypes.byref(out)) == -1
     assert lib.cstr_pda_table_info(None, None, None, None, None, None) == -1
+    assert lib.cstr_pda_table_rebuild(None, -1, None) == -1
     assert lib.cstr_pda_table_download(None, 0, 0, None, None, None) == -1
     assert lib.cstr_pda_workspace_create(None, 4, ctypes.byref(out)) == -1
     assert lib.cstr_pda_step(None, None, 0, 0, None, None, None, None, 4, None, None, None, 1,

@@ -119,6 +119,12 @@ def test_table_dyck_and_eos():
     vb, vo = make_vocab_json(1500, seed=3)
     table = build(P, vb, vo, eos_id=77)
     check_table(table, P, vb, vo, eos_id=77)
+    cstr.cstr_pda_table_rebuild(table, -1)             # same storage, no EOS token
+    torch.cuda.synchronize()
+    check_table(table, P, vb, vo)
+    cstr.cstr_pda_table_rebuild(table, 3)
+    torch.cuda.synchronize()
+    check_table(table, P, vb, vo, eos_id=3)
 
 
 def test_table_json_small_vocab_all_situations():
