@@ -70,7 +70,8 @@ typedef struct cstr_pda_workspace cstr_pda_workspace_t; /* per-stream scratch of
  * Validates every target, merges bytes that no state tells apart into
  * classes, and copies the class-major table to the device (16-bit entries up
  * to 32766 states, else 32-bit); returns the handle in *out.
- * Synchronous; allocates device memory.
+ * Synchronous; allocates device memory.  Each host thread keeps the device
+ * scratch of its last load (the raw table, at most 64 MB) for the next one.
  */
 int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
                   int32_t start_state, cstr_dfa_t **out);

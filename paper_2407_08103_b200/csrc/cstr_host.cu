@@ -38,7 +38,8 @@ static int check_device(int handle_device, const char *what)
 namespace {
 
 // Two order-independent 64-bit hashes per byte column of the raw table
-// (thread = byte, a block sums a slab of rows, slabs combine with atomicAdd).
+// (thread = byte, a block sums a slab of rows, slabs combine with atomicAdd);
+// the same pass checks that every target is a state or -1.
 __global__ void __launch_bounds__(256)
 dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_per_block,
                        unsigned long long *__restrict__ hashes)
@@ -47,8 +48,11 @@ dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_p
     const int q0 = blockIdx.x * rows_per_block;
     const int q1 = min(n_states, q0 + rows_per_block);
     unsigned long long h1 = 0, h2 = 0;
+    bool invalid = false;                    // a target outside [-1, n_states): hashes[513] != 0
     for (int q = q0; q < q1; ++q) {
-        unsigned long long x = (unsigned long long)(unsigned)raw[(long long)q * 256 + b] +
+        const int32_t target = raw[(long long)q * 256 + b];
+        invalid |= target < -1 || target >= n_states;
+        unsigned long long x = (unsigned long long)(unsigned)target +
                                ((unsigned long long)(unsigned)q << 32) + 0x9e3779b97f4a7c15ull;
         x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;        // splitmix64 finaliser: (q, value) -> 64 bits
         x ^= x >> 27; x *= 0x94d049bb133111ebull;
@@ -58,6 +62,8 @@ dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_p
     }
     atomicAdd(hashes + b, h1);
     atomicAdd(hashes + 256 + b, h2);
+    if (invalid)
+        atomicOr(hashes + 513, 1ull);
 }
 
 // Class-major code table from the raw table, proving the proposed classes on
@@ -100,13 +106,80 @@ dfa_build_table_kernel(const int32_t *__restrict__ raw, int n_states, int row, i
 }  // namespace
 
 
+// Host scan for the first target outside [-1, n_states): sets the error text and
+// returns CSTR_ERR_DFA, or 0 if the table is well formed.
+static int first_bad_target(const int32_t *trans, int32_t n_states)
+{
+    const int64_t n = (int64_t)n_states * 256;
+    int bad = 0;                   // branch-free so that the scan vectorises
+    for (int64_t i = 0; i < n; ++i)
+        bad |= (trans[i] < -1) | (trans[i] >= n_states);
+    if (!bad)
+        return 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (trans[i] < -1 || trans[i] >= n_states)
+            return cstr_fail(CSTR_ERR_DFA,
+                             "cstr_load_dfa: state %lld byte %lld has target %d outside [-1, %d)",
+                             (long long)(i / 256), (long long)(i % 256), trans[i], n_states);
+    }
+    return 0;
+}
+
+// Device scratch of cstr_load_dfa (the raw table and a few flags).  Allocating
+// and freeing it cost more than the load's kernels, so each host thread keeps
+// one block per process (at most kScratchKeep bytes, on the device it was last
+// used on); larger requests are allocated and freed per call.
+namespace {
+constexpr size_t kScratchKeep = 64u << 20;
+struct ScratchCache {
+    int device = -1;
+    unsigned char *ptr = nullptr;
+    size_t bytes = 0;
+};
+thread_local ScratchCache t_scratch;
+
+cudaError_t scratch_acquire(int device, size_t bytes, unsigned char **out, bool *cached)
+{
+    *cached = false;
+    if (bytes > kScratchKeep)
+        return cudaMalloc((void **)out, bytes);
+    ScratchCache &c = t_scratch;
+    if (c.ptr && (c.device != device || c.bytes < bytes)) {
+        int cur = -1;                            // free on the device that owns the block
+        cudaGetDevice(&cur);
+        cudaSetDevice(c.device);
+        cudaFree(c.ptr);
+        cudaSetDevice(cur);
+        c.ptr = nullptr;
+        c.bytes = 0;
+    }
+    if (!c.ptr) {
+        cudaError_t e = cudaMalloc((void **)&c.ptr, bytes);
+        if (e != cudaSuccess) {
+            c.ptr = nullptr;
+            return e;
+        }
+        c.device = device;
+        c.bytes = bytes;
+    }
+    *out = c.ptr;
+    *cached = true;
+    return cudaSuccess;
+}
+
+void scratch_release(unsigned char *ptr, bool cached)
+{
+    if (!cached)
+        cudaFree(ptr);
+}
+}  // namespace
+
 extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
 {
     if (!dfa)
         return;
     cudaFree(dfa->tt);
-    cudaFree(dfa->cls);
-    cudaFree(dfa->accept);
+    cudaFree(dfa->cls);                  // one allocation: byte classes, then the accept flags
     cudaFree(dfa->tstate);
     cudaFree(dfa->tset);
     cudaFree(dfa->ttarget);
@@ -128,17 +201,6 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
         return cstr_fail(CSTR_ERR_ARG, "cstr_load_dfa: start_state %d outside [0, %d)",
                          start_state, n_states);
     const int64_t n = (int64_t)n_states * 256;
-    int bad = 0;                   // branch-free so that the scan vectorises
-    for (int64_t i = 0; i < n; ++i)
-        bad |= (trans[i] < -1) | (trans[i] >= n_states);
-    if (bad) {
-        for (int64_t i = 0; i < n; ++i) {
-            if (trans[i] < -1 || trans[i] >= n_states)
-                return cstr_fail(CSTR_ERR_DFA,
-                                 "cstr_load_dfa: state %lld byte %lld has target %d outside [-1, %d)",
-                                 (long long)(i / 256), (long long)(i % 256), trans[i], n_states);
-        }
-    }
     cstr_dfa *d = new (std::nothrow) cstr_dfa();
     if (!d)
         return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
@@ -149,11 +211,12 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     d->row = ((int64_t)n_states + 1 + 255) / 256 * 256;
     const size_t esz = d->wide ? 4 : 2;
 
-    // The raw table goes to the device once; byte classes (bytes whose columns
-    // are identical in every state) and the class-major code table are made
-    // there: column hashes propose the classes, a second kernel proves them
-    // entry by entry while it writes the table, and only a hash collision (never
-    // seen) falls back to exact column comparisons on the host.
+    // The raw table goes to the device once; validation, byte classes (bytes whose
+    // columns are identical in every state) and the class-major code table are
+    // made there: one pass checks the targets and hashes the columns, the hashes
+    // propose the classes, a second kernel proves them entry by entry while it
+    // writes the table, and only a hash collision (never seen) falls back to
+    // exact column comparisons on the host.
     std::vector<uint8_t> flags;
     try {
         flags.resize(n_states);
@@ -164,27 +227,34 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     for (int32_t q = 0; q < n_states; ++q)
         flags[q] = accept[q] ? 1 : 0;
 
-    int32_t *raw = nullptr;
-    unsigned long long *hashes = nullptr;     // [2][256], then one mismatch flag
-    uint8_t *rep_dev = nullptr;
+    // temporaries in one block: [raw table][2 x 256 hashes, mismatch flag, invalid flag][256 reps]
+    const size_t raw_bytes = (size_t)n * 4, hash_bytes = 514 * 8;
     cudaError_t e = cudaGetDevice(&d->device);
+    unsigned char *temp = nullptr;
+    bool temp_cached = false;
     if (e == cudaSuccess)
-        e = cudaMalloc((void **)&raw, (size_t)n * 4);
+        e = scratch_acquire(d->device, raw_bytes + hash_bytes + 256, &temp, &temp_cached);
+    if (e != cudaSuccess) {
+        // No usable device: still tell the caller about a malformed table first.
+        const int rc_dfa = first_bad_target(trans, n_states);
+        const int rc = rc_dfa ? rc_dfa
+                              : cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                                          "cstr_load_dfa: %s", cudaGetErrorString(e));
+        delete d;
+        return rc;
+    }
+    int32_t *raw = (int32_t *)temp;
+    unsigned long long *hashes = (unsigned long long *)(temp + raw_bytes);
+    uint8_t *rep_dev = temp + raw_bytes + hash_bytes;
+    e = cudaMalloc((void **)&d->cls, 256 + (size_t)n_states);
+    d->accept = d->cls ? d->cls + 256 : nullptr;
     if (e == cudaSuccess)
-        e = cudaMalloc((void **)&hashes, 513 * 8);
-    if (e == cudaSuccess)
-        e = cudaMalloc((void **)&rep_dev, 256);
-    if (e == cudaSuccess)
-        e = cudaMalloc((void **)&d->cls, 256);
-    if (e == cudaSuccess)
-        e = cudaMalloc((void **)&d->accept, (size_t)n_states);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(raw, trans, (size_t)n * 4, cudaMemcpyHostToDevice);
+        e = cudaMemcpy(raw, trans, raw_bytes, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemcpy(d->accept, flags.data(), (size_t)n_states, cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
-        e = cudaMemset(hashes, 0, 513 * 8);
-    unsigned long long host_hash[513];
+        e = cudaMemset(hashes, 0, hash_bytes);
+    unsigned long long host_hash[514];
     if (e == cudaSuccess) {
         const int rows_per_block = 64;
         dfa_column_hash_kernel<<<(n_states + rows_per_block - 1) / rows_per_block, 256>>>(
@@ -192,7 +262,14 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
         e = cudaGetLastError();
     }
     if (e == cudaSuccess)
-        e = cudaMemcpy(host_hash, hashes, 512 * 8, cudaMemcpyDeviceToHost);
+        e = cudaMemcpy(host_hash, hashes, hash_bytes, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && host_hash[513] != 0) {       // some target is out of range: say which
+        scratch_release(temp, temp_cached);
+        cstr_free_dfa(d);
+        const int rc = first_bad_target(trans, n_states);
+        return rc ? rc : cstr_fail(CSTR_ERR_DFA, "cstr_load_dfa: a target is outside [-1, %d)",
+                                   n_states);
+    }
 
     uint8_t cls8[256], rep8[256];
     int n_classes = 0;
@@ -242,9 +319,7 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
             break;                               // proven (or failed): no second attempt
         e = cudaMemset(hashes + 512, 0, 8);      // a collision: redo with exact classes
     }
-    cudaFree(raw);
-    cudaFree(hashes);
-    cudaFree(rep_dev);
+    scratch_release(temp, temp_cached);
     if (e != cudaSuccess) {
         int rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
                            "cstr_load_dfa: %s", cudaGetErrorString(e));

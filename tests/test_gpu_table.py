@@ -229,3 +229,24 @@ def test_duplicate_column_pass_wide_entries_and_table_reuse():
     cstr.cstr_table_build(table, cstr.cstr_load_dfa(*wide), 300)      # and back, with an EOS token
     torch.cuda.synchronize()
     check_table(table, wide, vb, vo, eos_id=300, states=[0, 77, S - 1])
+
+
+def test_load_dfa_reports_bad_targets_and_reuses_its_scratch():
+    # the target check runs on the device; the message still names the first bad entry,
+    # and loads of different sizes in a row (the per-thread scratch shrinks and grows) stay exact
+    trans = np.full((300, 256), -1, dtype=np.int32)
+    acc = np.zeros(300, dtype=np.uint8)
+    trans[299, 255] = 300
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_load_dfa(trans, acc, 0)
+    assert e.value.code == -3 and "state 299 byte 255" in str(e.value)
+    trans[299, 255] = -2
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_load_dfa(trans, acc, 0)
+    assert e.value.code == -3
+    rng = np.random.default_rng(8)
+    vb, vo = random_vocab(rng, 700)
+    for S in (5, 900, 40, 2000, 3):
+        dfa = dense_random_dfa(rng, S, live=0.8)
+        (table,) = gpu_tables([dfa], vb, vo)
+        check_table(table, dfa, vb, vo, states=sorted(set([0, S // 2, S - 1])))
