@@ -68,3 +68,22 @@ def test_workloads_and_models():
     assert np.array_equal(t, target_logits(3, 0, [4, 5], 500))
     d = draft_logits(3, 0, [4, 5], 500)
     assert not np.array_equal(t, d) and np.corrcoef(t, d)[0, 1] > 0.7
+
+
+def test_pushdown_inputs_are_seeded_and_well_formed():
+    from synth import json_grammar_pda, json_pda, make_vocab_json, random_pda
+    vb, vo = make_vocab_json(5000, seed=3)
+    vb2, vo2 = make_vocab_json(5000, seed=3)
+    assert np.array_equal(vb, vb2) and np.array_equal(vo, vo2)
+    toks = [bytes(vb[vo[v]:vo[v + 1]]) for v in range(vo.size - 1)]
+    assert toks[:256] == [bytes([c]) for c in range(256)]
+    assert b"]]" in toks and b'{"' in toks and b"" in toks and len(toks) == 5000
+    for P in (json_pda(), json_grammar_pda(), random_pda(5), random_pda(5)):
+        n = P.n_edges
+        assert P.pop_off.size == n + 1 and P.push_off.size == n + 1
+        assert P.pop_off[-1] == P.pops.size and P.push_off[-1] == P.pushes.size
+        assert P.src.min() >= 0 and P.src.max() < P.n_states and P.tgt.max() < P.n_states
+        assert (P.pops < P.n_symbols).all() and (P.pushes < P.n_symbols).all()
+        assert np.diff(P.pop_off).max() <= 1 and np.diff(P.push_off).max() <= 3
+    a, b = random_pda(5), random_pda(5)
+    assert np.array_equal(a.src, b.src) and np.array_equal(a.pushes, b.pushes)
