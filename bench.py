@@ -290,8 +290,8 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
     # and as one CUDA graph of 32 steps (cstr_step only enqueues kernels, so a
     # sampling loop can be captured): removes the host launch cost that
     # dominates the small workloads
-    graph_ms = None
-    try:
+    def graph_time(rotate):
+        """32 steps per graph; rotate=False keeps one logits tensor (L2-resident when it fits)."""
         side = torch.cuda.Stream(device=dev)
         side.wait_stream(stream)
         g = torch.cuda.CUDAGraph()
@@ -299,7 +299,8 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
             dec.step(pool[0], noise=None if noise is None else noise[0], masked_out=out[0])
             with torch.cuda.graph(g, stream=side):
                 for i in range(32):
-                    dec.step(pool[i % pool_n], noise=None if noise is None else noise[i % len(noise)],
+                    k = i % pool_n if rotate else 0
+                    dec.step(pool[k], noise=None if noise is None else noise[k % len(noise)],
                              masked_out=out[i & 1])
                     torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
             g.replay()
@@ -309,10 +310,14 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
                 g.replay()
             g1.record(side)
             g1.synchronize()
-            graph_ms = g0.elapsed_time(g1) / (8 * 32)
         stream.wait_stream(side)
+        return g0.elapsed_time(g1) / (8 * 32)
+
+    graph_ms = graph_resident_ms = None
+    try:
+        graph_ms = graph_time(True)
+        graph_resident_ms = graph_time(False)
     except Exception as exc:  # pragma: no cover - depends on the box
-        graph_ms = None
         sys.stderr.write("graph timing of %s skipped: %r\n" % (name, exc))
     bytes_per_logit = 2 * esz + (4 if w.gumbel else 0) + 1.0 / 8.0
     step_bytes = B * V * bytes_per_logit
@@ -325,7 +330,7 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
         "workload": name, "vocab": V, "batch": B, "dfa_states": [int(d[0].shape[0]) for d in dfas],
         "dtype": w.dtype, "sampler": "gumbel-max" if w.gumbel else "greedy",
         "tables": len(tables), "step_kernel_ms": kernel_ms, "step_loop_ms": loop_ms,
-        "step_graph_ms": graph_ms,
+        "step_graph_ms": graph_ms, "step_graph_ms_same_tensor": graph_resident_ms,
         "logits_per_s": B * V / (kernel_ms * 1e-3),
         "roofline": {"bound": "hbm" if hbm_honest else "launch latency (working set sits in L2)",
                      "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
