@@ -482,20 +482,42 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
         desc.resize((size_t)vocab_size);
         for (int32_t v = 0; v <= vocab_size; ++v)
             off32[v] = (uint32_t)offsets[v];
-        for (int32_t v = 0; v < vocab_size; ++v)
-            order[v] = v;
         // lexicographic order of the byte strings (a prefix sorts before its
-        // extensions), ties by id: the depth-first order of the vocabulary trie
-        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
-            const uint32_t la = off32[a + 1] - off32[a], lb = off32[b + 1] - off32[b];
-            const uint32_t m = la < lb ? la : lb;
-            const int c = m ? memcmp(vocab_bytes + off32[a], vocab_bytes + off32[b], m) : 0;
-            if (c != 0)
-                return c < 0;
+        // extensions), ties by id: the depth-first order of the vocabulary trie.
+        // Sort keys carry the first 8 bytes as a big-endian integer, so that most
+        // comparisons never touch the strings.
+        struct SortKey {
+            uint64_t head;
+            uint32_t len;
+            int32_t id;
+        };
+        std::vector<SortKey> keys((size_t)vocab_size);
+        for (int32_t v = 0; v < vocab_size; ++v) {
+            const uint32_t len = off32[v + 1] - off32[v];
+            uint64_t head = 0;
+            for (uint32_t k = 0; k < 8; ++k)
+                head = (head << 8) | (k < len ? (uint64_t)vocab_bytes[off32[v] + k] : 0u);
+            keys[v].head = head;
+            keys[v].len = len;
+            keys[v].id = v;
+        }
+        std::sort(keys.begin(), keys.end(), [&](const SortKey &x, const SortKey &y) {
+            if (x.head != y.head)
+                return x.head < y.head;
+            const int32_t a = x.id, b = y.id;
+            const uint32_t la = x.len, lb = y.len;
+            if (la > 8 && lb > 8) {              // equal first 8 bytes: compare the rest
+                const uint32_t m = (la < lb ? la : lb) - 8;
+                const int c = memcmp(vocab_bytes + off32[a] + 8, vocab_bytes + off32[b] + 8, m);
+                if (c != 0)
+                    return c < 0;
+            }
             if (la != lb)
                 return la < lb;
             return a < b;
         });
+        for (int32_t i = 0; i < vocab_size; ++i)
+            order[i] = keys[i].id;
         for (int32_t i = 0; i < vocab_size; ++i) {
             const int32_t v = order[i];
             const uint8_t *cur = vocab_bytes + off32[v];
