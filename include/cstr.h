@@ -372,6 +372,47 @@ int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dty
                   int32_t batch, cstr_pda_workspace_t *ws, void *cuda_stream);
 
 /*
+ * cstr_pda_step that leaves the rows' situations untouched and writes the new
+ * ones to separate arrays, so that a caller can keep the situation after every
+ * drafted token (Section 4, Speculative decoding: the constraint has to be able
+ * to go back to the situation that followed an earlier token - for a push-down
+ * constraint that is the state together with the stack).
+ *   states_in, stacks_in, depths_in     DEVICE, read only
+ *   states_out, stacks_out, depths_out  DEVICE, same shapes; either all three
+ *                                       equal to the inputs (then it is
+ *                                       cstr_pda_step) or all three different
+ * A row that finishes (new state -1) gets a copy of its old stack and depth.
+ * Everything else as in cstr_pda_step.  Over batch x (k + 1) rows holding the
+ * draft's history, one call penalises the target model's logits at all drafted
+ * positions and decodes the target's own token and next situation at each.
+ */
+int cstr_pda_step_history(const cstr_pda_table_t *table, const void *logits, int32_t dtype,
+                          int64_t ld, const float *noise, const int32_t *states_in,
+                          const int32_t *stacks_in, const int32_t *depths_in, int32_t *states_out,
+                          int32_t *stacks_out, int32_t *depths_out, int32_t stack_cap,
+                          int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
+                          int32_t batch, cstr_pda_workspace_t *ws, void *cuda_stream);
+
+/*
+ * Greedy verification and rewind for speculative decoding under a push-down
+ * constraint (Section 4): as cstr_accept_draft, and the rewound situation
+ * includes the stack.
+ *   draft_tokens   DEVICE int32 [batch][k]
+ *   target_tokens, target_states, target_depths   DEVICE int32 [batch][k + 1]
+ *   target_stacks  DEVICE int32 [batch][k + 1][stack_cap]
+ *   n_accepted     DEVICE int32 [batch]          n = drafted tokens kept
+ *   out_tokens     DEVICE int32 [batch][k + 1]   target_tokens[0..n], then -1
+ *   states, depths DEVICE int32 [batch];  stacks DEVICE int32 [batch][stack_cap]:
+ *                  the target's situation after its token at position n
+ * Only enqueues one small kernel.
+ */
+int cstr_pda_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,
+                          const int32_t *target_states, const int32_t *target_stacks,
+                          const int32_t *target_depths, int32_t k, int32_t batch,
+                          int32_t stack_cap, int32_t *n_accepted, int32_t *out_tokens,
+                          int32_t *states, int32_t *stacks, int32_t *depths, void *cuda_stream);
+
+/*
  * Rows since the last call that were inactive for another reason than state
  * -1, active rows without a selectable token, and rows that finished because
  * their stack outgrew stack_cap.  Synchronises cuda_stream, then resets the

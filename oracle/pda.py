@@ -170,3 +170,18 @@ def step(pda, vocab_bytes, offsets, logits, states, stacks, depth, noise=None, e
     return dict(tokens=tokens, states=st, stacks=sk, depth=dp, masked=masked, accept=acc_out,
                 bad_state_rows=int(counters[0]), empty_mask_rows=int(counters[1]),
                 overflow_rows=int(counters[2]))
+
+
+def accept_draft(draft_tokens, target_tokens, target_states, target_stacks, target_depths):
+    """Greedy verification and rewind under a push-down constraint (Section 4): the
+    kept prefix and the emitted tokens are those of the finite-state rule
+    (``oracle.accept_draft``); the constraint goes back to the whole situation
+    - state, stack and depth - that followed the last token kept.
+    ``target_stacks`` int32 ``[B][k+1][cap]``, the others ``[B][k+1]`` / ``[B][k]``.
+    Returns (n_accepted, out_tokens, states, stacks [B][cap], depths)."""
+    import oracle
+    n, out, states = oracle.accept_draft(draft_tokens, target_tokens, target_states)
+    target_stacks = np.asarray(target_stacks, dtype=np.int32)
+    target_depths = np.asarray(target_depths, dtype=np.int32)
+    rows = np.arange(n.size)
+    return n, out, states, target_stacks[rows, n].copy(), target_depths[rows, n].copy()

@@ -142,6 +142,9 @@ struct cstr_pda_advance {
     const uint8_t *vbytes;         // DEVICE vocabulary bytes
     const uint32_t *voff;          // DEVICE [V + 1]
     int32_t n_states, eos_id, cap;
+    // situation before the step (read) and after it (written); the two sets may
+    // be the same arrays (in-place update) or different ones (state history)
+    const int32_t *states_in, *stacks_in, *depths_in;
     int32_t *states, *stacks, *depths;   // DEVICE [batch], [batch][cap], [batch]
     uint8_t *accept_out;           // DEVICE [batch] or null
     unsigned long long *counters;  // DEVICE [3]: bad rows, rows without a token, overflows

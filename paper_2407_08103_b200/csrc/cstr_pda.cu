@@ -587,14 +587,19 @@ extern "C" int cstr_pda_workspace_create(const cstr_pda_table_t *table, int32_t 
 
 // ----------------------------------------------------------------- step
 
-extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dtype,
-                             int64_t ld, const float *noise, int32_t *states, int32_t *stacks,
-                             int32_t *depths, int32_t stack_cap, int32_t *tokens_out,
-                             void *masked_out, uint8_t *accept_out, int32_t batch,
-                             cstr_pda_workspace_t *ws, void *cuda_stream)
+static int pda_step_common(const cstr_pda_table_t *table, const void *logits, int32_t dtype,
+                           int64_t ld, const float *noise, const int32_t *states_in,
+                           const int32_t *stacks_in, const int32_t *depths_in, int32_t *states,
+                           int32_t *stacks, int32_t *depths, int32_t stack_cap, int32_t *tokens_out,
+                           void *masked_out, uint8_t *accept_out, int32_t batch,
+                           cstr_pda_workspace_t *ws, void *cuda_stream)
 {
-    if (!table || !logits || !states || !stacks || !depths || !tokens_out || !masked_out || !ws)
+    if (!table || !logits || !states || !stacks || !depths || !states_in || !stacks_in ||
+        !depths_in || !tokens_out || !masked_out || !ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_pda_step: null pointer");
+    if ((stacks_in == stacks) != (depths_in == depths) || (stacks_in == stacks) != (states_in == states))
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_step_history: states, stacks and depths must be "
+                         "either all updated in place or all written to separate arrays");
     if (dtype != CSTR_F32 && dtype != CSTR_BF16)
         return cstr_fail(CSTR_ERR_DTYPE, "cstr_pda_step: unknown dtype %d", dtype);
     if (batch < 0 || stack_cap < 1)
@@ -630,9 +635,9 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     p.ndeep = table->ndeep;
     p.ldw = table->ldw;
     p.n_states = pda->n_states;
-    p.states = states;
-    p.stacks = stacks;
-    p.depths = depths;
+    p.states = states_in;
+    p.stacks = stacks_in;
+    p.depths = depths_in;
     p.cap = stack_cap;
     p.row_mask = ws->row_mask;
     p.row_buf = ws->row_buf;
@@ -650,7 +655,7 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     a.dtype = dtype;
     a.ld = ld;
     a.noise = noise;
-    a.states = states;
+    a.states = states_in;
     a.states_out = states;
     a.tokens_out = tokens_out;
     a.masked_out = masked_out;
@@ -668,6 +673,9 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     adv.n_states = pda->n_states;
     adv.eos_id = table->eos_id;
     adv.cap = stack_cap;
+    adv.states_in = states_in;
+    adv.stacks_in = stacks_in;
+    adv.depths_in = depths_in;
     adv.states = states;
     adv.stacks = stacks;
     adv.depths = depths;
@@ -678,6 +686,91 @@ extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, 
     a.V = table->V;
     a.ldw = table->ldw;
     return cstr_launch_step(a, stream);
+}
+
+extern "C" int cstr_pda_step(const cstr_pda_table_t *table, const void *logits, int32_t dtype,
+                             int64_t ld, const float *noise, int32_t *states, int32_t *stacks,
+                             int32_t *depths, int32_t stack_cap, int32_t *tokens_out,
+                             void *masked_out, uint8_t *accept_out, int32_t batch,
+                             cstr_pda_workspace_t *ws, void *cuda_stream)
+{
+    return pda_step_common(table, logits, dtype, ld, noise, states, stacks, depths, states, stacks,
+                           depths, stack_cap, tokens_out, masked_out, accept_out, batch, ws,
+                           cuda_stream);
+}
+
+extern "C" int cstr_pda_step_history(const cstr_pda_table_t *table, const void *logits,
+                                     int32_t dtype, int64_t ld, const float *noise,
+                                     const int32_t *states_in, const int32_t *stacks_in,
+                                     const int32_t *depths_in, int32_t *states_out,
+                                     int32_t *stacks_out, int32_t *depths_out, int32_t stack_cap,
+                                     int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
+                                     int32_t batch, cstr_pda_workspace_t *ws, void *cuda_stream)
+{
+    return pda_step_common(table, logits, dtype, ld, noise, states_in, stacks_in, depths_in,
+                           states_out, stacks_out, depths_out, stack_cap, tokens_out, masked_out,
+                           accept_out, batch, ws, cuda_stream);
+}
+
+// ---- speculative decoding: accept / rewind --------------------------------------
+//
+// As in the finite-state case, but the constraint's situation after a token is
+// a state plus a stack, so the history holds all three per drafted position and
+// the rewind copies the stack of the position it goes back to.
+
+namespace {
+
+__global__ void __launch_bounds__(128)
+pda_accept_draft_kernel(const int32_t *__restrict__ draft, const int32_t *__restrict__ tgt_tok,
+                        const int32_t *__restrict__ tgt_state, const int32_t *__restrict__ tgt_stacks,
+                        const int32_t *__restrict__ tgt_depth, int k, int batch, int cap,
+                        int32_t *__restrict__ n_accepted, int32_t *__restrict__ out_tokens,
+                        int32_t *__restrict__ states, int32_t *__restrict__ stacks,
+                        int32_t *__restrict__ depths)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= batch)
+        return;
+    const int32_t *d = draft + (long long)r * k;
+    const int32_t *t = tgt_tok + (long long)r * (k + 1);
+    int n = 0;
+    while (n < k && d[n] == t[n])
+        ++n;
+    for (int i = 0; i <= k; ++i)
+        out_tokens[(long long)r * (k + 1) + i] = (i <= n) ? t[i] : -1;
+    n_accepted[r] = n;
+    const long long at = (long long)r * (k + 1) + n;
+    states[r] = tgt_state[at];
+    const int depth = tgt_depth[at];
+    depths[r] = depth;
+    const int32_t *src = tgt_stacks + at * cap;
+    int32_t *dst = stacks + (long long)r * cap;
+    for (int i = 0; i < depth && i < cap; ++i)
+        dst[i] = src[i];
+}
+
+}  // namespace
+
+extern "C" int cstr_pda_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,
+                                     const int32_t *target_states, const int32_t *target_stacks,
+                                     const int32_t *target_depths, int32_t k, int32_t batch,
+                                     int32_t stack_cap, int32_t *n_accepted, int32_t *out_tokens,
+                                     int32_t *states, int32_t *stacks, int32_t *depths,
+                                     void *cuda_stream)
+{
+    if (!target_tokens || !target_states || !target_stacks || !target_depths || !n_accepted ||
+        !out_tokens || !states || !stacks || !depths || (k > 0 && !draft_tokens))
+        return cstr_fail(CSTR_ERR_NULL, "cstr_pda_accept_draft: null pointer");
+    if (k < 0 || batch < 0 || stack_cap < 1)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_pda_accept_draft: k = %d, batch = %d, stack_cap = %d",
+                         k, batch, stack_cap);
+    if (batch == 0)
+        return CSTR_OK;
+    pda_accept_draft_kernel<<<(batch + 127) / 128, 128, 0, (cudaStream_t)cuda_stream>>>(
+        draft_tokens, target_tokens, target_states, target_stacks, target_depths, k, batch,
+        stack_cap, n_accepted, out_tokens, states, stacks, depths);
+    CSTR_CUDA_TRY(cudaGetLastError());
+    return CSTR_OK;
 }
 
 extern "C" int cstr_pda_step_status(cstr_pda_workspace_t *ws, void *cuda_stream, int64_t *bad_rows,

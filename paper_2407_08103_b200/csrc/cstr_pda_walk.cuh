@@ -65,31 +65,42 @@ __device__ __forceinline__ int pda_walk(const cstr_pda_view &P, int q, const int
 // and stack edit.  `active` = the row had a usable state and stack.
 __device__ __forceinline__ void pda_traverse(const cstr_pda_advance &a, int r, bool active, int tok)
 {
-    const int q = a.states[r];
+    const int q = a.states_in[r];
+    const int d = a.depths_in[r];
+    const int32_t *s_in = a.stacks_in + (long long)r * a.cap;
+    int32_t *s_out = a.stacks + (long long)r * a.cap;
+    const bool in_place = s_in == s_out;
     int q2 = CSTR_DEAD;
+    int keep = (d >= 0 && d <= a.cap) ? d : 0;     // symbols of the old stack that stay
+    int d2 = d;
+    uint8_t loc[kLocMax];
+    int nloc = 0;
     if (!active) {
         if (q != -1)
             atomicAdd(a.counters + 0, 1ull);
     } else if (tok < 0) {
         atomicAdd(a.counters + 1, 1ull);
     } else if (tok != a.eos_id) {
-        const int d = a.depths[r];
-        int32_t *s = a.stacks + (long long)r * a.cap;
-        uint8_t loc[kLocMax];
-        int qn, cd, nloc;
+        int qn, cd, nl;
         const uint32_t b0 = a.voff[tok], b1 = a.voff[tok + 1];
-        if (pda_walk(a.P, q, s, 0, d, false, a.vbytes + b0, (int)(b1 - b0), loc, qn, cd, nloc) ==
+        if (pda_walk(a.P, q, s_in, 0, d, false, a.vbytes + b0, (int)(b1 - b0), loc, qn, cd, nl) ==
             WALK_OK) {
-            if (cd + nloc > a.cap) {
+            if (cd + nl > a.cap) {
                 atomicAdd(a.counters + 2, 1ull);
             } else {
-                for (int i = 0; i < nloc; ++i)
-                    s[cd + i] = loc[i];
-                a.depths[r] = cd + nloc;
+                keep = cd;
+                nloc = nl;
+                d2 = cd + nl;
                 q2 = qn;
             }
         }
     }
+    if (!in_place)                                  // the history keeps the old row untouched
+        for (int i = 0; i < keep; ++i)
+            s_out[i] = s_in[i];
+    for (int i = 0; i < nloc; ++i)
+        s_out[keep + i] = loc[i];
+    a.depths[r] = d2;
     a.states[r] = q2;
     if (a.accept_out)
         a.accept_out[r] = (q2 >= 0) ? (uint8_t)(a.accept[q2] != 0) : (uint8_t)0;

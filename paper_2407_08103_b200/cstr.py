@@ -30,7 +30,8 @@ EXPORTS = [
     "cstr_load_pda", "cstr_free_pda", "cstr_build_pda_table", "cstr_free_pda_table",
     "cstr_pda_table_rebuild", "cstr_pda_table_info", "cstr_pda_table_download",
     "cstr_pda_workspace_create",
-    "cstr_free_pda_workspace", "cstr_pda_step", "cstr_pda_step_status",
+    "cstr_free_pda_workspace", "cstr_pda_step", "cstr_pda_step_history",
+    "cstr_pda_accept_draft", "cstr_pda_step_status",
 ]
 
 _lib = None
@@ -392,10 +393,13 @@ def cstr_pda_workspace_create(table: PdaTable, max_batch: int) -> PdaWorkspace:
 
 
 def cstr_pda_step(table: PdaTable, logits, states, stacks, depths, tokens_out, masked_out,
-                  ws: PdaWorkspace, noise=None, accept_out=None, stream=None) -> None:
+                  ws: PdaWorkspace, noise=None, accept_out=None, stream=None,
+                  states_out=None, stacks_out=None, depths_out=None) -> None:
     """Enqueue one step of Algorithm 3.  CUDA tensors: ``logits`` / ``masked_out`` /
     ``noise`` as in ``cstr_step``; ``states`` / ``depths`` / ``tokens_out`` int32 ``[B]``;
-    ``stacks`` int32 ``[B][cap]`` (bottom first)."""
+    ``stacks`` int32 ``[B][cap]`` (bottom first).  With ``states_out`` /
+    ``stacks_out`` / ``depths_out`` given (all three) the inputs are left untouched
+    (``cstr_pda_step_history``)."""
     import torch
     if logits.dtype == torch.float32:
         dtype = CSTR_F32
@@ -422,11 +426,61 @@ def cstr_pda_step(table: PdaTable, logits, states, stacks, depths, tokens_out, m
     if stacks.dtype != torch.int32 or stacks.dim() != 2 or stacks.shape[0] < batch \
             or not stacks.is_contiguous():
         raise ValueError("stacks must be a contiguous int32 tensor [B][cap]")
+    outs = (states_out, stacks_out, depths_out)
+    if any(o is not None for o in outs):
+        if any(o is None for o in outs):
+            raise ValueError("states_out, stacks_out and depths_out go together")
+        for o, i in zip(outs, (states, stacks, depths)):
+            if o.dtype != torch.int32 or o.shape != i.shape or not o.is_contiguous():
+                raise ValueError("output situation arrays must match the input ones")
+        _check(lib().cstr_pda_step_history(
+            table.ptr, _dev_ptr(logits), ctypes.c_int32(dtype), ctypes.c_int64(logits.stride(0)),
+            _dev_ptr(noise), _dev_ptr(states), _dev_ptr(stacks), _dev_ptr(depths),
+            _dev_ptr(states_out), _dev_ptr(stacks_out), _dev_ptr(depths_out),
+            ctypes.c_int32(stacks.shape[1]), _dev_ptr(tokens_out), _dev_ptr(masked_out),
+            _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr, _stream_ptr(stream)))
+        return
     _check(lib().cstr_pda_step(table.ptr, _dev_ptr(logits), ctypes.c_int32(dtype),
                                ctypes.c_int64(logits.stride(0)), _dev_ptr(noise), _dev_ptr(states),
                                _dev_ptr(stacks), _dev_ptr(depths), ctypes.c_int32(stacks.shape[1]),
                                _dev_ptr(tokens_out), _dev_ptr(masked_out), _dev_ptr(accept_out),
                                ctypes.c_int32(batch), ws.ptr, _stream_ptr(stream)))
+
+
+def cstr_pda_step_history(table: PdaTable, logits, states_in, stacks_in, depths_in, states_out,
+                          stacks_out, depths_out, tokens_out, masked_out, ws: PdaWorkspace,
+                          **kw) -> None:
+    """``cstr_pda_step`` with separate input and output situations (state history)."""
+    cstr_pda_step(table, logits, states_in, stacks_in, depths_in, tokens_out, masked_out, ws,
+                  states_out=states_out, stacks_out=stacks_out, depths_out=depths_out, **kw)
+
+
+def cstr_pda_accept_draft(draft_tokens, target_tokens, target_states, target_stacks,
+                          target_depths, n_accepted, out_tokens, states, stacks, depths,
+                          stream=None) -> None:
+    """Greedy verification + rewind under a push-down constraint.  CUDA int32 tensors:
+    ``draft_tokens`` ``[B][k]``; ``target_tokens`` / ``target_states`` / ``target_depths`` /
+    ``out_tokens`` ``[B][k+1]``; ``target_stacks`` ``[B][k+1][cap]``; ``n_accepted`` /
+    ``states`` / ``depths`` ``[B]``; ``stacks`` ``[B][cap]``."""
+    import torch
+    B, k1 = target_tokens.shape
+    k = k1 - 1
+    cap = target_stacks.shape[2]
+    for name, t, shape in (("draft_tokens", draft_tokens, (B, k)), ("target_tokens", target_tokens, (B, k1)),
+                           ("target_states", target_states, (B, k1)),
+                           ("target_depths", target_depths, (B, k1)),
+                           ("target_stacks", target_stacks, (B, k1, cap)),
+                           ("out_tokens", out_tokens, (B, k1)), ("n_accepted", n_accepted, (B,)),
+                           ("states", states, (B,)), ("depths", depths, (B,)),
+                           ("stacks", stacks, (B, cap))):
+        if t.dtype != torch.int32 or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous int32 tensor of shape %s" % (name, shape))
+    _check(lib().cstr_pda_accept_draft(_dev_ptr(draft_tokens), _dev_ptr(target_tokens),
+                                       _dev_ptr(target_states), _dev_ptr(target_stacks),
+                                       _dev_ptr(target_depths), ctypes.c_int32(k), ctypes.c_int32(B),
+                                       ctypes.c_int32(cap), _dev_ptr(n_accepted),
+                                       _dev_ptr(out_tokens), _dev_ptr(states), _dev_ptr(stacks),
+                                       _dev_ptr(depths), _stream_ptr(stream)))
 
 
 def cstr_pda_step_status(ws: PdaWorkspace, stream=None):

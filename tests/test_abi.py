@@ -89,6 +89,10 @@ def test_null_and_range_errors(lib):
     assert lib.cstr_pda_step(None, None, 0, 0, None, None, None, None, 4, None, None, None, 1,
                              None, None) == -1
     assert lib.cstr_pda_step_status(None, None, None, None, None) == -1
+    assert lib.cstr_pda_step_history(None, None, 0, 0, None, None, None, None, None, None, None, 4,
+                                     None, None, None, 1, None, None) == -1
+    assert lib.cstr_pda_accept_draft(None, None, None, None, None, 1, 1, 4, None, None, None, None,
+                                     None, None) == -1
     # free functions accept NULL
     lib.cstr_free_pda(None)
     lib.cstr_free_pda_table(None)

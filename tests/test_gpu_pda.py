@@ -354,3 +354,86 @@ def test_grammar_built_json_pda():
         ref = run_both(P, table, ws, vb, vo, logits, states, stacks, depth)
         states, depth, stacks = ref["states"], ref["depth"], ref["stacks_full"]
     assert depth.max() >= 2
+
+
+def test_speculative_loop_pushdown():
+    # draft k tokens with cstr_pda_step_history (keeping every situation), verify all k + 1
+    # positions in one call over the history, accept / rewind; every array against the oracle
+    from synth.models import draft_logits, target_logits
+    P = json_pda(space=True)
+    vb, vo = make_vocab_json(1200, seed=6)
+    V = vo.size - 1
+    table = build(P, vb, vo)
+    B, k, cap = 6, 3, 8
+    ws = cstr.cstr_pda_workspace_create(table, B * (k + 1))
+    i32 = dict(dtype=torch.int32, device=DEV)
+    g_state = torch.full((B,), P.start, **i32)
+    g_stack = torch.zeros((B, cap), **i32)
+    g_depth = torch.zeros((B,), **i32)
+    o_state = np.full(B, P.start, np.int32)
+    o_stack = np.zeros((B, cap), np.int32)
+    o_depth = np.zeros(B, np.int32)
+    outs = [[] for _ in range(B)]
+    kept = 0
+    for rnd in range(5):
+        h_state = torch.zeros((B, k + 1), **i32)
+        h_stack = torch.zeros((B, k + 1, cap), **i32)
+        h_depth = torch.zeros((B, k + 1), **i32)
+        h_state[:, 0], h_stack[:, 0], h_depth[:, 0] = g_state, g_stack, g_depth
+        oh_state, oh_stack, oh_depth = [o_state], [o_stack], [o_depth]
+        drafts = torch.zeros((B, k), **i32)
+        o_drafts = np.zeros((B, k), np.int32)
+        for i in range(k):
+            prefixes = [outs[r] + [int(t) for t in o_drafts[r, :i]] for r in range(B)]
+            logits = np.stack([draft_logits(9, r, prefixes[r], V) for r in range(B)])
+            d_logits = to_dev_logits(logits)
+            tok = torch.empty((B,), **i32)
+            s_in, k_in, d_in = (h_state[:, i].contiguous(), h_stack[:, i].contiguous(),
+                                h_depth[:, i].contiguous())
+            s_out, k_out, d_out = torch.empty_like(s_in), torch.empty_like(k_in), torch.empty_like(d_in)
+            cstr.cstr_pda_step_history(table, d_logits, s_in, k_in, d_in, s_out, k_out, d_out, tok,
+                                       torch.empty_like(d_logits), ws)
+            h_state[:, i + 1], h_stack[:, i + 1], h_depth[:, i + 1] = s_out, k_out, d_out
+            drafts[:, i] = tok
+            ref = op.step(P, vb, vo, logits, oh_state[-1], oh_stack[-1], oh_depth[-1], threads=4)
+            assert np.array_equal(tok.cpu().numpy(), ref["tokens"])
+            assert np.array_equal(s_in.cpu().numpy(), oh_state[-1])        # inputs untouched
+            o_drafts[:, i] = ref["tokens"]
+            oh_state.append(ref["states"]); oh_stack.append(ref["stacks"]); oh_depth.append(ref["depth"])
+        # verification: one call over B x (k + 1) history rows
+        prefixes = [[outs[r] + [int(t) for t in o_drafts[r, :i]] for i in range(k + 1)] for r in range(B)]
+        tl = np.stack([target_logits(9, r, prefixes[r][i], V) for r in range(B) for i in range(k + 1)])
+        d_tl = to_dev_logits(tl)
+        n_rows = B * (k + 1)
+        t_tok = torch.empty((n_rows,), **i32)
+        t_state, t_stack, t_depth = (torch.empty((n_rows,), **i32), torch.empty((n_rows, cap), **i32),
+                                     torch.empty((n_rows,), **i32))
+        cstr.cstr_pda_step_history(table, d_tl, h_state.view(-1), h_stack.view(n_rows, cap),
+                                   h_depth.view(-1), t_state, t_stack, t_depth, t_tok,
+                                   torch.empty_like(d_tl), ws)
+        ref = op.step(P, vb, vo, tl, np.stack(oh_state, 1).reshape(-1),
+                      np.stack(oh_stack, 1).reshape(n_rows, cap), np.stack(oh_depth, 1).reshape(-1),
+                      threads=4)
+        assert np.array_equal(t_tok.cpu().numpy(), ref["tokens"])
+        assert np.array_equal(t_state.cpu().numpy(), ref["states"])
+        assert np.array_equal(t_depth.cpu().numpy(), ref["depth"])
+        n_acc = torch.empty((B,), **i32)
+        out_tok = torch.empty((B, k + 1), **i32)
+        cstr.cstr_pda_accept_draft(drafts, t_tok.view(B, k + 1), t_state.view(B, k + 1),
+                                   t_stack.view(B, k + 1, cap), t_depth.view(B, k + 1), n_acc,
+                                   out_tok, g_state, g_stack, g_depth)
+        torch.cuda.synchronize()
+        on, oout, o_state, o_stack, o_depth = op.accept_draft(
+            o_drafts, ref["tokens"].reshape(B, k + 1), ref["states"].reshape(B, k + 1),
+            ref["stacks"].reshape(B, k + 1, cap), ref["depth"].reshape(B, k + 1))
+        assert np.array_equal(n_acc.cpu().numpy(), on) and np.array_equal(out_tok.cpu().numpy(), oout)
+        assert np.array_equal(g_state.cpu().numpy(), o_state)
+        assert np.array_equal(g_depth.cpu().numpy(), o_depth)
+        gs = g_stack.cpu().numpy()
+        for r in range(B):
+            n = o_depth[r]
+            assert np.array_equal(gs[r, :n], o_stack[r, :n])
+            outs[r] += [int(t) for t in oout[r] if t >= 0]
+        o_stack = gs.copy()                              # beyond the depth both sides are free
+        kept += int(on.sum())
+    assert kept > 0 and max(len(o) for o in outs) >= 5

@@ -440,3 +440,63 @@ def test_bracketed_grammar_front_end():
         grammar_to_pda(r"<B>", {}, {"B": ("(", r"[a)]*", ")")})
     with pytest.raises(GrammarError):            # recursion outside a bracket
         grammar_to_pda(r"<m>", {"m": "a<m>?"}, {})
+
+
+# ------------------------------------------------ rewindable push-down constraint
+
+def pda_target_only(P, vb, vo, seed, row, n_tokens, cap):
+    from synth.models import target_logits
+    V = vo.size - 1
+    q, s, d, out = P.start, np.zeros((1, cap), np.int32), np.zeros(1, np.int32), []
+    while len(out) < n_tokens and q >= 0:
+        res = op.step(P, vb, vo, target_logits(seed, row, out, V)[None, :], [q], s, d)
+        tok = int(res["tokens"][0])
+        if tok < 0:
+            break
+        out.append(tok)
+        q, s, d = int(res["states"][0]), res["stacks"], res["depth"]
+    return out
+
+
+def pda_speculative(P, vb, vo, seed, row, n_tokens, k, cap):
+    """Draft k tokens keeping the history of situations, verify all k + 1 positions in
+    one batched step over the history, accept and rewind; repeat."""
+    from synth.models import draft_logits, target_logits
+    V = vo.size - 1
+    q, s, d, out, kept = P.start, np.zeros(cap, np.int32), 0, [], 0
+    while len(out) < n_tokens and q >= 0:
+        hq, hs, hd, draft = [q], [s], [d], []
+        for i in range(k):
+            res = op.step(P, vb, vo, draft_logits(seed, row, out + draft, V)[None, :], [hq[-1]],
+                          hs[-1][None, :], [hd[-1]])
+            draft.append(int(res["tokens"][0]))
+            hq.append(int(res["states"][0]))
+            hs.append(res["stacks"][0])
+            hd.append(int(res["depth"][0]))
+        tl = np.stack([target_logits(seed, row, out + draft[:i], V) for i in range(k + 1)])
+        res = op.step(P, vb, vo, tl, hq, np.stack(hs), hd)
+        n, toks, st, sk, dp = op.accept_draft(np.array([draft]), res["tokens"][None, :],
+                                              res["states"][None, :], res["stacks"][None, :, :],
+                                              res["depth"][None, :])
+        emitted = [int(t) for t in toks[0] if t >= 0]
+        out += emitted
+        q, s, d = int(st[0]), sk[0], int(dp[0])
+        kept += int(n[0])
+        if not emitted:
+            break
+    return out[:n_tokens], kept
+
+
+@pytest.mark.parametrize("k", [1, 3])
+def test_pda_speculative_equals_target_only(k):
+    # with greedy selection, draft / verify / rewind emits exactly what constrained
+    # decoding with the target model alone emits - stacks included in the rewind
+    P = json_pda(space=True)
+    vb, vo = small_json_vocab()
+    total_kept = 0
+    for row in range(3):
+        want = pda_target_only(P, vb, vo, 77, row, 12, cap=8)
+        got, kept = pda_speculative(P, vb, vo, 77, row, 12, k, cap=8)
+        assert got == want[:len(got)] and len(got) == len(want)
+        total_kept += kept
+    assert total_kept > 0
