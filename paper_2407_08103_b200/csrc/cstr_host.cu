@@ -23,7 +23,7 @@ int cstr_fail(int code, const char *fmt, ...)
 
 extern "C" const char *cstr_last_error(void) { return g_err; }
 
-static int check_device(int handle_device, const char *what)
+int cstr_check_device(int handle_device, const char *what)
 {
     int cur = -1;
     CSTR_CUDA_TRY(cudaGetDevice(&cur));
@@ -413,7 +413,7 @@ extern "C" int cstr_vocab_set_token_sets(cstr_vocab_t *vocab, const uint32_t *to
     if (n_labels < 1 || n_labels > 32)
         return cstr_fail(CSTR_ERR_ARG, "cstr_vocab_set_token_sets: n_labels = %d, need 1..32",
                          n_labels);
-    int rc = check_device(vocab->device, "vocabulary");
+    int rc = cstr_check_device(vocab->device, "vocabulary");
     if (rc)
         return rc;
     uint32_t *dev = nullptr;
@@ -605,7 +605,7 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     *out = nullptr;
     if (max_states < 1)
         return cstr_fail(CSTR_ERR_ARG, "cstr_table_create: max_states = %d, need >= 1", max_states);
-    int rc = check_device(vocab->device, "vocabulary");
+    int rc = cstr_check_device(vocab->device, "vocabulary");
     if (rc)
         return rc;
     cstr_table *t = new (std::nothrow) cstr_table();
@@ -671,7 +671,7 @@ extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int3
 {
     if (!table || !dfa)
         return cstr_fail(CSTR_ERR_NULL, "cstr_table_build: null pointer");
-    int rc = check_device(table->device, "table");
+    int rc = cstr_check_device(table->device, "table");
     if (rc)
         return rc;
     if (dfa->device != table->device)
@@ -745,7 +745,7 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
 {
     if (!t)
         return cstr_fail(CSTR_ERR_NULL, "cstr_table_download: null table");
-    int rc = check_device(t->device, "table");
+    int rc = cstr_check_device(t->device, "table");
     if (rc)
         return rc;
     if (state_lo < 0 || state_hi < state_lo || state_hi > t->n_states)
@@ -860,7 +860,7 @@ static int step_common(const cstr_table_t *const *tables, int32_t n_tables,
     if (batch > ws->max_batch)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_step: batch %d exceeds workspace capacity %d",
                          batch, ws->max_batch);
-    int rc = check_device(ws->device, "workspace");
+    int rc = cstr_check_device(ws->device, "workspace");
     if (rc)
         return rc;
     cstr_step_args a;
@@ -944,7 +944,7 @@ extern "C" int cstr_step_status(cstr_workspace_t *ws, void *cuda_stream, int64_t
 {
     if (!ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_step_status: null workspace");
-    int rc = check_device(ws->device, "workspace");
+    int rc = cstr_check_device(ws->device, "workspace");
     if (rc)
         return rc;
     cudaStream_t stream = (cudaStream_t)cuda_stream;

@@ -11,6 +11,10 @@
 // Set the calling thread's error message (printf-style) and return `code`.
 int cstr_fail(int code, const char *fmt, ...);
 
+// CSTR_OK if `handle_device` is the current CUDA device, else CSTR_ERR_DEVICE
+// (or CSTR_ERR_CUDA) with a message naming `what`.
+int cstr_check_device(int handle_device, const char *what);
+
 #define CSTR_CUDA_TRY(expr)                                                              \
     do {                                                                                 \
         cudaError_t e_ = (expr);                                                         \

@@ -213,16 +213,6 @@ pda_prepare_kernel(const __grid_constant__ PdaPrepParams p)
         p.row_mask[r] = out;
 }
 
-int check_device(int handle_device, const char *what)
-{
-    int cur = -1;
-    CSTR_CUDA_TRY(cudaGetDevice(&cur));
-    if (cur != handle_device)
-        return cstr_fail(CSTR_ERR_DEVICE, "%s was created on device %d but device %d is current",
-                         what, handle_device, cur);
-    return CSTR_OK;
-}
-
 int cuda_rc(cudaError_t e, const char *who)
 {
     return cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA, "%s: %s", who,
@@ -407,7 +397,7 @@ extern "C" int cstr_pda_table_rebuild(cstr_pda_table_t *t, int32_t eos_id, void 
 {
     if (!t)
         return cstr_fail(CSTR_ERR_NULL, "cstr_pda_table_rebuild: null table");
-    int rc = check_device(t->device, "PDA table");
+    int rc = cstr_check_device(t->device, "PDA table");
     if (rc)
         return rc;
     if (eos_id < -1 || eos_id >= t->V)
@@ -426,7 +416,7 @@ extern "C" int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *v
     if (!pda || !vocab || !out)
         return cstr_fail(CSTR_ERR_NULL, "cstr_build_pda_table: null pointer");
     *out = nullptr;
-    int rc = check_device(pda->device, "PDA");
+    int rc = cstr_check_device(pda->device, "PDA");
     if (rc)
         return rc;
     if (vocab->device != pda->device)
@@ -508,7 +498,7 @@ extern "C" int cstr_pda_table_download(const cstr_pda_table_t *t, int32_t state,
 {
     if (!t)
         return cstr_fail(CSTR_ERR_NULL, "cstr_pda_table_download: null table");
-    int rc = check_device(t->device, "PDA table");
+    int rc = cstr_check_device(t->device, "PDA table");
     if (rc)
         return rc;
     if (state < 0 || state >= t->pda->n_states || top < -1 || top >= t->pda->n_symbols)
@@ -548,7 +538,7 @@ extern "C" int cstr_pda_workspace_create(const cstr_pda_table_t *table, int32_t 
     if (max_batch < 1)
         return cstr_fail(CSTR_ERR_ARG, "cstr_pda_workspace_create: max_batch = %d, need >= 1",
                          max_batch);
-    int rc = check_device(table->device, "PDA table");
+    int rc = cstr_check_device(table->device, "PDA table");
     if (rc)
         return rc;
     cstr_pda_workspace *ws = new (std::nothrow) cstr_pda_workspace();
@@ -612,7 +602,7 @@ static int pda_step_common(const cstr_pda_table_t *table, const void *logits, in
     if (ld < table->V)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_pda_step: ld = %lld is below V = %d", (long long)ld,
                          table->V);
-    int rc = check_device(ws->device, "PDA workspace");
+    int rc = cstr_check_device(ws->device, "PDA workspace");
     if (rc)
         return rc;
     if (table->device != ws->device)
@@ -778,7 +768,7 @@ extern "C" int cstr_pda_step_status(cstr_pda_workspace_t *ws, void *cuda_stream,
 {
     if (!ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_pda_step_status: null workspace");
-    int rc = check_device(ws->device, "PDA workspace");
+    int rc = cstr_check_device(ws->device, "PDA workspace");
     if (rc)
         return rc;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
