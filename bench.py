@@ -200,6 +200,26 @@ def time_oracle_single_thread(dfa, vb, vo, pool, rows: int = 8):
     return rows * pool.shape[1] / (time.perf_counter() - t0)
 
 
+def time_oracle_table_build(dfa, vb, vo, budget_s: float = 3.0):
+    """The oracle's token table for slabs of states (all host threads) until the
+    budget is used: transitions/s, with what was timed."""
+    import oracle
+    threads = oracle.max_threads()
+    S, V = int(dfa[0].shape[0]), vo.size - 1
+    slab = min(S, 4 * threads)
+    oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=0, q_hi=min(S, threads), threads=threads)  # warm
+    done, lo, t0 = 0, 0, time.perf_counter()
+    while done == 0 or time.perf_counter() - t0 < budget_s:
+        hi = min(S, lo + slab)
+        oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=lo, q_hi=hi, threads=threads)
+        done += hi - lo
+        lo = hi if hi < S else 0
+    dt = time.perf_counter() - t0
+    return {"value": done * V / dt, "unit": "transitions/s", "cores": threads, "kind": "oracle",
+            "sample": "%d of %d states x %d tokens of %s in %.1f s (whole table extrapolates to "
+                      "%.1f s)" % (done, S, V, WORKLOAD, dt, S * V / (done * V / dt))}
+
+
 def time_oracle(w, dfa, vb, vo, pools, budget_s: float, max_steps: int):
     """The oracle as it stands, all host threads, whole-batch steps until the
     time budget is used (at least 2 steps).  Returns (logits/s, cores, sample text, s/step)."""
@@ -778,7 +798,8 @@ def main():
         v, cores, sample, _ = time_oracle(w, dfa, vb, vo, pools, args.cpu_seconds, 400)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                "cpu_model": cpu_model_string(), "host_threads_available": os.cpu_count(),
-               "single_thread_value": time_oracle_single_thread(dfa, vb, vo, pools[0])}
+               "single_thread_value": time_oracle_single_thread(dfa, vb, vo, pools[0]),
+               "table_build": time_oracle_table_build(dfa, vb, vo)}
 
     if rank != 0:
         if world > 1:
