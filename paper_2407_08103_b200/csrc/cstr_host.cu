@@ -501,7 +501,7 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
             keys[v].len = len;
             keys[v].id = v;
         }
-        std::sort(keys.begin(), keys.end(), [&](const SortKey &x, const SortKey &y) {
+        auto full_less = [&](const SortKey &x, const SortKey &y) {
             if (x.head != y.head)
                 return x.head < y.head;
             const int32_t a = x.id, b = y.id;
@@ -515,7 +515,44 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
             if (la != lb)
                 return la < lb;
             return a < b;
-        });
+        };
+        // Stable radix passes, least significant digit first: min(length, 9), then
+        // the head in four 16-bit digits.  Ids start in ascending order, so equal
+        // (head, length <= 8) keys - equal strings - end up ordered by id, and a
+        // token of at most 8 bytes precedes the longer ones it is a prefix of.
+        // Runs of longer tokens with equal heads are finished by comparison.
+        {
+            std::vector<SortKey> tmp((size_t)vocab_size);
+            std::vector<uint32_t> count(65536 + 1);
+            SortKey *src = keys.data(), *dst = tmp.data();
+            for (int pass = 0; pass < 5; ++pass) {
+                auto digit = [pass](const SortKey &k) -> uint32_t {
+                    if (pass == 0)
+                        return k.len < 9 ? k.len : 9u;
+                    return (uint32_t)(k.head >> (16 * (pass - 1))) & 0xffffu;
+                };
+                std::fill(count.begin(), count.end(), 0u);
+                for (int32_t i = 0; i < vocab_size; ++i)
+                    ++count[digit(src[i]) + 1];
+                for (uint32_t d = 0; d < 65536; ++d)
+                    count[d + 1] += count[d];
+                for (int32_t i = 0; i < vocab_size; ++i)
+                    dst[count[digit(src[i])]++] = src[i];
+                std::swap(src, dst);
+            }
+            if (src != keys.data())              // five passes: the result sits in tmp
+                memcpy(keys.data(), src, (size_t)vocab_size * sizeof(SortKey));
+        }
+        for (int32_t i = 0; i < vocab_size;) {
+            int32_t j = i + 1;
+            if (keys[i].len > 8) {
+                while (j < vocab_size && keys[j].head == keys[i].head && keys[j].len > 8)
+                    ++j;
+                if (j - i > 1)
+                    std::sort(keys.begin() + i, keys.begin() + j, full_less);
+            }
+            i = j;
+        }
         for (int32_t i = 0; i < vocab_size; ++i)
             order[i] = keys[i].id;
         for (int32_t i = 0; i < vocab_size; ++i) {
