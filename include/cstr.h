@@ -212,6 +212,7 @@ void cstr_free_workspace(cstr_workspace_t *ws);
  * index is out of range, and a row with no selectable token, get token -1,
  * state -1 and all -infinity; nothing out of bounds is ever touched.
  * Only enqueues work on cuda_stream (no allocation, no host synchronisation).
+ * With batch == 0 the per-row pointers may be NULL and nothing is enqueued.
  * The fast path needs logits / masked_out / noise 16-byte aligned with
  * ld * sizeof(element) a multiple of 16; other layouts take a slower kernel.
  */

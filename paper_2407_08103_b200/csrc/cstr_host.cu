@@ -885,6 +885,8 @@ static int step_common(const cstr_table_t *const *tables, int32_t n_tables,
                        int32_t *tokens_out, void *masked_out, uint8_t *accept_out, int32_t batch,
                        cstr_workspace_t *ws, void *cuda_stream)
 {
+    if (batch == 0 && tables && ws && (dtype == CSTR_F32 || dtype == CSTR_BF16))
+        return CSTR_OK;              // nothing to do: the per-row arrays may be empty (null)
     if (!tables || !logits || !states || !states_out || !tokens_out || !masked_out || !ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_step: null pointer");
     if (n_tables < 1 || n_tables > CSTR_MAX_TABLES)

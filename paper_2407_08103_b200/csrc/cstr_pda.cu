@@ -584,6 +584,8 @@ static int pda_step_common(const cstr_pda_table_t *table, const void *logits, in
                            void *masked_out, uint8_t *accept_out, int32_t batch,
                            cstr_pda_workspace_t *ws, void *cuda_stream)
 {
+    if (batch == 0 && table && ws && (dtype == CSTR_F32 || dtype == CSTR_BF16) && stack_cap >= 1)
+        return CSTR_OK;              // nothing to do: the per-row arrays may be empty (null)
     if (!table || !logits || !states || !stacks || !depths || !states_in || !stacks_in ||
         !depths_in || !tokens_out || !masked_out || !ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_pda_step: null pointer");

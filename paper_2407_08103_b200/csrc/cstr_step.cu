@@ -596,6 +596,8 @@ extern "C" int cstr_step_static(const cstr_table_t *const *tables, int32_t n_tab
                                 int32_t *tokens_out, void *masked_out, uint8_t *accept_out,
                                 int32_t batch, void *cuda_stream)
 {
+    if (batch == 0 && tables && (dtype == CSTR_F32 || dtype == CSTR_BF16))
+        return CSTR_OK;              // nothing to do: the per-row arrays may be empty (null)
     if (!tables || !logits || !states || !tokens_out || !masked_out)
         return cstr_fail(CSTR_ERR_NULL, "cstr_step_static: null pointer");
     if (n_tables < 1 || n_tables > CSTR_MAX_TABLES)

@@ -437,3 +437,26 @@ def test_speculative_loop_pushdown():
         o_stack = gs.copy()                              # beyond the depth both sides are free
         kept += int(on.sum())
     assert kept > 0 and max(len(o) for o in outs) >= 5
+
+
+def test_empty_batch_and_limits():
+    P = anbn_pda()
+    vb, vo = vocab_from_strings([b"a", b"b", b"bb", b"aaab"])
+    table = build(P, vb, vo)
+    ws = cstr.cstr_pda_workspace_create(table, 4)
+    i32 = dict(dtype=torch.int32, device=DEV)
+    logits = torch.empty((0, 4), device=DEV)
+    cstr.cstr_pda_step(table, logits, torch.empty((0,), **i32), torch.empty((0, 8), **i32),
+                       torch.empty((0,), **i32), torch.empty((0,), **i32), torch.empty_like(logits), ws)
+    torch.cuda.synchronize()
+    assert cstr.cstr_pda_step_status(ws) == (0, 0, 0)
+    # a batch beyond the workspace, and a vocabulary whose tokens could outgrow the walk's stack
+    big = torch.zeros((5, 4), device=DEV)
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_pda_step(table, big, torch.zeros((5,), **i32), torch.zeros((5, 8), **i32),
+                           torch.zeros((5,), **i32), torch.zeros((5,), **i32), torch.empty_like(big), ws)
+    assert e.value.code == -6
+    long_vb, long_vo = vocab_from_strings([b"a" * 300, b"b"])
+    with pytest.raises(cstr.CstrError) as e:
+        cstr.cstr_build_pda_table(load_pda(P), cstr.cstr_load_vocab(long_vb, long_vo))
+    assert e.value.code == -6

@@ -276,3 +276,19 @@ def test_many_rows_small_vocabulary():
     logits = rng.standard_normal((B, V)).astype(np.float32)
     states = rng.integers(-1, 20, size=B).astype(np.int32)
     run_step_both([dfa], tables, vb, vo, logits, states)
+
+
+def test_empty_batch_is_a_no_op():
+    # zero rows: every step entry point returns without touching anything
+    dfa = config_dfas("api_1k")[0]
+    vb, vo = config_vocab("api_1k")
+    (table,) = gpu_tables([dfa], vb, vo)
+    V = vo.size - 1
+    ws = cstr.cstr_workspace_create(4)
+    logits = torch.empty((0, V), device=DEV)
+    st = torch.empty((0,), dtype=torch.int32, device=DEV)
+    cstr.cstr_step([table], logits, st, st.clone(), torch.empty_like(logits), ws)
+    cstr.cstr_step_history([table], logits, st, st.clone(), st.clone(), torch.empty_like(logits), ws)
+    cstr.cstr_step_static([table], logits, st, st.clone(), torch.empty_like(logits))
+    torch.cuda.synchronize()
+    assert cstr.cstr_step_status(ws) == (0, 0)
