@@ -727,12 +727,11 @@ def main():
     dec.reset()
 
     def e2e_step(i):
-        buf = staging[i & 1]
-        buf.copy_(host_pool[i % POOL], non_blocking=True)
-        one_step(i, buf)
-        h_tok.copy_(dec.tokens, non_blocking=True)
-        h_st.copy_(dec.states, non_blocking=True)
-        stream.synchronize()               # the sampling loop needs the tokens on the host
+        # one C-ABI call: pinned host logits in (sliced uploads overlapped with the step
+        # kernels), tokens + states back on the host when it returns
+        cstr.cstr_step_host([table], host_pool[i % POOL], dec.states, h_tok, staging[0], staging[1],
+                            dec.tokens, dec.ws, states_host=h_st, stream=stream)
+        torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
 
     e2e_ms = float("nan")
     if not args.skip_e2e:
@@ -829,7 +828,8 @@ def main():
         e2e = {"value": logits_per_step * Ke / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * 8, "steps": Ke,
                "ms_per_step": e2e_ms / Ke,
-               "note": "pinned host logits -> device, cstr_step, tokens+states -> host, sync per step"}
+               "note": "cstr_step_host per step: pinned host logits -> device in 8 row slices overlapped "
+                       "with the step kernels, tokens + states -> host, synchronous"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak",

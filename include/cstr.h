@@ -222,6 +222,32 @@ int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t
               int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
 
 /*
+ * cstr_step for logits that live in HOST memory (the end-to-end form of the
+ * same recipe: Section 1, steps 1-3, for a model whose logits arrive on the
+ * host).  The rows are cut into a few slices; each slice is uploaded on an
+ * internal copy stream while the step kernels of earlier slices run on
+ * cuda_stream, and the tokens (and states) are copied back at the end.
+ *   logits_host  HOST  [batch][ld] of `dtype` (pinned memory uploads fastest)
+ *   noise_host   HOST  float [batch][ld] or NULL
+ *   states       DEVICE int32 [batch], in/out
+ *   tokens_host  HOST  int32 [batch]: the selected tokens
+ *   states_host  HOST  int32 [batch] or NULL: the new states
+ *   logits_dev   DEVICE staging [batch][ld] of `dtype`, overwritten
+ *   noise_dev    DEVICE staging float [batch][ld]; NULL exactly when noise_host is NULL
+ *   masked_out   DEVICE [batch][ld]: the penalised logits (may equal logits_dev)
+ *   tokens_dev   DEVICE int32 [batch]
+ * tables, row_table, accept_out, ws: as in cstr_step.  Synchronous: returns
+ * after the results are in tokens_host / states_host (it synchronises
+ * cuda_stream).  Allocates no device memory; its first call on a workspace
+ * creates the copy stream and a few events.
+ */
+int cstr_step_host(const cstr_table_t *const *tables, int32_t n_tables, const int32_t *row_table,
+                   const void *logits_host, int32_t dtype, int64_t ld, const float *noise_host,
+                   int32_t *states, int32_t *tokens_host, int32_t *states_host, void *logits_dev,
+                   float *noise_dev, void *masked_out, int32_t *tokens_dev, uint8_t *accept_out,
+                   int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
+
+/*
  * cstr_step that leaves the input states untouched and writes the new ones to
  * states_out, so that a caller can keep the state after every drafted token
  * (Section 4, Speculative decoding: the target model may reject drafted

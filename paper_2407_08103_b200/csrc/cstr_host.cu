@@ -838,6 +838,12 @@ extern "C" void cstr_free_workspace(cstr_workspace_t *ws)
     cudaFree(ws->cell);
     cudaFree(ws->ticket);
     cudaFree(ws->counters);
+    if (ws->host_ready) {
+        cudaStreamDestroy(ws->copy_stream);
+        for (int i = 0; i < CSTR_HOST_SLICES; ++i)
+            cudaEventDestroy(ws->slice_ready[i]);
+        cudaEventDestroy(ws->inputs_free);
+    }
     delete ws;
 }
 
@@ -960,6 +966,86 @@ extern "C" int cstr_step_history(const cstr_table_t *const *tables, int32_t n_ta
 {
     return step_common(tables, n_tables, row_table, logits, dtype, ld, noise, states_in,
                        states_out, tokens_out, masked_out, accept_out, batch, ws, cuda_stream);
+}
+
+// The step with its logits in host memory: rows are cut into slices whose
+// uploads run on a copy stream ahead of the step kernels of earlier slices.
+extern "C" int cstr_step_host(const cstr_table_t *const *tables, int32_t n_tables,
+                              const int32_t *row_table, const void *logits_host, int32_t dtype,
+                              int64_t ld, const float *noise_host, int32_t *states,
+                              int32_t *tokens_host, int32_t *states_host, void *logits_dev,
+                              float *noise_dev, void *masked_out, int32_t *tokens_dev,
+                              uint8_t *accept_out, int32_t batch, cstr_workspace_t *ws,
+                              void *cuda_stream)
+{
+    if (!tables || !ws)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_step_host: null pointer");
+    if (dtype != CSTR_F32 && dtype != CSTR_BF16)
+        return cstr_fail(CSTR_ERR_DTYPE, "cstr_step_host: unknown dtype %d", dtype);
+    if (batch < 0 || ld < 0)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_step_host: batch = %d, ld = %lld", batch, (long long)ld);
+    if (batch == 0)
+        return CSTR_OK;
+    if (!logits_host || !states || !tokens_host || !logits_dev || !masked_out || !tokens_dev ||
+        ((noise_host != nullptr) != (noise_dev != nullptr)))
+        return cstr_fail(CSTR_ERR_NULL, "cstr_step_host: null pointer (noise needs both its host "
+                         "array and its device staging array)");
+    if (batch > ws->max_batch)
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_step_host: batch %d exceeds workspace capacity %d",
+                         batch, ws->max_batch);
+    int rc = cstr_check_device(ws->device, "workspace");
+    if (rc)
+        return rc;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (!ws->host_ready) {                       // first use: streams and events, no device memory
+        CSTR_CUDA_TRY(cudaStreamCreateWithFlags(&ws->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < CSTR_HOST_SLICES; ++i)
+            CSTR_CUDA_TRY(cudaEventCreateWithFlags(&ws->slice_ready[i], cudaEventDisableTiming));
+        CSTR_CUDA_TRY(cudaEventCreateWithFlags(&ws->inputs_free, cudaEventDisableTiming));
+        ws->host_ready = 1;
+    }
+    // uploads may start once everything enqueued so far on the caller's stream is done
+    CSTR_CUDA_TRY(cudaEventRecord(ws->inputs_free, stream));
+    CSTR_CUDA_TRY(cudaStreamWaitEvent(ws->copy_stream, ws->inputs_free, 0));
+
+    const size_t esz = dtype == CSTR_BF16 ? 2 : 4;
+    const int n_slices = batch < CSTR_HOST_SLICES ? batch : CSTR_HOST_SLICES;
+    const int per = (batch + n_slices - 1) / n_slices;
+    for (int i = 0, r0 = 0; r0 < batch; ++i, r0 += per) {
+        const int rows = batch - r0 < per ? batch - r0 : per;
+        const size_t off = (size_t)r0 * (size_t)ld;
+        CSTR_CUDA_TRY(cudaMemcpyAsync((char *)logits_dev + off * esz,
+                                      (const char *)logits_host + off * esz,
+                                      (size_t)rows * (size_t)ld * esz, cudaMemcpyHostToDevice,
+                                      ws->copy_stream));
+        if (noise_host)
+            CSTR_CUDA_TRY(cudaMemcpyAsync(noise_dev + off, noise_host + off,
+                                          (size_t)rows * (size_t)ld * 4, cudaMemcpyHostToDevice,
+                                          ws->copy_stream));
+        CSTR_CUDA_TRY(cudaEventRecord(ws->slice_ready[i], ws->copy_stream));
+        CSTR_CUDA_TRY(cudaStreamWaitEvent(stream, ws->slice_ready[i], 0));
+        cstr_workspace sub = *ws;                // this slice's rows of the scratch
+        sub.cell += r0;
+        sub.ticket += r0;
+        sub.max_batch = rows;
+        rc = step_common(tables, n_tables, row_table ? row_table + r0 : nullptr,
+                         (const char *)logits_dev + off * esz, dtype, ld,
+                         noise_dev ? noise_dev + off : nullptr, states + r0, states + r0,
+                         tokens_dev + r0, (char *)masked_out + off * esz,
+                         accept_out ? accept_out + r0 : nullptr, rows, &sub, stream);
+        if (rc) {
+            cudaStreamSynchronize(ws->copy_stream);
+            cudaStreamSynchronize(stream);
+            return rc;
+        }
+    }
+    CSTR_CUDA_TRY(cudaMemcpyAsync(tokens_host, tokens_dev, (size_t)batch * 4, cudaMemcpyDeviceToHost,
+                                  stream));
+    if (states_host)
+        CSTR_CUDA_TRY(cudaMemcpyAsync(states_host, states, (size_t)batch * 4, cudaMemcpyDeviceToHost,
+                                      stream));
+    CSTR_CUDA_TRY(cudaStreamSynchronize(stream));
+    return CSTR_OK;
 }
 
 extern "C" int cstr_accept_draft(const int32_t *draft_tokens, const int32_t *target_tokens,

@@ -7,6 +7,7 @@
 #include "cstr.h"
 
 #define CSTR_DEAD (-1)
+#define CSTR_HOST_SLICES 8       // row slices of cstr_step_host
 
 // Set the calling thread's error message (printf-style) and return `code`.
 int cstr_fail(int code, const char *fmt, ...);
@@ -122,6 +123,12 @@ struct cstr_workspace {
     unsigned long long *cell;      // DEVICE [max_batch] packed (value, index) running maxima
     unsigned int *ticket;          // DEVICE [max_batch] arrival counters
     unsigned long long *counters;  // DEVICE [2] bad-state rows, empty-mask rows
+    // cstr_step_host only (created on its first use): a copy stream and one event
+    // per slice of rows, so that uploads run ahead of the step kernels
+    cudaStream_t copy_stream;
+    cudaEvent_t slice_ready[CSTR_HOST_SLICES];
+    cudaEvent_t inputs_free;
+    int host_ready;
 };
 
 // Byte-level PDA as the kernels read it.  act[(q * NT + t) * 256 + byte] is the

@@ -25,7 +25,7 @@ EXPORTS = [
     "cstr_vocab_set_token_sets", "cstr_free_vocab",
     "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
-    "cstr_step", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
+    "cstr_step", "cstr_step_host", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
     "cstr_step_static", "cstr_last_error",
     "cstr_load_pda", "cstr_free_pda", "cstr_build_pda_table", "cstr_free_pda_table",
     "cstr_pda_table_rebuild", "cstr_pda_table_info", "cstr_pda_table_download",
@@ -274,6 +274,51 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
                                        _dev_ptr(tokens_out), _dev_ptr(masked_out),
                                        _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
                                        _stream_ptr(stream)))
+
+
+def cstr_step_host(tables, logits_host, states, tokens_host, logits_dev, masked_out, tokens_dev,
+                   ws: Workspace, states_host=None, noise_host=None, noise_dev=None, row_table=None,
+                   accept_out=None, stream=None) -> None:
+    """``cstr_step`` for logits in host memory (synchronous).  ``logits_host`` /
+    ``noise_host`` / ``tokens_host`` / ``states_host`` are CPU tensors (pinned for speed),
+    ``logits_dev`` / ``noise_dev`` device staging tensors of the same shapes, the rest as
+    in ``cstr_step``."""
+    import torch
+    if isinstance(tables, Table):
+        tables = [tables]
+    if logits_host.dtype == torch.float32:
+        dtype = CSTR_F32
+    elif logits_host.dtype == torch.bfloat16:
+        dtype = CSTR_BF16
+    else:
+        raise TypeError("logits must be float32 or bfloat16")
+    if logits_host.is_cuda or logits_host.dim() != 2 or not logits_host.is_contiguous():
+        raise ValueError("logits_host must be a contiguous CPU tensor [B][ld]")
+    batch, ld = logits_host.shape
+    for name, t in (("logits_dev", logits_dev), ("masked_out", masked_out)):
+        if not t.is_cuda or t.dtype != logits_host.dtype or tuple(t.shape) != (batch, ld) \
+                or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous CUDA tensor shaped like logits_host" % name)
+    if (noise_host is None) != (noise_dev is None):
+        raise ValueError("noise_host and noise_dev go together")
+    if noise_host is not None:
+        for name, t, cuda in (("noise_host", noise_host, False), ("noise_dev", noise_dev, True)):
+            if t.is_cuda != cuda or t.dtype != torch.float32 or tuple(t.shape) != (batch, ld) \
+                    or not t.is_contiguous():
+                raise ValueError("%s must be a contiguous float32 tensor [B][ld]" % name)
+    for name, t, cuda in (("states", states, True), ("tokens_dev", tokens_dev, True),
+                          ("tokens_host", tokens_host, False), ("states_host", states_host, False),
+                          ("row_table", row_table, True)):
+        if t is not None and (t.is_cuda != cuda or t.dtype != torch.int32 or t.numel() < batch
+                              or not t.is_contiguous()):
+            raise ValueError("%s must be a contiguous int32 tensor with one entry per row" % name)
+    arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
+    _check(lib().cstr_step_host(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
+                                _dev_ptr(logits_host), ctypes.c_int32(dtype), ctypes.c_int64(ld),
+                                _dev_ptr(noise_host), _dev_ptr(states), _dev_ptr(tokens_host),
+                                _dev_ptr(states_host), _dev_ptr(logits_dev), _dev_ptr(noise_dev),
+                                _dev_ptr(masked_out), _dev_ptr(tokens_dev), _dev_ptr(accept_out),
+                                ctypes.c_int32(batch), ws.ptr, _stream_ptr(stream)))
 
 
 def cstr_step_history(tables, logits, states_in, states_out, tokens_out, masked_out, ws: Workspace,

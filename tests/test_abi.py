@@ -68,6 +68,8 @@ def test_null_and_range_errors(lib):
     assert lib.cstr_workspace_create(0, ctypes.byref(out)) == -2
     assert lib.cstr_step(None, 1, None, None, 0, 0, None, None, None, None, None, 1, None, None) == -1
     assert lib.cstr_step_status(None, None, None, None) == -1
+    assert lib.cstr_step_host(None, 1, None, None, 0, 0, None, None, None, None, None, None, None,
+                              None, None, 1, None, None) == -1
     assert lib.cstr_table_info(None, None, None, None, None) == -1
     # push-down entry points: validation that precedes every CUDA call
     z = np.zeros(2, dtype=np.int32)

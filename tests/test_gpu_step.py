@@ -292,3 +292,43 @@ def test_empty_batch_is_a_no_op():
     cstr.cstr_step_static([table], logits, st, st.clone(), torch.empty_like(logits))
     torch.cuda.synchronize()
     assert cstr.cstr_step_status(ws) == (0, 0)
+
+
+@pytest.mark.parametrize("dtype,gumbel,pinned", [("f32", False, True), ("bf16", True, False)])
+def test_step_host_matches_the_oracle(dtype, gumbel, pinned):
+    # logits in host memory (pinned or pageable), sliced uploads overlapped with the step
+    # kernels: every output as from the oracle, for a batch that does not divide into slices
+    dfa = config_dfas("json_32k")[0]
+    vb, vo = config_vocab("json_32k")
+    V = vo.size - 1
+    (table,) = gpu_tables([dfa], vb, vo)
+    B = 37
+    ws = cstr.cstr_workspace_create(64)
+    rng = np.random.default_rng(3)
+    states = rng.integers(-1, dfa[0].shape[0], size=B).astype(np.int32)
+    for t in range(3):
+        logits = normal_logits(9, t, range(B), V, sigma=2.0, dtype=dtype)
+        noise = gumbel_noise(1, t, range(B), V) if gumbel else None
+        h_logits = torch.from_numpy(logits)
+        h_logits = h_logits.view(torch.bfloat16) if dtype == "bf16" else h_logits
+        h_noise = None if noise is None else torch.from_numpy(noise)
+        if pinned:
+            h_logits = h_logits.pin_memory()
+        d_states = torch.from_numpy(states).to(DEV)
+        h_tok = torch.full((B,), -7, dtype=torch.int32)
+        h_st = torch.full((B,), -7, dtype=torch.int32)
+        d_logits = torch.empty(h_logits.shape, dtype=h_logits.dtype, device=DEV)
+        d_noise = None if noise is None else torch.empty((B, V), device=DEV)
+        d_masked = torch.empty_like(d_logits)
+        d_tok = torch.empty((B,), dtype=torch.int32, device=DEV)
+        d_acc = torch.empty((B,), dtype=torch.uint8, device=DEV)
+        cstr.cstr_step_host([table], h_logits, d_states, h_tok, d_logits, d_masked, d_tok, ws,
+                            states_host=h_st, noise_host=h_noise, noise_dev=d_noise, accept_out=d_acc)
+        ref = oracle.step([dfa], vb, vo, logits, states, noise=noise, threads=8)
+        assert np.array_equal(h_tok.numpy(), ref["tokens"])          # no synchronisation needed
+        assert np.array_equal(h_st.numpy(), ref["states"])
+        assert np.array_equal(d_states.cpu().numpy(), ref["states"])
+        assert np.array_equal(d_acc.cpu().numpy(), ref["accept"])
+        assert bits_equal(from_dev_logits(d_masked), ref["masked"])
+        states = ref["states"]
+    assert cstr.cstr_step_status(ws)[0] == 0
