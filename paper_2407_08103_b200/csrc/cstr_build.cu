@@ -20,6 +20,8 @@
 //     next-state entries with one vector store into the token's row;
 //     validity goes out as NS ballot words per (token, warp), which a second
 //     kernel bit-transposes into the state-major mask the step streams.
+#include <stdlib.h>
+
 #include "cstr_internal.cuh"
 
 namespace {
@@ -357,7 +359,7 @@ apply_terminals_kernel(const int32_t *__restrict__ tstate, const uint32_t *__res
 
 __device__ __forceinline__ unsigned long long class_string_hash(const uint8_t *__restrict__ cls,
                                                                 const uint8_t *__restrict__ b,
-                                                                unsigned n)
+                                                                unsigned n, unsigned long long keep)
 {
     unsigned long long h = 0x9e3779b97f4a7c15ull ^ (unsigned long long)n;
     for (unsigned k = 0; k < n; ++k) {
@@ -367,14 +369,15 @@ __device__ __forceinline__ unsigned long long class_string_hash(const uint8_t *_
     h ^= h >> 32;
     h *= 0xd6e8feb86659fd93ull;
     h ^= h >> 32;
-    return h | 1ull;                                     // 0 marks an empty slot
+    return (h & keep) | 1ull;                            // 0 marks an empty slot
 }
 
 // Each group's slot ends up holding the smallest sorted index of the group.
 __global__ void __launch_bounds__(256)
 group_insert_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
                     const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int i_begin,
-                    int i_end, int eos_id, unsigned long long *key, uint32_t *minv, uint32_t slots)
+                    int i_end, int eos_id, unsigned long long *key, uint32_t *minv, uint32_t slots,
+                    unsigned long long keep)
 {
     const int i = i_begin + blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= i_end)
@@ -383,7 +386,7 @@ group_insert_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ 
     if ((int)tok == eos_id)
         return;                                          // the EOS column is special: never shared
     const uint32_t b0 = off[tok], b1 = off[tok + 1];
-    const unsigned long long h = class_string_hash(cls, bytes + b0, b1 - b0);
+    const unsigned long long h = class_string_hash(cls, bytes + b0, b1 - b0, keep);
     uint32_t slot = (uint32_t)(h >> 20) & (slots - 1);
     for (uint32_t probe = 0; probe < slots; ++probe) {   // slots >= 4 V: an empty slot exists
         unsigned long long seen = *(volatile unsigned long long *)(key + slot);
@@ -404,8 +407,8 @@ __global__ void __launch_bounds__(256)
 group_resolve_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
                      const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int V,
                      int eos_id, const unsigned long long *__restrict__ key,
-                     const uint32_t *__restrict__ minv, uint32_t slots, uint32_t *__restrict__ rep,
-                     uint32_t *__restrict__ reptok)
+                     const uint32_t *__restrict__ minv, uint32_t slots, unsigned long long keep,
+                     uint32_t *__restrict__ rep, uint32_t *__restrict__ reptok)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= V)
@@ -415,7 +418,7 @@ group_resolve_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__
     unsigned rtok = tok;
     if ((int)tok != eos_id) {
         const uint32_t b0 = off[tok], n = off[tok + 1] - b0;
-        const unsigned long long h = class_string_hash(cls, bytes + b0, n);
+        const unsigned long long h = class_string_hash(cls, bytes + b0, n, keep);
         uint32_t slot = (uint32_t)(h >> 20) & (slots - 1);
         for (uint32_t probe = 0; probe < slots; ++probe) {
             const unsigned long long k = key[slot];
@@ -632,19 +635,28 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_key, 0, (size_t)t->group_slots * 8, stream));
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_min, 0xff, (size_t)t->group_slots * 4, stream));
         const unsigned g = (unsigned)((t->V + 255) / 256);
+        // Test hook: CSTR_TEST_GROUP_HASH_BITS=n keeps only n bits of the hash, which forces
+        // collisions and so exercises the exact comparison that makes grouping safe.
+        unsigned long long keep = ~0ull;
+        if (const char *bits = getenv("CSTR_TEST_GROUP_HASH_BITS")) {
+            const int n = atoi(bits);
+            if (n >= 1 && n < 64)
+                keep = (1ull << n) - 1ull;
+        }
         // A small first launch seeds the table: thousands of tokens share a few
         // popular class strings, and once a group's minimum is in place the bulk
         // of the tokens finds it with plain loads instead of same-address atomics.
         const int seed = 4096;
         group_insert_kernel<<<seed / 256, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, 0,
                                                             seed, t->eos_id, t->group_key,
-                                                            t->group_min, t->group_slots);
+                                                            t->group_min, t->group_slots, keep);
         group_insert_kernel<<<(unsigned)((t->V - seed + 255) / 256), 256, 0, stream>>>(
             vc->desc, vc->bytes, vc->off, dfa->cls, seed, t->V, t->eos_id, t->group_key,
-            t->group_min, t->group_slots);
+            t->group_min, t->group_slots, keep);
         group_resolve_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
                                                     t->eos_id, t->group_key, t->group_min,
-                                                    t->group_slots, t->group_rep, t->group_reptok);
+                                                    t->group_slots, keep, t->group_rep,
+                                                    t->group_reptok);
         const int n_blk = (t->V + 1023) / 1024;
         group_count_kernel<<<n_blk, 1024, 0, stream>>>(t->group_rep, t->V, t->group_blk);
         group_scan_kernel<<<1, 1024, 0, stream>>>(t->group_blk, n_blk, t->group_count);

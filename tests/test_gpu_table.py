@@ -250,3 +250,18 @@ def test_load_dfa_reports_bad_targets_and_reuses_its_scratch():
         dfa = dense_random_dfa(rng, S, live=0.8)
         (table,) = gpu_tables([dfa], vb, vo)
         check_table(table, dfa, vb, vo, states=sorted(set([0, S // 2, S - 1])))
+
+
+@pytest.mark.parametrize("bits", [3, 12])
+def test_duplicate_column_pass_survives_hash_collisions(monkeypatch, bits):
+    # with only a few hash bits kept, tokens of different class strings land in the same group;
+    # the exact comparison must then leave them on their own, and the table stays the oracle's
+    from synth import make_vocab_geometric
+    monkeypatch.setenv("CSTR_TEST_GROUP_HASH_BITS", str(bits))
+    vb, vo = make_vocab_geometric(9000, seed=5)
+    dfa = regex_to_dfa(r'"([^"\\]|\\.){0,1100}"')
+    (table,) = gpu_tables([dfa], vb, vo, eos_id=17)
+    S = dfa[0].shape[0]
+    rng = np.random.default_rng(bits)
+    check_table(table, dfa, vb, vo, eos_id=17,
+                states=sorted(set([0, 1, S - 1] + rng.integers(0, S, 20).tolist())))
