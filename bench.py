@@ -208,12 +208,11 @@ def time_oracle_table_build(dfa, vb, vo, budget_s: float = 3.0):
     S, V = int(dfa[0].shape[0]), vo.size - 1
     slab = min(S, 4 * threads)
     oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=0, q_hi=min(S, threads), threads=threads)  # warm
-    done, lo, t0 = 0, 0, time.perf_counter()
-    while done == 0 or time.perf_counter() - t0 < budget_s:
-        hi = min(S, lo + slab)
-        oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=lo, q_hi=hi, threads=threads)
-        done += hi - lo
-        lo = hi if hi < S else 0
+    done, t0 = 0, time.perf_counter()
+    while done < S and (done == 0 or time.perf_counter() - t0 < budget_s):
+        hi = min(S, done + slab)
+        oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=done, q_hi=hi, threads=threads)
+        done = hi
     dt = time.perf_counter() - t0
     return {"value": done * V / dt, "unit": "transitions/s", "cores": threads, "kind": "oracle",
             "sample": "%d of %d states x %d tokens of %s in %.1f s (whole table extrapolates to "
@@ -617,9 +616,13 @@ def main():
         return reduce_max(x, world, dev)
 
     # ---- set-up: vocabulary, DFA, table (the table build is timed below) ----
-    t_v0 = time.perf_counter()
-    vocab = cstr.cstr_load_vocab(vb, vo)
-    vocab_load_ms = (time.perf_counter() - t_v0) * 1e3   # once per LM: sort, descriptors, upload
+    torch.zeros(1, device=dev)                     # CUDA context and module load are not the vocabulary's cost
+    vocab_load_ms = []
+    for _ in range(2):                             # once per LM: sort, descriptors, upload
+        t_v0 = time.perf_counter()
+        vocab = cstr.cstr_load_vocab(vb, vo)
+        vocab_load_ms.append((time.perf_counter() - t_v0) * 1e3)
+    vocab_load_ms = min(vocab_load_ms)
     h_dfa = cstr.cstr_load_dfa(*dfa)
     table = cstr.cstr_table_create(vocab, S)
     build_ms = []
