@@ -265,3 +265,25 @@ def test_duplicate_column_pass_survives_hash_collisions(monkeypatch, bits):
     rng = np.random.default_rng(bits)
     check_table(table, dfa, vb, vo, eos_id=17,
                 states=sorted(set([0, 1, S - 1] + rng.integers(0, S, 20).tolist())))
+
+
+@pytest.mark.parametrize("n_states", [32766, 32767])
+def test_entry_width_boundary(n_states):
+    # 32,766 states are the most that 16-bit entries hold (the sink takes one more code);
+    # one state more switches the DFA and the table to 32-bit entries
+    trans = np.full((n_states, 256), -1, dtype=np.int32)
+    q = np.arange(n_states - 1)
+    trans[q, 0x61] = q + 1                          # a chain on 'a' ...
+    trans[:, 0x62] = np.arange(n_states)[::-1]      # ... and 'b' jumps to the mirrored state
+    acc = np.zeros(n_states, dtype=np.uint8)
+    acc[-1] = 1
+    dfa = (trans, acc, 0)
+    toks = [b"a", b"aa", b"b", b"ab", b"ba", b"bab", b"c", b"", b"a" * 40, b"aba" * 5] + \
+           [bytes([c]) for c in range(256)]
+    vb, vo = vocab_from_strings(toks)
+    (table,) = gpu_tables([dfa], vb, vo, eos_id=6)
+    S = n_states
+    check_table(table, dfa, vb, vo, eos_id=6,
+                states=[0, 1, 2, 255, 256, 16383, 16384, S - 42, S - 41, S - 3, S - 2, S - 1])
+    nxt, _ = cstr.cstr_table_download(table, S - 2, S)
+    assert nxt[0, 0] == S - 1 and nxt[1, 0] == -1 and nxt[1, 2] == 0
