@@ -335,8 +335,10 @@ void cstr_free_pda(cstr_pda_t *pda);
  *     deep[q][X] bit v = whether v has an edge depends on symbols below X
  *                        (cstr_pda_step decides those against the row's stack)
  * If eos_id >= 0 that token is allowed exactly in accepting states.
- * `pda` and `vocab` must outlive the table.  Tokens longer than
- * 255 / (largest push of an edge) bytes are rejected with CSTR_ERR_SHAPE.
+ * `pda` and `vocab` must outlive the table.  Limits (CSTR_ERR_SHAPE): at most
+ * 65,535 situations (states x (symbols + 1)); no token longer than
+ * 255 / (largest push of an edge) bytes.  Device memory: two rows of
+ * ceil(V / 32) words per situation and per state.
  * Allocates the table; the build kernel is enqueued on cuda_stream.
  */
 int cstr_build_pda_table(const cstr_pda_t *pda, const cstr_vocab_t *vocab, int32_t eos_id,
