@@ -263,23 +263,36 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
     // one padding word per 32 tokens: lane l then reads word 33 l + r, free of bank conflicts
     __shared__ uint32_t tile[8][1024 + 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // x = group of 8 ballot words, y = group of 32 mask words: CTAs that read
-    // the four 32-byte quarters of the same maskT lines are launched together
-    const int sb0 = blockIdx.x * 8;
-    const int w0 = blockIdx.y * 32;
-    for (int t = threadIdx.x; t < 1024; t += 256) {
-        const long long tokid = (long long)w0 * 32 + t;
-        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-        if (tokid < V) {
-            // after a duplicate-column pass only the representatives' rows were written
-            const long long rowid = reptok ? (long long)__ldg(reptok + tokid) : tokid;
-            const uint4 *src = (const uint4 *)(maskT + rowid * ldb + sb0);   // ldb, sb0 multiples of 8
-            a = __ldg(src);
-            b = __ldg(src + 1);
+    // x = group of 32 mask words, y = group of 8 ballot words: CTAs launched
+    // together write neighbouring 128-byte pieces of the same mask rows (the four
+    // CTAs that read the 32-byte quarters of one maskT line meet again in L2)
+    const int w0 = blockIdx.x * 32;
+    const int sb0 = blockIdx.y * 8;
+    // four tokens per thread; all row indices first, then all row loads, so that
+    // the dependent loads of the four tokens overlap
+    long long rowid[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const long long tokid = (long long)w0 * 32 + threadIdx.x + 256 * k;
+        // after a duplicate-column pass only the representatives' rows were written
+        rowid[k] = tokid < V ? (reptok ? (long long)__ldg(reptok + tokid) : tokid) : -1;
+    }
+    uint4 lo[4], hi[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        lo[k] = hi[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (rowid[k] >= 0) {
+            const uint4 *src = (const uint4 *)(maskT + rowid[k] * ldb + sb0);   // ldb, sb0 multiples of 8
+            lo[k] = __ldg(src);
+            hi[k] = __ldg(src + 1);
         }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int t = threadIdx.x + 256 * k;
         const int at = t + (t >> 5);
-        tile[0][at] = a.x; tile[1][at] = a.y; tile[2][at] = a.z; tile[3][at] = a.w;
-        tile[4][at] = b.x; tile[5][at] = b.y; tile[6][at] = b.z; tile[7][at] = b.w;
+        tile[0][at] = lo[k].x; tile[1][at] = lo[k].y; tile[2][at] = lo[k].z; tile[3][at] = lo[k].w;
+        tile[4][at] = hi[k].x; tile[5][at] = hi[k].y; tile[6][at] = hi[k].z; tile[7][at] = hi[k].w;
     }
     __syncthreads();
     const int sbw = sb0 + warp;
@@ -776,9 +789,9 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
             (int)(used * nt / 16));
         CSTR_CUDA_TRY(cudaGetLastError());
     }
-    dim3 tgrid((unsigned)((ballot_words + 7) / 8), (unsigned)(t->ldw / 32));
+    dim3 tgrid((unsigned)(t->ldw / 32), (unsigned)((ballot_words + 7) / 8));
     if (tgrid.y > 65535u)
-        return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: vocabulary too large for one launch");
+        return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: too many states for one launch");
     mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
                                                      ns, p.reptok);
     CSTR_CUDA_TRY(cudaGetLastError());
