@@ -303,9 +303,25 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
 #pragma unroll
     for (int r = 0; r < 32; ++r)
         x[r] = tile[warp][33 * lane + r];
-    uint32_t m = 0x0000ffffu;
+    // 32 x 32 bit transpose by block swaps of 16, 8, 4, 2 and 1 bits; the two
+    // coarse stages move whole bytes, which is one byte permute per word
 #pragma unroll
-    for (int j = 16; j >= 1; j >>= 1) {
+    for (int k = 0; k < 16; ++k) {
+        const uint32_t a = x[k], b = x[k + 16];
+        x[k] = __byte_perm(a, b, 0x5410);            // low half of a, low half of b
+        x[k + 16] = __byte_perm(a, b, 0x7632);       // high half of a, high half of b
+    }
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+        if ((k & 8) == 0) {
+            const uint32_t a = x[k], b = x[k + 8];
+            x[k] = __byte_perm(a, b, 0x6240);        // bytes a0 b0 a2 b2
+            x[k + 8] = __byte_perm(a, b, 0x7351);    // bytes a1 b1 a3 b3
+        }
+    }
+    uint32_t m = 0x0f0f0f0fu;
+#pragma unroll
+    for (int j = 4; j >= 1; j >>= 1) {
 #pragma unroll
         for (int k = 0; k < 32; ++k) {
             if ((k & j) == 0) {
