@@ -485,6 +485,41 @@ def time_build_only(torch, cstr, name, case, stream, repeats=4):
             "frac_of_hbm_peak": gbs / peak, "peak_kind": "of %s" % kind}
 
 
+def time_small_compiles(torch, cstr, vocab, stream):
+    """Compile cost of small constraints over the 256k vocabulary (the regime of the
+    paper's Table 1: one small regex against a large vocabulary): table build
+    kernels alone, and DFA load + build end to end on the host clock."""
+    from synth import constraints
+    from synth.regex_frontend import regex_to_dfa
+    pats = dict(constraints.SMALL_CONSTRAINTS)
+    pats["api_call"] = constraints.API_CALL_REGEX
+    pats["flat_json"] = constraints.FLAT_JSON_REGEX
+    out = []
+    for name, pat in pats.items():
+        dfa = regex_to_dfa(pat)
+        S = int(dfa[0].shape[0])
+        h = cstr.cstr_load_dfa(*dfa)
+        t = cstr.cstr_table_create(vocab, S)
+        ms = []
+        for _ in range(4):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            cstr.cstr_table_build(t, h, -1, stream)
+            a1.record(stream)
+            a1.synchronize()
+            ms.append(a0.elapsed_time(a1))
+        e2e = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            h2 = cstr.cstr_load_dfa(*dfa)
+            cstr.cstr_table_build(t, h2, -1, stream)
+            torch.cuda.synchronize()
+            e2e.append((time.perf_counter() - t0) * 1e3)
+        out.append({"constraint": name, "dfa_states": S, "build_ms": float(np.mean(ms[1:])),
+                    "dfa_load_plus_build_ms": float(min(e2e))})
+    return out
+
+
 def time_small_batches(torch, cstr, table, V, dev, stream, batches=(1, 8, 64)):
     """Step latency for small batches at the full vocabulary (fp32, greedy): 64
     steps captured in one CUDA graph, logits rotating through a pool larger than
@@ -775,6 +810,10 @@ def main():
     if rank == 0 and world == 1 and not args.skip_other_workloads and args.case == "full":
         small = time_small_batches(torch, cstr, table, V, dev, stream)
 
+    small_compiles = None
+    if not args.skip_build_bench and rank == 0 and args.case == "full":
+        small_compiles = time_small_compiles(torch, cstr, vocab, stream)
+
     wildcard = None
     if not args.skip_build_bench and rank == 0 and args.case == "full":
         wildcard = time_wildcard_build(torch, cstr, vocab, vb, vo, stream, measured_hbm_peak()[0])
@@ -864,6 +903,7 @@ def main():
         "dfa_load_ms": dfa_load_ms,
         "vocab_load_ms": vocab_load_ms,
         "wildcard_table_build": wildcard,
+        "small_constraint_compiles": small_compiles,
         "speculative_verify": spec,
         "pushdown_step": pushdown,
         "small_batch_step_latency": small,

@@ -30,6 +30,15 @@ FLAT_JSON_REGEX = (
 STRING_LITERAL_REGEX = r'"([^"\\]|\\.){0,4096}"'
 
 
+# Small constraints of the kinds the paper times in its Table 1 (a multiple-choice answer, an
+# ISO date-time, an IPv4 address), written here from their usual definitions.
+SMALL_CONSTRAINTS = {
+    "multiple_choice": r"(A|B|C|D)",
+    "iso_date_time": r"[0-9]{4}-[0-9]{2}-[0-9]{2}T[0-9]{2}:[0-9]{2}:[0-9]{2}(Z|[+-][0-9]{2}:[0-9]{2})",
+    "ipv4_address": r"((25[0-5]|2[0-4][0-9]|1?[0-9]?[0-9])\.){3}(25[0-5]|2[0-4][0-9]|1?[0-9]?[0-9])",
+}
+
+
 def schema40_regex(seed: int = 0, n_keys: int = 40) -> str:
     """JSON object with ``n_keys`` required keys k00.. in fixed order; value
     types cycle string / integer / true|false / enum of 8 seeded random
