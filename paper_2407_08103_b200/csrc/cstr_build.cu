@@ -591,6 +591,85 @@ expand_rows_kernel(const uint32_t *__restrict__ reptok, unsigned char *__restric
         __stcs(dst + k, __ldg(src + k));
 }
 
+// ---- small automata ----------------------------------------------------------
+//
+// With a handful of states the lane = state walker uses a fraction of its lanes
+// and its per-token cost is all bookkeeping.  Here a lane owns a token instead and walks it from every state
+// in turn, eight at a time: the byte classes of the token's first 16 bytes sit in registers,
+// the class-major DFA table in shared memory, eight results at a time leave as
+// one 16-byte store into the token's row of next, and the validity of a state
+// over the warp's 32 tokens is one ballot = one word of mask, so no transpose
+// pass is needed.  16-bit tables only.
+constexpr int kSmallStates = 16;     // beyond this the trie walker's shared prefixes win (measured)
+
+__global__ void __launch_bounds__(256)
+build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restrict__ cls,
+                   const uint8_t *__restrict__ accept, const uint8_t *__restrict__ bytes,
+                   const uint32_t *__restrict__ off, unsigned short *__restrict__ next,
+                   uint32_t *__restrict__ mask, unsigned lds, long long ldw, int row, int n_states,
+                   int n_classes, int V, int W, int eos_id)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][row]
+    uint8_t *s_cls = smem + (size_t)n_classes * row * 2;      // [256]
+    for (int i = threadIdx.x; i < n_classes * row / 8; i += blockDim.x)
+        ((uint4 *)s_tt)[i] = __ldg((const uint4 *)tt + i);    // row is a multiple of 256 entries
+    for (int i = threadIdx.x; i < 256; i += blockDim.x)
+        s_cls[i] = cls[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (w >= W)
+        return;
+    const int v = w * 32 + lane;
+    const bool in = v < V;
+    const uint32_t b0 = in ? off[v] : 0u;
+    const int len = in ? (int)(off[v + 1] - b0) : 0;
+    const bool is_eos = in && v == eos_id;
+    unsigned long long c_lo = 0ull, c_hi = 0ull;              // classes of bytes 0..7 and 8..15
+    for (int k = 0; k < len && k < 16; ++k) {
+        const unsigned long long c = (unsigned long long)s_cls[bytes[b0 + k]] << (8 * (k & 7));
+        if (k < 8)
+            c_lo |= c;
+        else
+            c_hi |= c;
+    }
+    const unsigned sink = (unsigned)CSTR_PERM(n_states) * 2u;
+    const unsigned row_bytes = (unsigned)row * 2u;
+    const unsigned char *tb = (const unsigned char *)s_tt;
+    unsigned short *out = next + (unsigned long long)(in ? v : 0) * lds;
+    const bool walks = in && len > 0 && !is_eos;
+    for (int q0 = 0; q0 < n_states; q0 += 8) {
+        // eight states side by side: one class extraction per byte, eight
+        // independent shared-memory lookups (the sink maps to itself)
+        unsigned cur[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            cur[j] = (walks && q0 + j < n_states) ? (unsigned)CSTR_PERM(q0 + j) * 2u : sink;
+        if (walks) {
+            for (int k = 0; k < len; ++k) {
+                const unsigned c = k < 16 ? (unsigned)((k < 8 ? c_lo : c_hi) >> (8 * (k & 7))) & 0xffu
+                                          : (unsigned)s_cls[bytes[b0 + k]];
+                const unsigned char *rowp = tb + c * row_bytes;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    cur[j] = *(const unsigned short *)(rowp + cur[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int q = q0 + j;
+            const bool ok = is_eos ? (q < n_states && accept[q] != 0) : cur[j] != sink;
+            const unsigned word = __ballot_sync(kFull, in && ok);
+            if (lane == 0 && q < n_states)
+                mask[(long long)q * ldw + w] = word;
+        }
+        if (in)                                                // lds is a multiple of 256 entries
+            *(uint4 *)(out + q0) = make_uint4(cur[0] | (cur[1] << 16), cur[2] | (cur[3] << 16),
+                                              cur[4] | (cur[5] << 16), cur[6] | (cur[7] << 16));
+    }
+}
+
 template <typename ST, typename NT, int NS, bool SMEM>
 cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
                         cudaStream_t stream)
@@ -629,6 +708,28 @@ cudaError_t launch_trie_ns(int ns, bool in_smem, const BuildParams &p, dim3 grid
 
 }  // namespace
 
+// Post-pass for automata with terminal-label edges (no-op otherwise).
+static int launch_terminals(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
+{
+    const cstr_vocab *vc = t->vocab;
+    const int S = dfa->n_states;
+    if (dfa->n_term_states > 0) {
+        const unsigned sink = (unsigned)CSTR_PERM(S) << (dfa->wide ? 2 : 1);
+        const unsigned agrid = (unsigned)((t->V + 255) / 256);
+        if (t->wide)
+            apply_terminals_kernel<uint32_t><<<agrid, 256, 0, stream>>>(
+                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
+                vc->off, t->V, t->eos_id, sink, (uint32_t *)t->next, t->lds, t->mask, t->ldw);
+        else
+            apply_terminals_kernel<uint16_t><<<agrid, 256, 0, stream>>>(
+                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
+                vc->off, t->V, t->eos_id, sink & 0xffffu, (uint16_t *)t->next, t->lds, t->mask,
+                t->ldw);
+        CSTR_CUDA_TRY(cudaGetLastError());
+    }
+    return CSTR_OK;
+}
+
 int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
 {
     const cstr_vocab *vc = t->vocab;
@@ -652,6 +753,22 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     if (dfa->wide && !t->wide)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
     const size_t st = dfa->wide ? 4 : 2;
+
+    // Small automata: one lane per token, all states in turn, mask words by ballot.
+    const size_t small_smem = (size_t)dfa->n_classes * (size_t)dfa->row * 2 + 256;
+    if (!dfa->wide && !t->wide && dfa->n_states <= kSmallStates && small_smem <= 160 * 1024) {
+        if (small_smem > 48 * 1024)
+            CSTR_CUDA_TRY(cudaFuncSetAttribute(build_small_kernel,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)small_smem));
+        const int warps = 8;
+        build_small_kernel<<<(unsigned)((t->W + warps - 1) / warps), warps * 32, small_smem, stream>>>(
+            (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off,
+            (unsigned short *)t->next, t->mask, (unsigned)t->lds, t->ldw, (int)dfa->row,
+            dfa->n_states, dfa->n_classes, t->V, t->W, t->eos_id);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        return launch_terminals(t, dfa, stream);
+    }
 
     // Duplicate-column pass for large automata with few byte classes over a large
     // vocabulary (elsewhere class strings rarely repeat, or the walk is too short
@@ -812,19 +929,5 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
                                                      ns, p.reptok);
     CSTR_CUDA_TRY(cudaGetLastError());
 
-    if (dfa->n_term_states > 0) {
-        const unsigned sink = (unsigned)CSTR_PERM(S) << (dfa->wide ? 2 : 1);
-        const unsigned agrid = (unsigned)((t->V + 255) / 256);
-        if (t->wide)
-            apply_terminals_kernel<uint32_t><<<agrid, 256, 0, stream>>>(
-                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
-                vc->off, t->V, t->eos_id, sink, (uint32_t *)t->next, t->lds, t->mask, t->ldw);
-        else
-            apply_terminals_kernel<uint16_t><<<agrid, 256, 0, stream>>>(
-                dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
-                vc->off, t->V, t->eos_id, sink & 0xffffu, (uint16_t *)t->next, t->lds, t->mask,
-                t->ldw);
-        CSTR_CUDA_TRY(cudaGetLastError());
-    }
-    return CSTR_OK;
+    return launch_terminals(t, dfa, stream);
 }
