@@ -130,6 +130,7 @@ static int first_bad_target(const int32_t *trans, int32_t n_states)
 // one block per process (at most kScratchKeep bytes, on the device it was last
 // used on); larger requests are allocated and freed per call.
 namespace {
+constexpr int32_t kHostPathStates = 512;   // cstr_load_dfa: at or below, no device pre-processing
 constexpr size_t kScratchKeep = 64u << 20;
 struct ScratchCache {
     int device = -1;
@@ -226,6 +227,69 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     }
     for (int32_t q = 0; q < n_states; ++q)
         flags[q] = accept[q] ? 1 : 0;
+
+    // Small automata: everything on the host (the table is a few hundred KB at
+    // most), two allocations and two uploads instead of a dozen driver calls.
+    if (n_states <= kHostPathStates) {
+        int rc = first_bad_target(trans, n_states);
+        if (rc) {
+            delete d;
+            return rc;
+        }
+        uint8_t cls_h[256], rep_h[256];
+        int nc = 0;
+        for (int b = 0; b < 256; ++b) {              // classes numbered by their smallest byte
+            int found = -1;
+            for (int c = 0; c < nc && found < 0; ++c) {
+                bool same = true;
+                for (int32_t q = 0; q < n_states && same; ++q)
+                    same = trans[(size_t)q * 256 + b] == trans[(size_t)q * 256 + rep_h[c]];
+                if (same)
+                    found = c;
+            }
+            if (found < 0) {
+                found = nc;
+                rep_h[nc++] = (uint8_t)b;
+            }
+            cls_h[b] = (uint8_t)found;
+        }
+        d->n_classes = nc;
+        std::vector<uint16_t> tt_h;                  // n_states <= 32766 here: 16-bit entries
+        std::vector<uint8_t> small_h;
+        try {
+            tt_h.resize((size_t)nc * (size_t)d->row);
+            small_h.resize(256 + (size_t)n_states);
+        } catch (const std::bad_alloc &) {
+            delete d;
+            return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+        }
+        for (int c = 0; c < nc; ++c)
+            for (int64_t q = 0; q < d->row; ++q) {
+                const int32_t t = q < n_states ? trans[(size_t)q * 256 + rep_h[c]] : -1;
+                tt_h[(size_t)c * d->row + CSTR_PERM(q)] =
+                    (uint16_t)(CSTR_PERM(t >= 0 ? t : n_states) * 2);
+            }
+        memcpy(small_h.data(), cls_h, 256);
+        memcpy(small_h.data() + 256, flags.data(), (size_t)n_states);
+        cudaError_t e = cudaGetDevice(&d->device);
+        if (e == cudaSuccess)
+            e = cudaMalloc((void **)&d->cls, small_h.size());
+        d->accept = d->cls ? d->cls + 256 : nullptr;
+        if (e == cudaSuccess)
+            e = cudaMalloc(&d->tt, tt_h.size() * 2);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->cls, small_h.data(), small_h.size(), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(d->tt, tt_h.data(), tt_h.size() * 2, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            rc = cstr_fail(e == cudaErrorMemoryAllocation ? CSTR_ERR_NOMEM : CSTR_ERR_CUDA,
+                           "cstr_load_dfa: %s", cudaGetErrorString(e));
+            cstr_free_dfa(d);
+            return rc;
+        }
+        *out = d;
+        return CSTR_OK;
+    }
 
     // temporaries in one block: [raw table][2 x 256 hashes, mismatch flag, invalid flag][256 reps]
     const size_t raw_bytes = (size_t)n * 4, hash_bytes = 514 * 8;
