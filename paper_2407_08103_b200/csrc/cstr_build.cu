@@ -600,6 +600,7 @@ expand_rows_kernel(const uint32_t *__restrict__ reptok, unsigned char *__restric
 // one 16-byte store into the token's row of next, and the validity of a state
 // over the warp's 32 tokens is one ballot = one word of mask, so no transpose
 // pass is needed.  16-bit tables only.
+constexpr int kLaneTokenStates = 32;   // beyond this the trie walker's shared prefixes win (measured)
 constexpr int kSmallStates = 16;     // beyond this the trie walker's shared prefixes win (measured)
 
 __global__ void __launch_bounds__(256)
@@ -667,6 +668,82 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
         if (in)                                                // lds is a multiple of 256 entries
             *(uint4 *)(out + q0) = make_uint4(cur[0] | (cur[1] << 16), cur[2] | (cur[3] << 16),
                                               cur[4] | (cur[5] << 16), cur[6] | (cur[7] << 16));
+    }
+}
+
+// ---- automata of 17 to 32 states ------------------------------------------------
+//
+// The same lane = token walk for automata of 17 to 32 states, with two changes: a warp takes 32 tokens of EQUAL LENGTH (the vocabulary's
+// by-length order), so no lane idles while a longer neighbour finishes, and a
+// lane keeps its token's validity bits itself - word k of the token's maskT
+// row holds states 32 k .. 32 k + 31 - for the transpose pass (one state per
+// ballot word, NS = 1).  Eight states per round, one class extraction per byte,
+// eight independent shared-memory lookups.
+__global__ void __launch_bounds__(256)
+build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restrict__ cls,
+                        const uint8_t *__restrict__ accept, const uint8_t *__restrict__ bytes,
+                        const uint32_t *__restrict__ off, const uint32_t *__restrict__ by_len,
+                        unsigned short *__restrict__ next, uint32_t *__restrict__ maskT,
+                        unsigned lds, unsigned ldb, int row, int n_states, int n_classes, int V,
+                        int eos_id)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][row]
+    uint8_t *s_cls = smem + (size_t)n_classes * row * 2;      // [256]
+    for (int i = threadIdx.x; i < n_classes * row / 8; i += blockDim.x)
+        ((uint4 *)s_tt)[i] = __ldg((const uint4 *)tt + i);    // row is a multiple of 256 entries
+    for (int i = threadIdx.x; i < 256; i += blockDim.x)
+        s_cls[i] = cls[i];
+    __syncthreads();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool in = i < V;
+    const unsigned v = in ? by_len[i] : 0u;
+    const uint32_t b0 = in ? off[v] : 0u;
+    const int len = in ? (int)(off[v + 1] - b0) : 0;
+    const bool is_eos = in && (int)v == eos_id;
+    unsigned long long c_lo = 0ull, c_hi = 0ull;              // classes of bytes 0..7 and 8..15
+    for (int k = 0; k < len && k < 16; ++k) {
+        const unsigned long long c = (unsigned long long)s_cls[bytes[b0 + k]] << (8 * (k & 7));
+        if (k < 8)
+            c_lo |= c;
+        else
+            c_hi |= c;
+    }
+    const unsigned sink = (unsigned)CSTR_PERM(n_states) * 2u;
+    const unsigned row_bytes = (unsigned)row * 2u;
+    const unsigned char *tb = (const unsigned char *)s_tt;
+    uint32_t *mrow = maskT + (unsigned long long)v * ldb;
+    const bool walks = in && len > 0 && !is_eos;
+    uint32_t bits = 0u;
+    for (int q0 = 0; q0 < n_states; q0 += 8) {
+        unsigned cur[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            cur[j] = (walks && q0 + j < n_states) ? (unsigned)CSTR_PERM(q0 + j) * 2u : sink;
+        if (walks) {
+            for (int k = 0; k < len; ++k) {
+                const unsigned c = k < 16 ? (unsigned)((k < 8 ? c_lo : c_hi) >> (8 * (k & 7))) & 0xffu
+                                          : (unsigned)s_cls[bytes[b0 + k]];
+                const unsigned char *rowp = tb + c * row_bytes;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    cur[j] = *(const unsigned short *)(rowp + cur[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int q = q0 + j;
+            const bool ok = is_eos ? (q < n_states && accept[q] != 0) : cur[j] != sink;
+            bits |= (uint32_t)ok << (q & 31);
+        }
+        if (in && (((q0 + 8) & 31) == 0 || q0 + 8 >= n_states)) {   // a word of 32 states is complete
+            mrow[q0 >> 5] = bits;
+            bits = 0u;
+        }
+        if (in)                                                // lds is a multiple of 256 entries
+            *(uint4 *)(next + (unsigned long long)v * lds + q0) =
+                make_uint4(cur[0] | (cur[1] << 16), cur[2] | (cur[3] << 16), cur[4] | (cur[5] << 16),
+                           cur[6] | (cur[7] << 16));
     }
 }
 
@@ -766,6 +843,27 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
             (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off,
             (unsigned short *)t->next, t->mask, (unsigned)t->lds, t->ldw, (int)dfa->row,
             dfa->n_states, dfa->n_classes, t->V, t->W, t->eos_id);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        return launch_terminals(t, dfa, stream);
+    }
+
+    // A little larger: lane = token over tokens of equal length, then the transpose pass.
+    const int lane_token_states = kLaneTokenStates;
+    const size_t lt_smem = small_smem;
+    if (!dfa->wide && !t->wide && dfa->n_states <= lane_token_states && lt_smem <= 160 * 1024) {
+        if (lt_smem > 48 * 1024)
+            CSTR_CUDA_TRY(cudaFuncSetAttribute(build_lane_token_kernel,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)lt_smem));
+        build_lane_token_kernel<<<(unsigned)((t->V + 255) / 256), 256, lt_smem, stream>>>(
+            (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off, vc->by_len,
+            (unsigned short *)t->next, t->maskT, (unsigned)t->lds, (unsigned)t->ldb, (int)dfa->row,
+            dfa->n_states, dfa->n_classes, t->V, t->eos_id);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        const int words = (dfa->n_states + 31) / 32;
+        dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
+        mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
+                                                      dfa->n_states, t->V, 1, nullptr);
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }

@@ -500,6 +500,7 @@ extern "C" void cstr_free_vocab(cstr_vocab_t *v)
     cudaFree(v->bytes);
     cudaFree(v->off);
     cudaFree(v->desc);
+    cudaFree(v->by_len);
     cudaFree(v->tsets);
     delete v;
 }
@@ -649,6 +650,26 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
         return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_vocab: out of host memory");
     }
     vh->max_len = max_len;
+    // token ids by length (counting sort, stable in the id): a warp that takes 32
+    // consecutive entries walks tokens of the same length
+    std::vector<uint32_t> by_len;
+    try {
+        by_len.resize((size_t)vocab_size);
+        std::vector<uint32_t> start(66, 0u);
+        for (int32_t v = 0; v < vocab_size; ++v) {
+            const uint32_t n = off32[v + 1] - off32[v];
+            ++start[(n < 64 ? n : 64) + 1];
+        }
+        for (int k = 0; k < 65; ++k)
+            start[k + 1] += start[k];
+        for (int32_t v = 0; v < vocab_size; ++v) {
+            const uint32_t n = off32[v + 1] - off32[v];
+            by_len[start[n < 64 ? n : 64]++] = (uint32_t)v;
+        }
+    } catch (const std::bad_alloc &) {
+        delete vh;
+        return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_vocab: out of host memory");
+    }
 
     cudaError_t e = cudaGetDevice(&vh->device);
     if (e == cudaSuccess)
@@ -657,6 +678,11 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
         e = cudaMalloc((void **)&vh->off, ((size_t)vocab_size + 1) * sizeof(uint32_t));
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&vh->desc, (size_t)vocab_size * sizeof(uint4));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->by_len, (size_t)vocab_size * sizeof(uint32_t));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(vh->by_len, by_len.data(), by_len.size() * sizeof(uint32_t),
+                       cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMemset(vh->bytes, 0, (size_t)total + 16);
     if (e == cudaSuccess && total > 0)

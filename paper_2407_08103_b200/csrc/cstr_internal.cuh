@@ -75,6 +75,7 @@ struct cstr_vocab {
     uint4 *desc;       // DEVICE [V], sorted order
     uint32_t max_len;
     int32_t n_labels;  // terminal labels with a token set (0 = none attached)
+    uint32_t *by_len;  // DEVICE [V] token ids ordered by length (then id): warps of equal-length tokens
     uint32_t *tsets;   // DEVICE [V] bit t: token belongs to label t's set
 };
 

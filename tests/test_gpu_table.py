@@ -287,3 +287,17 @@ def test_entry_width_boundary(n_states):
                 states=[0, 1, 2, 255, 256, 16383, 16384, S - 42, S - 41, S - 3, S - 2, S - 1])
     nxt, _ = cstr.cstr_table_download(table, S - 2, S)
     assert nxt[0, 0] == S - 1 and nxt[1, 0] == -1 and nxt[1, 2] == 0
+
+
+@pytest.mark.parametrize("S", [4, 16, 17, 25, 32, 33])
+def test_small_automaton_kernels(S):
+    # up to 16 states: lane = token with ballots; 17..32: lane = token over tokens of equal
+    # length + transpose; 33: the trie walker.  Long tokens, empty tokens, an EOS token.
+    rng = np.random.default_rng(S)
+    dfa = dense_random_dfa(rng, S, live=0.85)
+    vb, vo = random_vocab(rng, 1500 + S, max_len=40)
+    eos = int(rng.integers(vo.size - 1))
+    (table,) = gpu_tables([dfa], vb, vo, eos_id=eos)
+    check_table(table, dfa, vb, vo, eos_id=eos)
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo)
