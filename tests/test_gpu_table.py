@@ -132,6 +132,21 @@ def test_config_256k_sampled_states(name):
     assert np.array_equal(live, pop)
 
 
+def test_small_constraints_over_the_256k_vocabulary():
+    # The small-constraint compiles the benchmark times (2 to 56 states over 256,000 tokens:
+    # the lane = token kernels and the smallest trie-walker variant), whole tables.
+    from synth import constraints
+    vb, vo = config_vocab("string_256k")
+    pats = dict(constraints.SMALL_CONSTRAINTS)
+    pats["api_call"] = constraints.API_CALL_REGEX
+    pats["flat_json"] = constraints.FLAT_JSON_REGEX
+    dfas = [regex_to_dfa(p) for p in pats.values()]
+    assert sorted(d[0].shape[0] for d in dfas) == [2, 11, 24, 26, 56]
+    tables = gpu_tables(dfas, vb, vo)
+    for table, dfa in zip(tables, dfas):
+        check_table(table, dfa, vb, vo)
+
+
 def test_long_shared_prefixes_and_long_suffixes():
     # Tokens that share far more than the 8 bytes the walk keeps on its stack,
     # suffixes longer than the 8 bytes carried inline, exact duplicates, and a
