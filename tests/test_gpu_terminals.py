@@ -70,6 +70,19 @@ def test_summary_bullets_decode():
     assert finished < B          # bullets of wildcard tokens keep most rows alive
 
 
+def test_summary_bullets_table_over_the_256k_vocabulary():
+    # The wildcard build the benchmark times: the same constraint, 256,000 tokens, whole table.
+    dfa, term = split(regex_to_dfa(r"Summary:(\n\* (?P<PARAGRAPH_TOKEN>)+){3,5}", ["PARAGRAPH_TOKEN"]))
+    vb, vo = config_vocab("string_256k")
+    V = vo.size - 1
+    has_nl = np.zeros(V, dtype=bool)
+    pos = np.nonzero(vb == 0x0A)[0]
+    has_nl[np.searchsorted(vo, pos, side="right") - 1] = True
+    sets = (~has_nl).astype(np.uint32)
+    tables = gpu_tables([dfa], vb, vo, term_trans=[term], token_sets=sets)
+    check_table(tables[0], dfa, vb, vo, term_trans=term, token_sets=sets)
+
+
 def test_mixed_tables_with_and_without_labels():
     rng = np.random.default_rng(9)
     vb, vo = random_vocab(rng, 3000, max_len=4)
