@@ -60,7 +60,8 @@ def parse_args():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--build-only", default=None, metavar="WORKLOAD",
                     help="time only the token-table build of one workload (with --case small: the "
-                         "4,099-state string DFA / a 4,096-state random DFA) and print its entry; "
+                         "4,099-state string DFA / a 4,096-state random DFA; small_constraints: the five "
+                         "small-constraint compiles over the 256,000-token vocabulary) and print its entry; "
                          "for profiler captures, not a bench line")
     ap.add_argument("--pushdown-only", action="store_true",
                     help="time only the push-down step leg (batch 128 with --case small) and print "
@@ -624,6 +625,12 @@ def main():
     from synth import normal_logits
     libbuild.build_library()
 
+    if args.build_only == "small_constraints":
+        from synth.configs import config_vocab
+        vb, vo = config_vocab("string_256k")
+        print(json.dumps({"small_constraint_compiles": time_small_compiles(
+            torch, cstr, cstr.cstr_load_vocab(vb, vo), torch.cuda.current_stream())}))
+        return
     if args.build_only:
         print(json.dumps({"table_build": time_build_only(torch, cstr, args.build_only, args.case,
                                                          torch.cuda.current_stream())}))
