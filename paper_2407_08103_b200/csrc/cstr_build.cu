@@ -603,6 +603,37 @@ expand_rows_kernel(const uint32_t *__restrict__ reptok, unsigned char *__restric
 constexpr int kLaneTokenStates = 32;   // beyond this the trie walker's shared prefixes win (measured)
 constexpr int kSmallStates = 16;     // beyond this the trie walker's shared prefixes win (measured)
 
+// Shared-memory table of the lane = token kernels.  The permuted slots of the
+// global table put the states of a small automaton on a handful of banks, and
+// its 512-byte rows put every class on the same ones; 32 lanes looking up
+// unrelated (class, state) entries would collide there.  So a CTA stages a
+// compact copy: entry [c][s], s = 0 .. n_states (the last is the sink), holds
+// 2 x the plain target state, and a row takes an odd number of 32-bit words,
+// which spreads the classes over the banks.  Walks run on these compact codes;
+// a result is turned back into the table's permuted code when it is stored.
+__host__ __device__ inline int compact_stride(int n_states)   // in 16-bit entries
+{
+    return 2 * (((n_states + 2) / 2) | 1);
+}
+
+__device__ __forceinline__ void stage_compact_table(const unsigned short *__restrict__ tt, int row,
+                                                    int n_states, int n_classes,
+                                                    unsigned short *s_tab)
+{
+    const int per = n_states + 1, stride = compact_stride(n_states);
+    for (int i = threadIdx.x; i < n_classes * per; i += blockDim.x) {
+        const int c = i / per, st = i - c * per;
+        const unsigned code = __ldg(tt + (size_t)c * row + CSTR_PERM(st));
+        s_tab[c * stride + st] = (unsigned short)(CSTR_UNPERM(code >> 1) << 1);
+    }
+}
+
+__device__ __forceinline__ unsigned permuted_code(unsigned compact)
+{
+    const unsigned st = compact >> 1;
+    return (unsigned)CSTR_PERM(st) << 1;
+}
+
 __global__ void __launch_bounds__(256)
 build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restrict__ cls,
                    const uint8_t *__restrict__ accept, const uint8_t *__restrict__ bytes,
@@ -611,10 +642,9 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
                    int n_classes, int V, int W, int eos_id)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][row]
-    uint8_t *s_cls = smem + (size_t)n_classes * row * 2;      // [256]
-    for (int i = threadIdx.x; i < n_classes * row / 8; i += blockDim.x)
-        ((uint4 *)s_tt)[i] = __ldg((const uint4 *)tt + i);    // row is a multiple of 256 entries
+    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][compact_stride]
+    uint8_t *s_cls = smem + (size_t)n_classes * compact_stride(n_states) * 2;   // [256]
+    stage_compact_table(tt, row, n_states, n_classes, s_tt);
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
         s_cls[i] = cls[i];
     __syncthreads();
@@ -635,8 +665,8 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
         else
             c_hi |= c;
     }
-    const unsigned sink = (unsigned)CSTR_PERM(n_states) * 2u;
-    const unsigned row_bytes = (unsigned)row * 2u;
+    const unsigned sink = (unsigned)n_states * 2u;
+    const unsigned row_bytes = (unsigned)compact_stride(n_states) * 2u;
     const unsigned char *tb = (const unsigned char *)s_tt;
     unsigned short *out = next + (unsigned long long)(in ? v : 0) * lds;
     const bool walks = in && len > 0 && !is_eos;
@@ -646,7 +676,7 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
         unsigned cur[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            cur[j] = (walks && q0 + j < n_states) ? (unsigned)CSTR_PERM(q0 + j) * 2u : sink;
+            cur[j] = (walks && q0 + j < n_states) ? (unsigned)(q0 + j) * 2u : sink;
         if (walks) {
             for (int k = 0; k < len; ++k) {
                 const unsigned c = k < 16 ? (unsigned)((k < 8 ? c_lo : c_hi) >> (8 * (k & 7))) & 0xffu
@@ -665,6 +695,9 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
             if (lane == 0 && q < n_states)
                 mask[(long long)q * ldw + w] = word;
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            cur[j] = permuted_code(cur[j]);
         if (in)                                                // lds is a multiple of 256 entries
             *(uint4 *)(out + q0) = make_uint4(cur[0] | (cur[1] << 16), cur[2] | (cur[3] << 16),
                                               cur[4] | (cur[5] << 16), cur[6] | (cur[7] << 16));
@@ -688,10 +721,9 @@ build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__
                         int eos_id)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][row]
-    uint8_t *s_cls = smem + (size_t)n_classes * row * 2;      // [256]
-    for (int i = threadIdx.x; i < n_classes * row / 8; i += blockDim.x)
-        ((uint4 *)s_tt)[i] = __ldg((const uint4 *)tt + i);    // row is a multiple of 256 entries
+    unsigned short *s_tt = (unsigned short *)smem;            // [n_classes][compact_stride]
+    uint8_t *s_cls = smem + (size_t)n_classes * compact_stride(n_states) * 2;   // [256]
+    stage_compact_table(tt, row, n_states, n_classes, s_tt);
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
         s_cls[i] = cls[i];
     __syncthreads();
@@ -709,8 +741,8 @@ build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__
         else
             c_hi |= c;
     }
-    const unsigned sink = (unsigned)CSTR_PERM(n_states) * 2u;
-    const unsigned row_bytes = (unsigned)row * 2u;
+    const unsigned sink = (unsigned)n_states * 2u;
+    const unsigned row_bytes = (unsigned)compact_stride(n_states) * 2u;
     const unsigned char *tb = (const unsigned char *)s_tt;
     uint32_t *mrow = maskT + (unsigned long long)v * ldb;
     const bool walks = in && len > 0 && !is_eos;
@@ -719,7 +751,7 @@ build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__
         unsigned cur[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            cur[j] = (walks && q0 + j < n_states) ? (unsigned)CSTR_PERM(q0 + j) * 2u : sink;
+            cur[j] = (walks && q0 + j < n_states) ? (unsigned)(q0 + j) * 2u : sink;
         if (walks) {
             for (int k = 0; k < len; ++k) {
                 const unsigned c = k < 16 ? (unsigned)((k < 8 ? c_lo : c_hi) >> (8 * (k & 7))) & 0xffu
@@ -740,6 +772,9 @@ build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__
             mrow[q0 >> 5] = bits;
             bits = 0u;
         }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            cur[j] = permuted_code(cur[j]);
         if (in)                                                // lds is a multiple of 256 entries
             *(uint4 *)(next + (unsigned long long)v * lds + q0) =
                 make_uint4(cur[0] | (cur[1] << 16), cur[2] | (cur[3] << 16), cur[4] | (cur[5] << 16),
@@ -832,12 +867,10 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     const size_t st = dfa->wide ? 4 : 2;
 
     // Small automata: one lane per token, all states in turn, mask words by ballot.
-    const size_t small_smem = (size_t)dfa->n_classes * (size_t)dfa->row * 2 + 256;
-    if (!dfa->wide && !t->wide && dfa->n_states <= kSmallStates && small_smem <= 160 * 1024) {
-        if (small_smem > 48 * 1024)
-            CSTR_CUDA_TRY(cudaFuncSetAttribute(build_small_kernel,
-                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)small_smem));
+    const size_t small_smem =          // at most 256 x 34 x 2 + 256 bytes
+        dfa->n_states <= kLaneTokenStates
+            ? (size_t)dfa->n_classes * (size_t)compact_stride(dfa->n_states) * 2 + 256 : 0;
+    if (!dfa->wide && !t->wide && dfa->n_states <= kSmallStates) {
         const int warps = 8;
         build_small_kernel<<<(unsigned)((t->W + warps - 1) / warps), warps * 32, small_smem, stream>>>(
             (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off,
@@ -850,11 +883,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     // A little larger: lane = token over tokens of equal length, then the transpose pass.
     const int lane_token_states = kLaneTokenStates;
     const size_t lt_smem = small_smem;
-    if (!dfa->wide && !t->wide && dfa->n_states <= lane_token_states && lt_smem <= 160 * 1024) {
-        if (lt_smem > 48 * 1024)
-            CSTR_CUDA_TRY(cudaFuncSetAttribute(build_lane_token_kernel,
-                                               cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)lt_smem));
+    if (!dfa->wide && !t->wide && dfa->n_states <= lane_token_states) {
         build_lane_token_kernel<<<(unsigned)((t->V + 255) / 256), 256, lt_smem, stream>>>(
             (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off, vc->by_len,
             (unsigned short *)t->next, t->maskT, (unsigned)t->lds, (unsigned)t->ldb, (int)dfa->row,
