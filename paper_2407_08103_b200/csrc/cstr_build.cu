@@ -600,7 +600,7 @@ expand_rows_kernel(const uint32_t *__restrict__ reptok, unsigned char *__restric
 // one 16-byte store into the token's row of next, and the validity of a state
 // over the warp's 32 tokens is one ballot = one word of mask, so no transpose
 // pass is needed.  16-bit tables only.
-constexpr int kLaneTokenStates = 32;   // beyond this the trie walker's shared prefixes win (measured)
+constexpr int kLaneTokenStates = 64;   // beyond this the trie walker's shared prefixes win (measured)
 constexpr int kSmallStates = 16;     // beyond this the trie walker's shared prefixes win (measured)
 
 // Shared-memory table of the lane = token kernels.  The permuted slots of the
@@ -704,9 +704,9 @@ build_small_kernel(const unsigned short *__restrict__ tt, const uint8_t *__restr
     }
 }
 
-// ---- automata of 17 to 32 states ------------------------------------------------
+// ---- automata of 17 to 64 states ------------------------------------------------
 //
-// The same lane = token walk for automata of 17 to 32 states, with two changes: a warp takes 32 tokens of EQUAL LENGTH (the vocabulary's
+// The same lane = token walk for automata of 17 to 64 states, with two changes: a warp takes 32 tokens of EQUAL LENGTH (the vocabulary's
 // by-length order), so no lane idles while a longer neighbour finishes, and a
 // lane keeps its token's validity bits itself - word k of the token's maskT
 // row holds states 32 k .. 32 k + 31 - for the transpose pass (one state per
@@ -867,7 +867,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     const size_t st = dfa->wide ? 4 : 2;
 
     // Small automata: one lane per token, all states in turn, mask words by ballot.
-    const size_t small_smem =          // at most 256 x 34 x 2 + 256 bytes
+    const size_t small_smem =          // at most 256 x 66 x 2 + 256 bytes
         dfa->n_states <= kLaneTokenStates
             ? (size_t)dfa->n_classes * (size_t)compact_stride(dfa->n_states) * 2 + 256 : 0;
     if (!dfa->wide && !t->wide && dfa->n_states <= kSmallStates) {

@@ -304,10 +304,10 @@ def test_entry_width_boundary(n_states):
     assert nxt[0, 0] == S - 1 and nxt[1, 0] == -1 and nxt[1, 2] == 0
 
 
-@pytest.mark.parametrize("S", [4, 16, 17, 25, 32, 33])
+@pytest.mark.parametrize("S", [4, 16, 17, 25, 32, 33, 64, 65])
 def test_small_automaton_kernels(S):
-    # up to 16 states: lane = token with ballots; 17..32: lane = token over tokens of equal
-    # length + transpose; 33: the trie walker.  Long tokens, empty tokens, an EOS token.
+    # up to 16 states: lane = token with ballots; 17..64: lane = token over tokens of equal
+    # length + transpose; 65: the trie walker.  Long tokens, empty tokens, an EOS token.
     rng = np.random.default_rng(S)
     dfa = dense_random_dfa(rng, S, live=0.85)
     vb, vo = random_vocab(rng, 1500 + S, max_len=40)
