@@ -171,7 +171,9 @@ int cstr_table_info(const cstr_table_t *table, int32_t *n_states, int32_t *vocab
  * form, whatever the device layout is:
  *   mask_host  HOST uint32 [(state_hi-state_lo)][W]      or NULL
  *   next_host  HOST int32  [(state_hi-state_lo)][V]      or NULL   (-1 = no edge)
- * Synchronises cuda_stream first.
+ * Synchronises cuda_stream first and before it returns.  When next_host is
+ * given it allocates (and frees) a device staging buffer of at most 256 MB,
+ * decodes slabs of states into it on cuda_stream and copies them down.
  */
 int cstr_table_download(const cstr_table_t *table, int32_t state_lo, int32_t state_hi,
                         uint32_t *mask_host, int32_t *next_host, void *cuda_stream);

@@ -704,6 +704,46 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
 
 // ---------------------------------------------------------------- table
 
+namespace {
+
+// Logical view of a slab of states for cstr_table_download: out[q - q_lo][v] =
+// state reached from q on token v, -1 for "no edge".  The device table is
+// token-major (next[v][q]) and holds codes (CSTR_PERM(target) << shift, the sink
+// n_states meaning "no edge"), so this is a decode plus a 32 x 32 tiled
+// transpose through shared memory.  Block (32, 8); tile x = 32 tokens, y = 32
+// states starting at a multiple of 32.
+template <typename NT>
+__global__ void __launch_bounds__(256)
+table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo, int rows,
+                    int q_tile0, int n_states, int shift, int32_t *__restrict__ out)
+{
+    __shared__ int32_t tile[32][33];
+    const int v0 = blockIdx.x * 32;
+    const int q0 = (q_tile0 + (int)blockIdx.y) * 32;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int v = v0 + ty + 8 * k, q = q0 + tx;
+        int32_t u = -1;
+        if (v < V && q < n_states) {                     // q < lds: inside the token's row
+            const int32_t code = (int32_t)next[(long long)v * lds + q];
+            u = CSTR_UNPERM(code >> shift);
+            if (u == n_states)
+                u = -1;
+        }
+        tile[ty + 8 * k][tx] = u;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int q = q0 + ty + 8 * k, v = v0 + tx;
+        if (q >= q_lo && q < q_lo + rows && v < V)
+            out[(long long)(q - q_lo) * V + v] = tile[tx][ty + 8 * k];
+    }
+}
+
+}  // namespace
+
 extern "C" void cstr_free_table(cstr_table_t *t)
 {
     if (!t)
@@ -888,33 +928,44 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
                                    cudaMemcpyDeviceToHost));
     }
     if (next_host) {
-        // The device table is token-major; bring the state columns down and
-        // transpose on the host, a slab of states at a time.
-        const size_t esz = t->wide ? 4 : 2;
-        const int32_t slab = 64;
-        std::vector<uint8_t> tmp;
-        try {
-            tmp.resize((size_t)slab * (size_t)t->V * esz);
-        } catch (const std::bad_alloc &) {
-            return cstr_fail(CSTR_ERR_NOMEM, "cstr_table_download: out of host memory");
+        // The device table is token-major and holds codes; a kernel decodes and
+        // transposes a slab of states into the logical layout, which then comes
+        // down as one contiguous copy per slab.
+        const int64_t slab_bytes_max = 256ll << 20;
+        int64_t slab = slab_bytes_max / ((int64_t)t->V * 4);
+        slab = slab < 32 ? 32 : slab / 32 * 32;
+        if (slab > rows)
+            slab = rows;
+        int32_t *stage = nullptr;
+        CSTR_CUDA_TRY(cudaMalloc((void **)&stage, (size_t)slab * (size_t)t->V * 4));
+        cudaError_t e = cudaSuccess;
+        for (int64_t r0 = 0; r0 < rows && e == cudaSuccess; r0 += slab) {
+            const int32_t nr = (int32_t)(rows - r0 < slab ? rows - r0 : slab);
+            const int32_t q_lo = state_lo + (int32_t)r0;
+            // grid x = tiles of 32 tokens, y = tiles of 32 states (tiles start at multiples of 32;
+            // a slab has at most a few hundred of them)
+            const int32_t q_tile0 = q_lo / 32;
+            const uint32_t s_tiles = (uint32_t)((q_lo + nr + 31) / 32 - q_tile0);
+            const uint32_t v_tiles = (uint32_t)((t->V + 31) / 32);
+            dim3 grid(v_tiles, s_tiles), block(32, 8);
+            if (t->wide)
+                table_decode_kernel<uint32_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
+                    (const uint32_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
+                    t->code_shift, stage);
+            else
+                table_decode_kernel<uint16_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
+                    (const uint16_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
+                    t->code_shift, stage);
+            e = cudaGetLastError();
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(next_host + r0 * t->V, stage, (size_t)nr * (size_t)t->V * 4,
+                                    cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream);
+            if (e == cudaSuccess)
+                e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
         }
-        for (int32_t r0 = 0; r0 < rows; r0 += slab) {
-            const int32_t nr = rows - r0 < slab ? rows - r0 : slab;
-            CSTR_CUDA_TRY(cudaMemcpy2D(tmp.data(), (size_t)nr * esz,
-                                       (const uint8_t *)t->next + (size_t)(state_lo + r0) * esz,
-                                       (size_t)t->lds * esz, (size_t)nr * esz, (size_t)t->V,
-                                       cudaMemcpyDeviceToHost));
-            for (int32_t v = 0; v < t->V; ++v) {
-                for (int32_t r = 0; r < nr; ++r) {
-                    const size_t at = (size_t)v * nr + r;
-                    const int32_t x = t->wide ? ((const int32_t *)tmp.data())[at]
-                                              : (int32_t)((const uint16_t *)tmp.data())[at];
-                    // device entries are codes of permuted ids; the sink n_states means "no edge"
-                    const int32_t u = CSTR_UNPERM(x >> t->code_shift);
-                    next_host[(int64_t)(r0 + r) * t->V + v] = (u == t->n_states) ? -1 : u;
-                }
-            }
-        }
+        cudaFree(stage);
+        if (e != cudaSuccess)
+            return cstr_fail(CSTR_ERR_CUDA, "cstr_table_download: %s", cudaGetErrorString(e));
     }
     return CSTR_OK;
 }

@@ -227,6 +227,45 @@ def cstr_workspace_create(max_batch: int) -> Workspace:
     return Workspace(out)
 
 
+def _step_tensor_checks(logits, masked_out, noise, per_row, vocab_ld=None):
+    """Argument checks shared by the step wrappers; returns ``(dtype code, ld, batch)``.
+
+    ``per_row`` lists ``(name, tensor or None, torch dtype)`` for the arrays that hold
+    one entry per row.  Every check runs before anything is handed to the library: a
+    short or wrongly typed per-row tensor would otherwise become an out-of-bounds
+    device write."""
+    import torch
+    if logits.dtype == torch.float32:
+        dtype = CSTR_F32
+    elif logits.dtype == torch.bfloat16:
+        dtype = CSTR_BF16
+    else:
+        raise TypeError("logits must be float32 or bfloat16")
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be [B][ld] with unit inner stride")
+    ld = logits.stride(0) if vocab_ld is None else vocab_ld
+    batch = logits.shape[0]
+    if masked_out is None:
+        raise ValueError("masked_out is required")
+    for name, t in (("masked_out", masked_out), ("noise", noise)):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0)
+                              or t.shape[0] != batch):
+            raise ValueError("%s must have the layout of logits" % name)
+    if masked_out.dtype != logits.dtype:
+        raise TypeError("masked_out must have the dtype of logits")
+    if noise is not None and noise.dtype != torch.float32:
+        raise TypeError("noise must be float32")
+    for name, t, dt in per_row:
+        if t is not None and (t.dtype != dt or t.numel() < batch or not t.is_contiguous()):
+            raise ValueError("%s must be a contiguous %s tensor with one entry per row" % (name, dt))
+    tensors = [("logits", logits), ("masked_out", masked_out), ("noise", noise)]
+    tensors += [(name, t) for name, t, _ in per_row]
+    for name, t in tensors:
+        if t is not None and (not t.is_cuda or t.device != logits.device):
+            raise ValueError("%s must be a CUDA tensor on the device of logits" % name)
+    return dtype, ld, batch
+
+
 def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noise=None,
               row_table=None, accept_out=None, vocab_ld: int | None = None, stream=None,
               states_out=None) -> None:
@@ -238,28 +277,13 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
     import torch
     if isinstance(tables, Table):
         tables = [tables]
-    if logits.dtype == torch.float32:
-        dtype = CSTR_F32
-    elif logits.dtype == torch.bfloat16:
-        dtype = CSTR_BF16
-    else:
-        raise TypeError("logits must be float32 or bfloat16")
-    if logits.dim() != 2 or logits.stride(1) != 1:
-        raise ValueError("logits must be [B][ld] with unit inner stride")
-    ld = logits.stride(0) if vocab_ld is None else vocab_ld
-    batch = logits.shape[0]
-    for name, t in (("masked_out", masked_out), ("noise", noise)):
-        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0) or t.shape[0] != batch):
-            raise ValueError("%s must have the layout of logits" % name)
-    if masked_out.dtype != logits.dtype:
-        raise TypeError("masked_out must have the dtype of logits")
-    if noise is not None and noise.dtype != torch.float32:
-        raise TypeError("noise must be float32")
-    for name, t, dt in (("states", states, torch.int32), ("states_out", states_out, torch.int32),
-                        ("tokens_out", tokens_out, torch.int32),
-                        ("row_table", row_table, torch.int32), ("accept_out", accept_out, torch.uint8)):
-        if t is not None and (t.dtype != dt or t.numel() < batch or not t.is_contiguous()):
-            raise ValueError("%s must be a contiguous %s tensor with one entry per row" % (name, dt))
+    if states is None or tokens_out is None:
+        raise ValueError("states and tokens_out are required")
+    dtype, ld, batch = _step_tensor_checks(
+        logits, masked_out, noise,
+        (("states", states, torch.int32), ("states_out", states_out, torch.int32),
+         ("tokens_out", tokens_out, torch.int32), ("row_table", row_table, torch.int32),
+         ("accept_out", accept_out, torch.uint8)), vocab_ld)
     arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
     if states_out is None:
         _check(lib().cstr_step(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
@@ -350,29 +374,22 @@ def cstr_step_static(tables, logits, states, tokens_out, masked_out, noise=None,
     """``cstr_step`` for callers that must not allocate: no workspace, the scratch
     is a fixed array inside the library (at most ``CSTR_STATIC_MAX_BATCH`` rows;
     calls that may overlap on the GPU must be ordered by the caller).  Same
-    tensors and results as ``cstr_step``."""
+    tensors, argument checks and results as ``cstr_step``."""
     import torch
     if isinstance(tables, Table):
         tables = [tables]
-    if logits.dtype == torch.float32:
-        dtype = CSTR_F32
-    elif logits.dtype == torch.bfloat16:
-        dtype = CSTR_BF16
-    else:
-        raise TypeError("logits must be float32 or bfloat16")
-    if logits.dim() != 2 or logits.stride(1) != 1:
-        raise ValueError("logits must be [B][ld] with unit inner stride")
-    batch = logits.shape[0]
-    for name, t in (("masked_out", masked_out), ("noise", noise)):
-        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.stride(0) != logits.stride(0)
-                              or t.shape[0] != batch):
-            raise ValueError("%s must have the layout of logits" % name)
+    if states is None or tokens_out is None:
+        raise ValueError("states and tokens_out are required")
+    dtype, ld, batch = _step_tensor_checks(
+        logits, masked_out, noise,
+        (("states", states, torch.int32), ("tokens_out", tokens_out, torch.int32),
+         ("row_table", row_table, torch.int32), ("accept_out", accept_out, torch.uint8)))
     arr = (ctypes.c_void_p * len(tables))(*[t.ptr.value for t in tables])
     _check(lib().cstr_step_static(arr, ctypes.c_int32(len(tables)), _dev_ptr(row_table),
-                                  _dev_ptr(logits), ctypes.c_int32(dtype),
-                                  ctypes.c_int64(logits.stride(0)), _dev_ptr(noise),
-                                  _dev_ptr(states), _dev_ptr(tokens_out), _dev_ptr(masked_out),
-                                  _dev_ptr(accept_out), ctypes.c_int32(batch), _stream_ptr(stream)))
+                                  _dev_ptr(logits), ctypes.c_int32(dtype), ctypes.c_int64(ld),
+                                  _dev_ptr(noise), _dev_ptr(states), _dev_ptr(tokens_out),
+                                  _dev_ptr(masked_out), _dev_ptr(accept_out), ctypes.c_int32(batch),
+                                  _stream_ptr(stream)))
 
 
 def cstr_step_status(ws: Workspace, stream=None):

@@ -110,3 +110,52 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(cstr, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         cstr.lib()
+
+
+@pytest.mark.parametrize("entry", ["cstr_step", "cstr_step_static", "cstr_step_history"])
+def test_step_wrappers_reject_bad_row_tensors_before_any_launch(monkeypatch, entry):
+    # a short or wrongly typed per-row tensor would be an out-of-bounds device write; the
+    # binding must refuse it without reaching the library (lib() is made to fail here)
+    import torch
+
+    def no_library():
+        raise AssertionError("the library was reached")
+    monkeypatch.setattr(cstr, "lib", no_library)
+    B, V = 4, 8
+    logits = torch.zeros(B, V)
+    good = dict(states=torch.zeros(B, dtype=torch.int32), tokens_out=torch.zeros(B, dtype=torch.int32),
+                masked_out=torch.zeros(B, V), accept_out=torch.zeros(B, dtype=torch.uint8),
+                row_table=torch.zeros(B, dtype=torch.int32), noise=torch.zeros(B, V))
+
+    def call(**over):
+        a = dict(good)
+        a.update(over)
+        table = cstr.Table(None)
+        if entry == "cstr_step_static":
+            cstr.cstr_step_static([table], logits, a["states"], a["tokens_out"], a["masked_out"],
+                                  noise=a["noise"], row_table=a["row_table"], accept_out=a["accept_out"])
+        elif entry == "cstr_step":
+            cstr.cstr_step([table], logits, a["states"], a["tokens_out"], a["masked_out"], None,
+                           noise=a["noise"], row_table=a["row_table"], accept_out=a["accept_out"])
+        else:
+            cstr.cstr_step_history([table], logits, a["states"], a["states"].clone(), a["tokens_out"],
+                                   a["masked_out"], None, noise=a["noise"], row_table=a["row_table"],
+                                   accept_out=a["accept_out"])
+
+    with pytest.raises(ValueError, match="tokens_out"):
+        call(tokens_out=torch.zeros(B - 1, dtype=torch.int32))
+    with pytest.raises(ValueError, match="states"):
+        call(states=torch.zeros(B, dtype=torch.int64))
+    with pytest.raises(ValueError, match="accept_out"):
+        call(accept_out=torch.zeros(B, dtype=torch.int32))
+    with pytest.raises(ValueError, match="row_table"):
+        call(row_table=torch.zeros(2 * B, dtype=torch.int32)[::2])
+    with pytest.raises(TypeError, match="masked_out"):
+        call(masked_out=torch.zeros(B, V, dtype=torch.bfloat16))
+    with pytest.raises(TypeError, match="noise"):
+        call(noise=torch.zeros(B, V, dtype=torch.float64))
+    with pytest.raises(ValueError, match="masked_out"):
+        call(masked_out=torch.zeros(B, V + 1))
+    # well-formed arguments that live on the CPU are refused too (last check, still before the library)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        call()

@@ -114,22 +114,65 @@ def test_config_schema40_128k():
     check_table(table, dfa, vb, vo, slab=123)
 
 
-@pytest.mark.parametrize("name", ["string_256k", "random10k_256k"])
-def test_config_256k_sampled_states(name):
-    # Full-size build; the oracle recomputes whole rows for a sample of states
-    # (first, last, slab edges, random), each row being 256,000 transitions.
-    dfa = config_dfas(name)[0]
-    vb, vo = config_vocab(name)
-    (table,) = gpu_tables([dfa], vb, vo)
+def whole_table_parity(table, dfa, vb, vo, slab=256):
+    """Every state of a full-size table against the oracle, streamed in slabs of states so
+    that neither side ever holds the table on the host; returns the number of live edges."""
     S = dfa[0].shape[0]
-    rng = np.random.default_rng(1)
-    sample = sorted(set([0, 1, 15, 16, 17, S - 17, S - 2, S - 1] + rng.integers(0, S, size=40).tolist()))
-    check_table(table, dfa, vb, vo, states=sample)
+    threads = min(oracle.max_threads(), 32)
+    live_total = 0
+    for lo in range(0, S, slab):
+        hi = min(S, lo + slab)
+        nxt, mask = cstr.cstr_table_download(table, lo, hi)
+        o_next, o_mask = oracle.token_table(dfa[0], dfa[1], vb, vo, q_lo=lo, q_hi=hi, threads=threads)
+        assert np.array_equal(nxt, o_next), "next-state rows %d..%d differ" % (lo, hi)
+        assert np.array_equal(mask, o_mask), "mask rows %d..%d differ" % (lo, hi)
+        live_total += int((o_next >= 0).sum())
+    return live_total
+
+
+def test_config_string_256k_whole_table():
+    # all 8,195 x 256,000 transitions and all mask words
+    dfa = config_dfas("string_256k")[0]
+    vb, vo = config_vocab("string_256k")
+    (table,) = gpu_tables([dfa], vb, vo)
+    check_table(table, dfa, vb, vo, states=[0])          # shape information, first row
+    assert whole_table_parity(table, dfa, vb, vo) > 0
     # popcount of every mask row equals the count of live entries, for a slab of rows
     nxt, mask = cstr.cstr_table_download(table, 100, 132)
     live = (nxt >= 0).sum(axis=1)
     pop = np.unpackbits(mask.view(np.uint8), axis=1).sum(axis=1)
     assert np.array_equal(live, pop)
+
+
+def test_config_random10k_256k_whole_tables_of_all_eight_dfas():
+    # 8 x 10,000 x 256,000 transitions: each automaton is built into the same table storage
+    # (a rebuild) and compared completely before the next one is built
+    dfas = config_dfas("random10k_256k")
+    assert len(dfas) == 8
+    vb, vo = config_vocab("random10k_256k")
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    table = cstr.cstr_table_create(vocab, 10000)
+    for dfa in dfas:
+        cstr.cstr_table_build(table, cstr.cstr_load_dfa(*dfa))
+        torch.cuda.synchronize()
+        assert cstr.cstr_table_info(table)["start_state"] == dfa[2]
+        assert whole_table_parity(table, dfa, vb, vo) > 0
+
+
+def test_download_slabs_of_any_alignment():
+    # the download decodes on the device in tiles of 32 states: ranges that start and end
+    # anywhere, single rows, the last partial tile, and 32-bit entries
+    rng = np.random.default_rng(31)
+    vb, vo = random_vocab(rng, 1000)
+    for S in (70, 300):
+        dfa = dense_random_dfa(rng, S, live=0.8)
+        (table,) = gpu_tables([dfa], vb, vo)
+        full_next, full_mask = oracle.token_table(dfa[0], dfa[1], vb, vo)
+        for lo, hi in [(0, S), (1, 2), (31, 33), (S - 1, S), (5, 69), (33, 64), (7, 7)]:
+            nxt, mask = cstr.cstr_table_download(table, lo, hi)
+            assert np.array_equal(nxt, full_next[lo:hi]) and np.array_equal(mask, full_mask[lo:hi])
+        nxt, _ = cstr.cstr_table_download(table, 3, 40, want_mask=False)
+        assert np.array_equal(nxt, full_next[3:40])
 
 
 def test_small_constraints_over_the_256k_vocabulary():

@@ -4,8 +4,10 @@ Some hosts of the library cannot call the CUDA allocator while they run (all
 device memory already handed to a cache pool, a fixed memory budget, or no
 tolerance for cudaMalloc's device-wide synchronisation).  ``cstr_step_static``
 serves them with a fixed scratch array inside the library; here it must give
-exactly what ``cstr_step`` gives, on two consecutive calls that share that
-array.  Collected last so that a failure here cannot hide any other test.
+exactly what ``cstr_step`` gives - and what the CPU oracle gives - on
+consecutive calls that share that array, and the device's free memory must not
+move across its calls.  Collected last so that a failure here cannot hide any
+other test.
 """
 import ctypes
 
@@ -13,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2407_08103_b200 import cstr
 from synth import gumbel_noise, normal_logits
 from synth.configs import config_dfas, config_vocab
@@ -21,7 +24,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def test_static_step_matches_workspace_step_twice():
+def test_static_step_matches_workspace_step_and_oracle_without_allocating():
     dfa = config_dfas("json_32k")[0]
     vb, vo = config_vocab("json_32k")
     V = vo.size - 1
@@ -37,17 +40,29 @@ def test_static_step_matches_workspace_step_twice():
     start[6] = dfa[0].shape[0] + 3                  # an out-of-range state
     st_a = torch.from_numpy(start).to(DEV)
     st_b = st_a.clone()
-    for call in range(2):                           # second call reuses the shared array
-        logits = torch.from_numpy(normal_logits(21, call, range(B), V)).to(DEV)
-        noise = torch.from_numpy(gumbel_noise(22, call, range(B), V)).to(DEV) if call else None
-        tok_a = torch.full((B,), -5, dtype=torch.int32, device=DEV)
-        tok_b = torch.full((B,), -6, dtype=torch.int32, device=DEV)
-        acc_a = torch.full((B,), 7, dtype=torch.uint8, device=DEV)
-        acc_b = torch.full((B,), 8, dtype=torch.uint8, device=DEV)
-        out_a = torch.empty_like(logits)
-        out_b = torch.empty_like(logits)
-        cstr.cstr_step([table], logits, st_a, tok_a, out_a, ws, noise=noise, accept_out=acc_a)
-        cstr.cstr_step_static([table], logits, st_b, tok_b, out_b, noise=noise, accept_out=acc_b)
+    o_states = start.copy()
+    # every tensor of all three calls exists before the first one, so that the free-memory
+    # readings below see only what the entry point itself does
+    n_calls = 3
+    h_logits = [normal_logits(21, c, range(B), V) for c in range(n_calls)]
+    h_noise = [gumbel_noise(22, c, range(B), V) if c else None for c in range(n_calls)]
+    logits = [torch.from_numpy(x).to(DEV) for x in h_logits]
+    noise = [None if x is None else torch.from_numpy(x).to(DEV) for x in h_noise]
+    tok_a = torch.full((B,), -5, dtype=torch.int32, device=DEV)
+    tok_b = torch.full((B,), -6, dtype=torch.int32, device=DEV)
+    acc_a = torch.full((B,), 7, dtype=torch.uint8, device=DEV)
+    acc_b = torch.full((B,), 8, dtype=torch.uint8, device=DEV)
+    out_a = torch.empty_like(logits[0])
+    out_b = torch.empty_like(logits[0])
+    free_before_second = None
+    for call in range(n_calls):                     # later calls reuse the shared array
+        if call == 1:
+            torch.cuda.synchronize()
+            free_before_second = torch.cuda.mem_get_info()[0]       # cudaMemGetInfo
+        cstr.cstr_step([table], logits[call], st_a, tok_a, out_a, ws, noise=noise[call],
+                       accept_out=acc_a)
+        cstr.cstr_step_static([table], logits[call], st_b, tok_b, out_b, noise=noise[call],
+                              accept_out=acc_b)
         torch.cuda.synchronize()
         # integer outputs and the masked logits (copies or -inf) must be identical bit for bit
         assert torch.equal(tok_a, tok_b)
@@ -55,6 +70,16 @@ def test_static_step_matches_workspace_step_twice():
         assert torch.equal(acc_a, acc_b)
         assert torch.equal(out_a.view(torch.int32), out_b.view(torch.int32))
         assert int((tok_a >= 0).sum()) >= B - 2
+        # ... and they are the oracle's
+        ref = oracle.step([dfa], vb, vo, h_logits[call], o_states, noise=h_noise[call], threads=8)
+        assert np.array_equal(tok_b.cpu().numpy(), ref["tokens"])
+        assert np.array_equal(st_b.cpu().numpy(), ref["states"])
+        assert np.array_equal(acc_b.cpu().numpy(), ref["accept"])
+        assert np.array_equal(out_b.cpu().numpy().view(np.uint32), ref["masked"].view(np.uint32))
+        o_states = ref["states"]
+    # the one property the entry point exists for: the device's free memory did not move
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before_second
     assert int(tok_a[5]) == -1 and int(tok_a[6]) == -1
 
 
