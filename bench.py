@@ -36,10 +36,56 @@ POOL = 4
 BYTES_PER_LOGIT_F32_GREEDY = 4 + 4 + 1.0 / 8.0    # read + masked write + mask bit
 BYTES_PER_TRANSITION = 2 + 1.0 / 8.0              # int16 next entry + mask bit, stores only
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one full-size step launch (512 x 256,000 fp32),
-# from the ncu capture summarised in profiles/step_vec_kernel_fp32_full_size_traffic.md; set to
-# None whenever step_vec_kernel changes until the capture is repeated.
-STEP_TRAFFIC_BYTES = 994.0e6
+NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one step launch of the small profiling case
+# (`--case small`: 128 rows x 256,000 fp32 logits), from the ncu capture summarised in
+# profiles/step_vec_kernel_fp32_small_case.md, with the SHA-256 of the kernel source the
+# capture ran.  The bench scales it to its own launch by the logits processed (the traffic
+# is proportional to them) and reports null when the source has changed since.
+STEP_TRAFFIC_SMALL_CASE_BYTES = None
+STEP_TRAFFIC_SMALL_CASE_LOGITS = 128 * 256000
+STEP_TRAFFIC_SOURCE_SHA256 = None
+STEP_KERNEL_SOURCE = os.path.join(ROOT, "paper_2407_08103_b200", "csrc", "cstr_step.cu")
+
+
+def file_sha256(path: str) -> str:
+    import hashlib
+    with open(path, "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()
+
+
+def step_traffic_bytes(logits_per_launch: int):
+    """DRAM traffic of one step launch, scaled from the recorded small-case capture; None
+    when there is no capture or the step kernel's source is no longer the captured one."""
+    if STEP_TRAFFIC_SMALL_CASE_BYTES is None or STEP_TRAFFIC_SOURCE_SHA256 is None:
+        return None
+    try:
+        if file_sha256(STEP_KERNEL_SOURCE) != STEP_TRAFFIC_SOURCE_SHA256:
+            return None
+    except OSError:
+        return None
+    return STEP_TRAFFIC_SMALL_CASE_BYTES * (logits_per_launch / STEP_TRAFFIC_SMALL_CASE_LOGITS)
+
+
+def roofline_entry(achieved_gbs: float, peak: float, peak_kind: str, bound: str = "hbm",
+                   traffic=None, **extra):
+    """A roofline object: achieved algorithmic GB/s against the measured copy rate and,
+    beside it, against the nominal 8 TB/s."""
+    d = {"bound": bound, "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
+         "frac": achieved_gbs / peak, "traffic": traffic, "peak_kind": "of %s" % peak_kind,
+         "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS}
+    d.update(extra)
+    return d
+
+
+def inputs_sha256(dfa, vb, vo, first_logits_row) -> str:
+    """One digest over the seeded inputs (DFA table, accept flags, vocabulary, first logits
+    row), so that two bench lines can be seen to have run on the same data."""
+    import hashlib
+    h = hashlib.sha256()
+    for a in (dfa[0], dfa[1], vb, vo, first_logits_row):
+        h.update(np.ascontiguousarray(a).tobytes())
+    return h.hexdigest()
 
 
 def parse_args():
@@ -63,6 +109,9 @@ def parse_args():
                          "4,099-state string DFA / a 4,096-state random DFA; small_constraints: the five "
                          "small-constraint compiles over the 256,000-token vocabulary) and print its entry; "
                          "for profiler captures, not a bench line")
+    ap.add_argument("--walker", default="trie", choices=["trie", "dense"],
+                    help="with --build-only: trie = cstr_table_build, dense = cstr_table_build_dense "
+                         "(every token from its first byte; the baseline the trie walk is compared with)")
     ap.add_argument("--pushdown-only", action="store_true",
                     help="time only the push-down step leg (batch 128 with --case small) and print "
                          "its entry; for profiler captures, not a bench line")
@@ -238,7 +287,8 @@ def time_oracle(w, dfa, vb, vo, pools, budget_s: float, max_steps: int):
     return B * V * done / dt, threads, sample, dt / done
 
 
-def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak, steps=48):
+def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak, peak_kind,
+                        steps=48):
     """Step-kernel and table-build timing of one of the other workloads: device
     generated seeded logits (timing only; parity is covered by the tests), a
     pool of tensors larger than twice the L2 where the batch allows, finished
@@ -339,6 +389,16 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
         graph_resident_ms = graph_time(False)
     except Exception as exc:  # pragma: no cover - depends on the box
         sys.stderr.write("graph timing of %s skipped: %r\n" % (name, exc))
+    # the same table by the per-token walker without the trie (the pair "trie vs dense")
+    dense = []
+    for _ in range(3):
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        cstr.cstr_table_build_dense(tables[0], handles[0], -1, stream)
+        a1.record(stream)
+        a1.synchronize()
+        dense.append(a0.elapsed_time(a1))
+    dense_ms = float(np.mean(dense[1:]))
     bytes_per_logit = 2 * esz + (4 if w.gumbel else 0) + 1.0 / 8.0
     step_bytes = B * V * bytes_per_logit
     gbs = step_bytes / (kernel_ms * 1e-3) / 1e9
@@ -352,16 +412,19 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
         "tables": len(tables), "step_kernel_ms": kernel_ms, "step_loop_ms": loop_ms,
         "step_graph_ms": graph_ms, "step_graph_ms_same_tensor": graph_resident_ms,
         "logits_per_s": B * V / (kernel_ms * 1e-3),
-        "roofline": {"bound": "hbm" if hbm_honest else "launch latency (working set sits in L2)",
-                     "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                     "traffic": None, "bytes_per_logit": bytes_per_logit,
-                     "logits_pool": "%d tensors x %.1f MB" % (pool_n, tensor_bytes / 1e6)},
+        "roofline": roofline_entry(
+            gbs, peak, peak_kind,
+            bound="hbm" if hbm_honest else "launch latency (working set sits in L2)",
+            bytes_per_logit=bytes_per_logit,
+            logits_pool="%d tensors x %.1f MB" % (pool_n, tensor_bytes / 1e6)),
         "table_build": {"dfa_states": S0, "ms": bms, "transitions_per_s": S0 * V / (bms * 1e-3),
-                        "store_gbs": bgbs, "frac_of_hbm_peak": bgbs / peak},
+                        "dense_walker_ms": dense_ms,
+                        "roofline": roofline_entry(bgbs, peak, peak_kind,
+                                                   note="stores of next + mask only")},
     }
 
 
-def time_wildcard_build(torch, cstr, vocab, vb, vo, stream, peak):
+def time_wildcard_build(torch, cstr, vocab, vb, vo, stream, peak, peak_kind):
     """Table build of a constraint with terminal-label (wildcard) edges over the
     256k vocabulary: the paper's bulleted-summary example (Section 2.5.1), with
     PARAGRAPH_TOKEN = the newline-free tokens."""
@@ -387,11 +450,13 @@ def time_wildcard_build(torch, cstr, vocab, vb, vo, stream, peak):
     return {"workload": "summary bullets with PARAGRAPH_TOKEN wildcard x vocab 256,000",
             "dfa_states": S, "states_with_terminal_edges": int((term >= 0).any(axis=1).sum()),
             "ms": best, "transitions_per_s": S * V / (best * 1e-3),
-            "store_gbs": S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9,
-            "frac_of_hbm_peak": S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9 / peak}
+            "roofline": roofline_entry(S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9, peak,
+                                       peak_kind, bound="launch latency (tens of microseconds)",
+                                       note="stores of next + mask only")}
 
 
-def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=512, steps=48):
+def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, peak_kind, V=256000, B=512,
+                  steps=48):
     """Push-down step (Algorithm 3) on a nested-JSON PDA over a 256,000-token
     vocabulary with structural multi-bracket tokens, batch 512, fp32, greedy:
     table build (allocation + kernel) and the two-kernel step (situation
@@ -446,14 +511,14 @@ def time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak, V=256000, B=5
             "table_build_ms": float(np.mean(build_ms)), "table_create_and_build_ms": create_ms,
             "table_transitions_per_s": n_cfg * V / (float(np.mean(build_ms)) * 1e-3),
             "step_ms": ms, "logits_per_s": B * V / (ms * 1e-3),
-            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
-                         "frac": gbs / peak, "traffic": None,
-                         "note": "two kernels per step (situation lookup, fused step); 8.125 algorithmic bytes per logit"},
+            "roofline": roofline_entry(gbs, peak, peak_kind,
+                                       note="two kernels per step (situation lookup, fused step); "
+                                            "8.125 algorithmic bytes per logit"),
             "mean_stack_depth": depth_sum / probes, "max_stack_depth": depth_max,
             "status_rows": {"bad": bad, "empty_mask": empty, "overflow": overflow}}
 
 
-def time_build_only(torch, cstr, name, case, stream, repeats=4):
+def time_build_only(torch, cstr, name, case, stream, repeats=4, walker="trie"):
     """Token-table build of one workload's (first) DFA over its vocabulary."""
     from synth import random_range_dfa
     from synth.configs import CONFIGS, config_dfas, config_vocab
@@ -474,16 +539,19 @@ def time_build_only(torch, cstr, name, case, stream, repeats=4):
     for _ in range(repeats):
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record(stream)
-        cstr.cstr_table_build(table, h, -1, stream)
+        if walker == "dense":
+            cstr.cstr_table_build_dense(table, h, -1, stream)
+        else:
+            cstr.cstr_table_build(table, h, -1, stream)
         a1.record(stream)
         a1.synchronize()
         ms.append(a0.elapsed_time(a1))
     best = float(np.mean(ms[1:]))
     peak, kind = measured_hbm_peak()
     gbs = S * V * BYTES_PER_TRANSITION / (best * 1e-3) / 1e9
-    return {"workload": name + (" (small case)" if case == "small" else ""), "dfa_states": S,
-            "vocab": V, "ms": best, "transitions_per_s": S * V / (best * 1e-3), "store_gbs": gbs,
-            "frac_of_hbm_peak": gbs / peak, "peak_kind": "of %s" % kind}
+    return {"workload": name + (" (small case)" if case == "small" else ""), "walker": walker,
+            "dfa_states": S, "vocab": V, "ms": best, "transitions_per_s": S * V / (best * 1e-3),
+            "roofline": roofline_entry(gbs, peak, kind, note="stores of next + mask only")}
 
 
 def time_small_compiles(torch, cstr, vocab, stream):
@@ -633,11 +701,12 @@ def main():
         return
     if args.build_only:
         print(json.dumps({"table_build": time_build_only(torch, cstr, args.build_only, args.case,
-                                                         torch.cuda.current_stream())}))
+                                                         torch.cuda.current_stream(),
+                                                         walker=args.walker)}))
         return
     if args.pushdown_only:
         entry = time_pushdown(torch, cstr, PushdownDecoder, dev, torch.cuda.current_stream(),
-                              measured_hbm_peak()[0], B=128 if args.case == "small" else 512,
+                              *measured_hbm_peak(), B=128 if args.case == "small" else 512,
                               steps=max(args.steps, 1) if args.steps < 100 else 48)
         print(json.dumps({"pushdown_step": entry}))
         return
@@ -760,36 +829,86 @@ def main():
         spec_ms = float(np.mean(sp[2:]))
         spec = {"sequences": seqs, "drafted_tokens": kk, "rows": B, "ms": spec_ms,
                 "logits_per_s": B * V / (spec_ms * 1e-3),
-                "frac_of_hbm_peak": B * V * BYTES_PER_LOGIT_F32_GREEDY / (spec_ms * 1e-3) / 1e9
-                / measured_hbm_peak()[0],
+                "roofline": roofline_entry(B * V * BYTES_PER_LOGIT_F32_GREEDY / (spec_ms * 1e-3) / 1e9,
+                                           *measured_hbm_peak()),
                 "kernels": "step_vec_kernel over the state history + accept_draft_kernel"}
 
-    # ---- end to end: pinned host logits in, tokens + states out, every step ----
+    # ---- end to end: pinned host logits in, results out, every step -------------
+    # twice: tokens + states back (what a sampler needs), and with the penalised logits
+    # copied back to pinned host memory as well (every result of the step)
     staging = [torch.empty((B, V), dtype=torch.float32, device=dev) for _ in range(2)]
     h_tok = torch.empty(B, dtype=torch.int32).pin_memory()
     h_st = torch.empty(B, dtype=torch.int32).pin_memory()
+    h_masked = torch.empty((B, V), dtype=torch.float32).pin_memory()
     Ke = min(K, 64)
-    dec.reset()
 
-    def e2e_step(i):
+    def e2e_step(i, with_masked):
         # one C-ABI call: pinned host logits in (sliced uploads overlapped with the step
-        # kernels), tokens + states back on the host when it returns
+        # kernels), tokens + states (+ penalised logits) back on the host when it returns
         cstr.cstr_step_host([table], host_pool[i % POOL], dec.states, h_tok, staging[0], staging[1],
-                            dec.tokens, dec.ws, states_host=h_st, stream=stream)
+                            dec.tokens, dec.ws, states_host=h_st,
+                            masked_host=h_masked if with_masked else None, stream=stream)
         torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
 
-    e2e_ms = float("nan")
+    e2e_ms = e2e_full_ms = float("nan")
     if not args.skip_e2e:
-        for i in range(3):
-            e2e_step(i)
-        barrier()
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record(stream)
-        for i in range(Ke):
-            e2e_step(i)
-        f1.record(stream)
-        barrier()
-        e2e_ms = max_over_ranks(f0.elapsed_time(f1))
+        for with_masked in (False, True):
+            dec.reset()
+            for i in range(3):
+                e2e_step(i, with_masked)
+            barrier()
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(stream)
+            for i in range(Ke):
+                e2e_step(i, with_masked)
+            f1.record(stream)
+            barrier()
+            if with_masked:
+                e2e_full_ms = max_over_ranks(f0.elapsed_time(f1))
+            else:
+                e2e_ms = max_over_ranks(f0.elapsed_time(f1))
+
+    # ---- the bandwidth-bound bf16 legs: the same table, 512 x 256,000 bf16 logits,
+    # greedy and Gumbel-max (device-generated seeded values: timing only)
+    bf16_legs = None
+    if rank == 0 and args.case == "full" and not args.skip_other_workloads:
+        bf16_legs = []
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(w.logits_seed + 7)
+        bpool = [torch.randn((B, V), generator=gen, device=dev).to(torch.bfloat16) for _ in range(POOL)]
+        bout = [torch.empty((B, V), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        u = torch.rand((B, V), generator=gen, device=dev).clamp_(1e-20, 1 - 1e-7)
+        gnoise = [-torch.log(-torch.log(u)), None]
+        u = torch.rand((B, V), generator=gen, device=dev).clamp_(1e-20, 1 - 1e-7)
+        gnoise[1] = -torch.log(-torch.log(u))
+        del u
+        peak_now, kind_now = measured_hbm_peak()
+        for gumbel in (False, True):
+            dec.reset()
+            bp = []
+            for i in range(36):
+                b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                b0.record(stream)
+                dec.step(bpool[i % POOL], noise=gnoise[i & 1] if gumbel else None,
+                         masked_out=bout[i & 1], stream=stream)
+                b1.record(stream)
+                torch.where(dec.states < 0, start_vec, dec.states, out=dec.states)
+                if i >= 4:
+                    bp.append((b0, b1))
+            torch.cuda.synchronize()
+            ms = float(np.mean([a.elapsed_time(b) for a, b in bp]))
+            bpl = 2 + 2 + (4 if gumbel else 0) + 1.0 / 8.0
+            bf16_legs.append({
+                "workload": "%s table, batch %d x vocab %d, bf16 logits, %s" %
+                            (WORKLOAD, B, V, "gumbel-max (fp32 noise)" if gumbel else "greedy"),
+                "kernel": "step_vec_kernel<bf16, %s>" % ("noise" if gumbel else "greedy"),
+                "step_kernel_ms": ms, "logits_per_s": B * V / (ms * 1e-3),
+                "roofline": roofline_entry(B * V * bpl / (ms * 1e-3) / 1e9, peak_now, kind_now,
+                                           bytes_per_logit=bpl,
+                                           logits_pool="%d tensors x %.1f MB" % (POOL, B * V * 2 / 1e6))})
+        del bpool, bout, gnoise
+        torch.cuda.empty_cache()
+        dec.reset()
     sampler.stop_flag.set()
     sampler.join(timeout=2)
     clocks = sampler.summary(t_dev0, t_dev1)
@@ -823,20 +942,20 @@ def main():
 
     wildcard = None
     if not args.skip_build_bench and rank == 0 and args.case == "full":
-        wildcard = time_wildcard_build(torch, cstr, vocab, vb, vo, stream, measured_hbm_peak()[0])
+        wildcard = time_wildcard_build(torch, cstr, vocab, vb, vo, stream, *measured_hbm_peak())
 
     # ---- the other four workloads (single-GPU runs only) --------------------
     others, pushdown = None, None
     if rank == 0 and world == 1 and not args.skip_other_workloads and args.case == "full":
         del dev_pool, staging, out_bufs
         torch.cuda.empty_cache()
-        peak_now, _ = measured_hbm_peak()
-        pushdown = time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak_now)
+        peak_now, kind_now = measured_hbm_peak()
+        pushdown = time_pushdown(torch, cstr, PushdownDecoder, dev, stream, peak_now, kind_now)
         torch.cuda.empty_cache()
         others = []
         for name in ("api_1k", "json_32k", "schema40_128k", "random10k_256k"):
             others.append(time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream,
-                                              peak_now))
+                                              peak_now, kind_now))
             torch.cuda.empty_cache()
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1) --------
@@ -868,9 +987,8 @@ def main():
         gbs = s_states * V * BYTES_PER_TRANSITION / (ms_best * 1e-3) / 1e9
         return {"workload": workload, "dfa_states": s_states, "vocab": V, "ms": ms_best,
                 "value": tps, "unit": "transitions/s",
-                "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
-                             "frac": gbs / peak, "traffic": None,
-                             "note": "stores of next (int16) + mask only; of %s copy rate" % peak_kind}}
+                "roofline": roofline_entry(gbs, peak, peak_kind,
+                                           note="stores of next (int16) + mask only")}
 
     e2e = None
     if not args.skip_e2e:
@@ -878,7 +996,15 @@ def main():
                "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * 8, "steps": Ke,
                "ms_per_step": e2e_ms / Ke,
                "note": "cstr_step_host per step: pinned host logits -> device in 8 row slices overlapped "
-                       "with the step kernels, tokens + states -> host, synchronous"}
+                       "with the step kernels, tokens + states -> host, synchronous; the penalised "
+                       "logits stay on the device",
+               "with_masked_logits": {
+                   "value": logits_per_step * Ke / (e2e_full_ms * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": B * V * 4, "d2h_bytes_per_step": B * V * 4 + B * 8,
+                   "steps": Ke, "ms_per_step": e2e_full_ms / Ke,
+                   "note": "the same call with masked_host given: every result of the step (tokens, "
+                           "states and the penalised logits) is in pinned host memory when it returns; "
+                           "downloads of earlier slices overlap the uploads of later ones"}}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak",
@@ -892,14 +1018,14 @@ def main():
         "e2e": e2e,
         "gpu_launches": K,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak,
-                     "traffic": STEP_TRAFFIC_BYTES if args.case == "full" else None,
-                     "kernel": "step_vec_kernel<fp32, greedy>", "kernel_ms": kernel_ms,
-                     "kernel_ms_best": kernel_ms_best, "launches_timed": ks,
-                     "bytes_per_launch": step_bytes, "peak_kind": "of %s" % peak_kind,
-                     "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "active_row_fraction_at_end": active_frac},
+        "roofline": roofline_entry(
+            achieved, peak, peak_kind, traffic=step_traffic_bytes(B * V),
+            traffic_source="ncu DRAM counters of the small profiling case (128 rows), scaled by "
+                           "the logits per launch; null when the kernel source changed since",
+            kernel="step_vec_kernel<fp32, greedy>", kernel_ms=kernel_ms,
+            kernel_ms_best=kernel_ms_best, launches_timed=ks, bytes_per_launch=step_bytes,
+            active_row_fraction_at_end=active_frac),
+        "inputs_sha256": inputs_sha256(dfa, vb, vo, host_pool[0][0].numpy()),
         "cpu_baseline": cpu,
         "table_build": [build_entry(bt, S, WORKLOAD)] +
                        ([build_entry(build_random, 10000 if args.case == "full" else 4096,
@@ -915,6 +1041,7 @@ def main():
         "pushdown_step": pushdown,
         "small_batch_step_latency": small,
         "other_workloads": others,
+        "bf16_step_512x256k": bf16_legs,
         "status_rows": {"bad_state": bad, "empty_mask": empty},
     }
     print(json.dumps(line))

@@ -71,7 +71,8 @@ typedef struct cstr_pda_workspace cstr_pda_workspace_t; /* per-stream scratch of
  * classes, and copies the class-major table to the device (16-bit entries up
  * to 32766 states, else 32-bit); returns the handle in *out.
  * Synchronous; allocates device memory.  Each host thread keeps the device
- * scratch of its last load (the raw table, at most 64 MB) for the next one.
+ * scratch of its last load (the raw table, at most 64 MB) for the next one
+ * and frees it when the thread ends.
  */
 int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_t n_states,
                   int32_t start_state, cstr_dfa_t **out);
@@ -152,6 +153,18 @@ int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states, cstr_table_
  */
 int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
                      void *cuda_stream);
+
+/*
+ * The same table as cstr_table_build, computed the plain way: every token is
+ * walked from its first byte for every state, as if the detokenizing
+ * transducer were Algorithm 1's one chain per token with no prefix shared
+ * between tokens (Section 2.3 describes the compact, trie-shaped T_V that
+ * cstr_table_build walks instead).  Same arguments, same results, slower; it
+ * exists so that the saving of the trie walk can be measured on any
+ * constraint.
+ */
+int cstr_table_build_dense(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                           void *cuda_stream);
 
 /*
  * One-call form: load the vocabulary from HOST arrays (as cstr_load_vocab),
@@ -237,17 +250,21 @@ int cstr_step(const cstr_table_t *const *tables, int32_t n_tables, const int32_t
  *   logits_dev   DEVICE staging [batch][ld] of `dtype`, overwritten
  *   noise_dev    DEVICE staging float [batch][ld]; NULL exactly when noise_host is NULL
  *   masked_out   DEVICE [batch][ld]: the penalised logits (may equal logits_dev)
+ *   masked_host  HOST   [batch][ld] of `dtype`, or NULL: when given, the penalised
+ *                logits are also copied there, slice by slice on a third stream
+ *                while later slices upload and run
  *   tokens_dev   DEVICE int32 [batch]
  * tables, row_table, accept_out, ws: as in cstr_step.  Synchronous: returns
- * after the results are in tokens_host / states_host (it synchronises
- * cuda_stream).  Allocates no device memory; its first call on a workspace
- * creates the copy stream and a few events.
+ * after the results are in tokens_host / states_host / masked_host (it
+ * synchronises cuda_stream and its own copy streams, on failure too, so the
+ * host buffers are never in use once it has returned).  Allocates no device
+ * memory; its first call on a workspace creates two copy streams and a few events.
  */
 int cstr_step_host(const cstr_table_t *const *tables, int32_t n_tables, const int32_t *row_table,
                    const void *logits_host, int32_t dtype, int64_t ld, const float *noise_host,
                    int32_t *states, int32_t *tokens_host, int32_t *states_host, void *logits_dev,
-                   float *noise_dev, void *masked_out, int32_t *tokens_dev, uint8_t *accept_out,
-                   int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
+                   float *noise_dev, void *masked_out, void *masked_host, int32_t *tokens_dev,
+                   uint8_t *accept_out, int32_t batch, cstr_workspace_t *ws, void *cuda_stream);
 
 /*
  * cstr_step that leaves the input states untouched and writes the new ones to

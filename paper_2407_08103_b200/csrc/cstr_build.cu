@@ -20,8 +20,6 @@
 //     next-state entries with one vector store into the token's row;
 //     validity goes out as NS ballot words per (token, warp), which a second
 //     kernel bit-transposes into the state-major mask the step streams.
-#include <stdlib.h>
-
 #include "cstr_internal.cuh"
 
 namespace {
@@ -31,6 +29,13 @@ constexpr int kDepth = CSTR_STACK_DEPTH;
 constexpr int kDedupMaxClasses = 16;    // duplicate-column pass: automata with at most this many
 constexpr int kDedupMinTokens = 8192;   // byte classes, vocabularies of at least this many tokens
 constexpr int kDedupMinStates = 2048;   // and enough states for the walk to outweigh the extra passes
+
+#ifdef CSTR_TESTING
+// Checking build only: the duplicate-column pass keeps this many bits of its
+// hash, so that tests can force collisions and exercise the exact comparison
+// that makes grouping safe.  The release library has no such switch.
+unsigned long long g_test_hash_keep = ~0ull;
+#endif
 
 struct BuildParams {
     const void *tt;            // [n_classes][row]
@@ -782,6 +787,46 @@ build_lane_token_kernel(const unsigned short *__restrict__ tt, const uint8_t *__
     }
 }
 
+// ---- per-token walker without the trie ---------------------------------------
+//
+// Algorithm 1 taken literally: every token is its own chain of the detokenizing
+// transducer, walked from its first byte for every state, with no prefix shared
+// between tokens.  One thread per (state, token): a CTA holds 256 consecutive
+// states of one token, looks the class-major table up through L1 / L2, stores
+// its entry of the token's row and contributes its bit to the ballot word of
+// its 32 states.  Kept as the baseline that shows what walking the trie-shaped
+// T_V (Section 2.3) saves; cstr_table_build never takes this path.
+template <typename ST, typename NT>
+__global__ void __launch_bounds__(256)
+build_dense_kernel(const __grid_constant__ BuildParams p)
+{
+    constexpr int ESZ = (int)sizeof(ST);
+    typedef typename Unit<ESZ>::type SU;
+    const unsigned v = blockIdx.x;
+    const int q = blockIdx.y * 256 + threadIdx.x;
+    const unsigned sink = (unsigned)CSTR_PERM(p.n_states) * ESZ;
+    const bool in = q < p.n_states;
+    unsigned cur = in ? (unsigned)CSTR_PERM(q) * ESZ : sink;
+    const uint32_t b0 = __ldg(p.off + v), n = __ldg(p.off + v + 1) - b0;
+    const bool is_eos = (int)v == p.eos_id;
+    const unsigned char *g_tt = (const unsigned char *)p.tt;
+    bool ok;
+    if (is_eos || n == 0) {
+        ok = is_eos && in && p.accept[q] != 0;
+        cur = sink;
+    } else {
+        for (uint32_t k = 0; k < n; ++k) {
+            const unsigned c = __ldg(p.cls + __ldg(p.bytes + b0 + k));
+            cur = (unsigned)__ldg((const SU *)(g_tt + (size_t)c * p.row * ESZ + cur));
+        }
+        ok = cur != sink;
+    }
+    ((NT *)p.next)[(unsigned long long)v * p.lds + q] = (NT)cur;       // q < lds (a multiple of 256)
+    const unsigned word = __ballot_sync(kFull, ok);
+    if ((threadIdx.x & 31) == 0)
+        p.maskT[(unsigned long long)v * p.ldb + (q >> 5)] = word;      // word k: states 32 k .. 32 k + 31
+}
+
 template <typename ST, typename NT, int NS, bool SMEM>
 cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
                         cudaStream_t stream)
@@ -820,6 +865,16 @@ cudaError_t launch_trie_ns(int ns, bool in_smem, const BuildParams &p, dim3 grid
 
 }  // namespace
 
+#ifdef CSTR_TESTING
+extern "C" int cstr_test_set_group_hash_bits(int32_t bits)
+{
+    if (bits < 0 || bits > 64)
+        return cstr_fail(CSTR_ERR_ARG, "cstr_test_set_group_hash_bits: bits = %d, need 0..64", bits);
+    g_test_hash_keep = (bits == 0 || bits == 64) ? ~0ull : (1ull << bits) - 1ull;
+    return CSTR_OK;
+}
+#endif
+
 // Post-pass for automata with terminal-label edges (no-op otherwise).
 static int launch_terminals(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
 {
@@ -842,7 +897,7 @@ static int launch_terminals(cstr_table *t, const cstr_dfa *dfa, cudaStream_t str
     return CSTR_OK;
 }
 
-int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
+int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, bool dense_walk)
 {
     const cstr_vocab *vc = t->vocab;
     BuildParams p;
@@ -865,6 +920,25 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
     if (dfa->wide && !t->wide)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
     const size_t st = dfa->wide ? 4 : 2;
+
+    if (dense_walk) {                  // the baseline walker: every token from its first byte
+        p.count_dev = nullptr;
+        p.reptok = nullptr;
+        dim3 grid((unsigned)t->V, (unsigned)((dfa->n_states + 255) / 256));
+        if (!dfa->wide && !t->wide)
+            build_dense_kernel<int16_t, int16_t><<<grid, 256, 0, stream>>>(p);
+        else if (!dfa->wide && t->wide)
+            build_dense_kernel<int16_t, int32_t><<<grid, 256, 0, stream>>>(p);
+        else
+            build_dense_kernel<int32_t, int32_t><<<grid, 256, 0, stream>>>(p);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        const int words = (dfa->n_states + 31) / 32;
+        dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
+        mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
+                                                      dfa->n_states, t->V, 1, nullptr);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        return launch_terminals(t, dfa, stream);
+    }
 
     // Small automata: one lane per token, all states in turn, mask words by ballot.
     const size_t small_smem =          // at most 256 x 66 x 2 + 256 bytes
@@ -908,14 +982,10 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream)
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_key, 0, (size_t)t->group_slots * 8, stream));
         CSTR_CUDA_TRY(cudaMemsetAsync(t->group_min, 0xff, (size_t)t->group_slots * 4, stream));
         const unsigned g = (unsigned)((t->V + 255) / 256);
-        // Test hook: CSTR_TEST_GROUP_HASH_BITS=n keeps only n bits of the hash, which forces
-        // collisions and so exercises the exact comparison that makes grouping safe.
         unsigned long long keep = ~0ull;
-        if (const char *bits = getenv("CSTR_TEST_GROUP_HASH_BITS")) {
-            const int n = atoi(bits);
-            if (n >= 1 && n < 64)
-                keep = (1ull << n) - 1ull;
-        }
+#ifdef CSTR_TESTING
+        keep = g_test_hash_keep;     // checking build only: fewer hash bits force collisions
+#endif
         // A small first launch seeds the table: thousands of tokens share a few
         // popular class strings, and once a group's minimum is in place the bulk
         // of the tokens finds it with plain loads instead of same-address atomics.

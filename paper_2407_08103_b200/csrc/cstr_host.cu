@@ -33,6 +33,50 @@ int cstr_check_device(int handle_device, const char *what)
     return CSTR_OK;
 }
 
+// --------------------------------------------- checking build: bounds record
+
+#ifdef CSTR_BOUNDS_CHECK
+#include <mutex>
+#include "cstr_debug.h"
+
+namespace {
+std::mutex g_oob_mutex;
+unsigned long long *g_oob_ptr[64] = {nullptr};
+}  // namespace
+
+unsigned long long *cstr_oob_record()
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64)
+        return nullptr;
+    std::lock_guard<std::mutex> lock(g_oob_mutex);
+    if (!g_oob_ptr[device]) {
+        unsigned long long *ptr = nullptr;
+        if (cudaMalloc((void **)&ptr, 32) != cudaSuccess || cudaMemset(ptr, 0, 32) != cudaSuccess)
+            return nullptr;
+        g_oob_ptr[device] = ptr;
+    }
+    return g_oob_ptr[device];
+}
+
+extern "C" int cstr_debug_bounds_status(uint64_t *out, int32_t reset)
+{
+    if (!out)
+        return cstr_fail(CSTR_ERR_NULL, "cstr_debug_bounds_status: null pointer");
+    unsigned long long *rec = cstr_oob_record();
+    if (!rec)
+        return cstr_fail(CSTR_ERR_CUDA, "cstr_debug_bounds_status: no record on this device");
+    CSTR_CUDA_TRY(cudaDeviceSynchronize());
+    unsigned long long host[4];
+    CSTR_CUDA_TRY(cudaMemcpy(host, rec, 32, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 4; ++i)
+        out[i] = host[i];
+    if (reset)
+        CSTR_CUDA_TRY(cudaMemset(rec, 0, 32));
+    return CSTR_OK;
+}
+#endif
+
 // ------------------------------------------------------------------ DFA
 
 namespace {
@@ -136,6 +180,23 @@ struct ScratchCache {
     int device = -1;
     unsigned char *ptr = nullptr;
     size_t bytes = 0;
+    // A host thread that ends gives its block back (a pool that recycles threads
+    // would otherwise leak one block per dead thread).  At process exit the CUDA
+    // runtime may already be gone; the calls then fail harmlessly.
+    ~ScratchCache()
+    {
+        if (!ptr)
+            return;
+        int cur = -1;
+        if (cudaGetDevice(&cur) != cudaSuccess)
+            return;
+        if (cur != device && cudaSetDevice(device) != cudaSuccess)
+            return;
+        cudaFree(ptr);
+        if (cur != device)
+            cudaSetDevice(cur);
+        ptr = nullptr;
+    }
 };
 thread_local ScratchCache t_scratch;
 
@@ -833,8 +894,8 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     return CSTR_OK;
 }
 
-extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
-                                void *cuda_stream)
+static int table_build_common(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                              void *cuda_stream, bool dense_walk)
 {
     if (!table || !dfa)
         return cstr_fail(CSTR_ERR_NULL, "cstr_table_build: null pointer");
@@ -861,7 +922,19 @@ extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int3
     table->code_shift = dfa->wide ? 2 : 1;
     CSTR_CUDA_TRY(cudaMemcpyAsync(table->accept, dfa->accept, (size_t)dfa->n_states,
                                   cudaMemcpyDeviceToDevice, stream));
-    return cstr_launch_build(table, dfa, stream);
+    return cstr_launch_build(table, dfa, stream, dense_walk);
+}
+
+extern "C" int cstr_table_build(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                                void *cuda_stream)
+{
+    return table_build_common(table, dfa, eos_id, cuda_stream, false);
+}
+
+extern "C" int cstr_table_build_dense(cstr_table_t *table, const cstr_dfa_t *dfa, int32_t eos_id,
+                                      void *cuda_stream)
+{
+    return table_build_common(table, dfa, eos_id, cuda_stream, true);
 }
 
 extern "C" int cstr_build_token_table(const cstr_dfa_t *dfa, const uint8_t *vocab_bytes,
@@ -981,8 +1054,11 @@ extern "C" void cstr_free_workspace(cstr_workspace_t *ws)
     cudaFree(ws->counters);
     if (ws->host_ready) {
         cudaStreamDestroy(ws->copy_stream);
-        for (int i = 0; i < CSTR_HOST_SLICES; ++i)
+        cudaStreamDestroy(ws->down_stream);
+        for (int i = 0; i < CSTR_HOST_SLICES; ++i) {
             cudaEventDestroy(ws->slice_ready[i]);
+            cudaEventDestroy(ws->slice_done[i]);
+        }
         cudaEventDestroy(ws->inputs_free);
     }
     delete ws;
@@ -1109,15 +1185,28 @@ extern "C" int cstr_step_history(const cstr_table_t *const *tables, int32_t n_ta
                        states_out, tokens_out, masked_out, accept_out, batch, ws, cuda_stream);
 }
 
+// Wait for everything cstr_step_host has in flight (uploads, kernels, downloads).
+static cudaError_t host_drain(cstr_workspace *ws, cudaStream_t stream)
+{
+    cudaError_t e = cudaStreamSynchronize(ws->copy_stream);
+    const cudaError_t e1 = cudaStreamSynchronize(stream);
+    const cudaError_t e2 = cudaStreamSynchronize(ws->down_stream);
+    if (e == cudaSuccess)
+        e = e1;
+    if (e == cudaSuccess)
+        e = e2;
+    return e;
+}
+
 // The step with its logits in host memory: rows are cut into slices whose
 // uploads run on a copy stream ahead of the step kernels of earlier slices.
 extern "C" int cstr_step_host(const cstr_table_t *const *tables, int32_t n_tables,
                               const int32_t *row_table, const void *logits_host, int32_t dtype,
                               int64_t ld, const float *noise_host, int32_t *states,
                               int32_t *tokens_host, int32_t *states_host, void *logits_dev,
-                              float *noise_dev, void *masked_out, int32_t *tokens_dev,
-                              uint8_t *accept_out, int32_t batch, cstr_workspace_t *ws,
-                              void *cuda_stream)
+                              float *noise_dev, void *masked_out, void *masked_host,
+                              int32_t *tokens_dev, uint8_t *accept_out, int32_t batch,
+                              cstr_workspace_t *ws, void *cuda_stream)
 {
     if (!tables || !ws)
         return cstr_fail(CSTR_ERR_NULL, "cstr_step_host: null pointer");
@@ -1140,8 +1229,11 @@ extern "C" int cstr_step_host(const cstr_table_t *const *tables, int32_t n_table
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (!ws->host_ready) {                       // first use: streams and events, no device memory
         CSTR_CUDA_TRY(cudaStreamCreateWithFlags(&ws->copy_stream, cudaStreamNonBlocking));
-        for (int i = 0; i < CSTR_HOST_SLICES; ++i)
+        CSTR_CUDA_TRY(cudaStreamCreateWithFlags(&ws->down_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < CSTR_HOST_SLICES; ++i) {
             CSTR_CUDA_TRY(cudaEventCreateWithFlags(&ws->slice_ready[i], cudaEventDisableTiming));
+            CSTR_CUDA_TRY(cudaEventCreateWithFlags(&ws->slice_done[i], cudaEventDisableTiming));
+        }
         CSTR_CUDA_TRY(cudaEventCreateWithFlags(&ws->inputs_free, cudaEventDisableTiming));
         ws->host_ready = 1;
     }
@@ -1155,16 +1247,21 @@ extern "C" int cstr_step_host(const cstr_table_t *const *tables, int32_t n_table
     for (int i = 0, r0 = 0; r0 < batch; ++i, r0 += per) {
         const int rows = batch - r0 < per ? batch - r0 : per;
         const size_t off = (size_t)r0 * (size_t)ld;
-        CSTR_CUDA_TRY(cudaMemcpyAsync((char *)logits_dev + off * esz,
-                                      (const char *)logits_host + off * esz,
-                                      (size_t)rows * (size_t)ld * esz, cudaMemcpyHostToDevice,
-                                      ws->copy_stream));
-        if (noise_host)
-            CSTR_CUDA_TRY(cudaMemcpyAsync(noise_dev + off, noise_host + off,
-                                          (size_t)rows * (size_t)ld * 4, cudaMemcpyHostToDevice,
-                                          ws->copy_stream));
-        CSTR_CUDA_TRY(cudaEventRecord(ws->slice_ready[i], ws->copy_stream));
-        CSTR_CUDA_TRY(cudaStreamWaitEvent(stream, ws->slice_ready[i], 0));
+        cudaError_t ce = cudaMemcpyAsync((char *)logits_dev + off * esz,
+                                         (const char *)logits_host + off * esz,
+                                         (size_t)rows * (size_t)ld * esz, cudaMemcpyHostToDevice,
+                                         ws->copy_stream);
+        if (ce == cudaSuccess && noise_host)
+            ce = cudaMemcpyAsync(noise_dev + off, noise_host + off, (size_t)rows * (size_t)ld * 4,
+                                 cudaMemcpyHostToDevice, ws->copy_stream);
+        if (ce == cudaSuccess)
+            ce = cudaEventRecord(ws->slice_ready[i], ws->copy_stream);
+        if (ce == cudaSuccess)
+            ce = cudaStreamWaitEvent(stream, ws->slice_ready[i], 0);
+        if (ce != cudaSuccess) {
+            host_drain(ws, stream);
+            return cstr_fail(CSTR_ERR_CUDA, "cstr_step_host: %s", cudaGetErrorString(ce));
+        }
         cstr_workspace sub = *ws;                // this slice's rows of the scratch
         sub.cell += r0;
         sub.ticket += r0;
@@ -1174,18 +1271,33 @@ extern "C" int cstr_step_host(const cstr_table_t *const *tables, int32_t n_table
                          noise_dev ? noise_dev + off : nullptr, states + r0, states + r0,
                          tokens_dev + r0, (char *)masked_out + off * esz,
                          accept_out ? accept_out + r0 : nullptr, rows, &sub, stream);
+        if (rc == CSTR_OK && masked_host) {      // this slice's penalised logits go down on a third
+            cudaError_t e = cudaEventRecord(ws->slice_done[i], stream);     // stream, beside the uploads
+            if (e == cudaSuccess)
+                e = cudaStreamWaitEvent(ws->down_stream, ws->slice_done[i], 0);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync((char *)masked_host + off * esz, (const char *)masked_out + off * esz,
+                                    (size_t)rows * (size_t)ld * esz, cudaMemcpyDeviceToHost,
+                                    ws->down_stream);
+            if (e != cudaSuccess)
+                rc = cstr_fail(CSTR_ERR_CUDA, "cstr_step_host: %s", cudaGetErrorString(e));
+        }
         if (rc) {
-            cudaStreamSynchronize(ws->copy_stream);
-            cudaStreamSynchronize(stream);
+            host_drain(ws, stream);
             return rc;
         }
     }
-    CSTR_CUDA_TRY(cudaMemcpyAsync(tokens_host, tokens_dev, (size_t)batch * 4, cudaMemcpyDeviceToHost,
-                                  stream));
-    if (states_host)
-        CSTR_CUDA_TRY(cudaMemcpyAsync(states_host, states, (size_t)batch * 4, cudaMemcpyDeviceToHost,
-                                      stream));
-    CSTR_CUDA_TRY(cudaStreamSynchronize(stream));
+    cudaError_t e = cudaMemcpyAsync(tokens_host, tokens_dev, (size_t)batch * 4,
+                                    cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess && states_host)
+        e = cudaMemcpyAsync(states_host, states, (size_t)batch * 4, cudaMemcpyDeviceToHost, stream);
+    // every exit, failures included, waits for all three streams: the caller's host
+    // buffers must not be in use by a copy once the call has returned
+    const cudaError_t e2 = host_drain(ws, stream);
+    if (e == cudaSuccess)
+        e = e2;
+    if (e != cudaSuccess)
+        return cstr_fail(CSTR_ERR_CUDA, "cstr_step_host: %s", cudaGetErrorString(e));
     return CSTR_OK;
 }
 

@@ -25,6 +25,50 @@ int cstr_check_device(int handle_device, const char *what);
                              "%s failed: %s", #expr, cudaGetErrorString(e_));            \
     } while (0)
 
+// Checking build (-DCSTR_BOUNDS_CHECK): kernels compare every index they form
+// into a table, vocabulary or logits array with the array's extent before the
+// access.  A violation is counted in a 4-word record on the device (count,
+// then site / index / extent of the first one) and the access is skipped; no
+// trap, no assert.  In the release build CSTR_INB is the constant true and
+// the checks vanish.
+#define CSTR_SITE_BUILD_TT 1        // builder: DFA table lookup
+#define CSTR_SITE_BUILD_NEXT 2      // builder: store into next
+#define CSTR_SITE_BUILD_MASKT 3     // builder: ballot words
+#define CSTR_SITE_BUILD_VOCAB 4     // builder: descriptors, offsets, bytes
+#define CSTR_SITE_BUILD_STACK 5     // builder: shared-memory stack / staged table
+#define CSTR_SITE_TRANSPOSE 6       // mask transpose: maskT read, mask write
+#define CSTR_SITE_GROUP 7           // duplicate-column pass scratch
+#define CSTR_SITE_EXPAND 8          // duplicate-column pass: row copies
+#define CSTR_SITE_TERMINALS 9       // terminal-label post-pass
+#define CSTR_SITE_STEP_LOGITS 10    // step: logits / noise / masked output
+#define CSTR_SITE_STEP_MASK 11      // step: mask words
+#define CSTR_SITE_STEP_NEXT 12      // step: next-state gather, accept flag
+#define CSTR_SITE_STEP_ROW 13       // step: per-row arrays and scratch
+#define CSTR_SITE_DOWNLOAD 14       // table download decode
+#define CSTR_SITE_PDA 15            // push-down kernels
+#ifdef CSTR_BOUNDS_CHECK
+// Device address of the current device's record (allocated on first use), or null.
+unsigned long long *cstr_oob_record();
+__device__ __forceinline__ bool cstr_in_bounds(unsigned long long *rec, long long idx,
+                                               long long extent, int site)
+{
+    if (idx >= 0 && idx < extent)
+        return true;
+    if (rec && atomicAdd(rec, 1ull) == 0ull) {
+        rec[1] = (unsigned long long)site;
+        rec[2] = (unsigned long long)idx;
+        rec[3] = (unsigned long long)extent;
+    }
+    return false;
+}
+#define CSTR_INB(rec, idx, extent, site) \
+    cstr_in_bounds((rec), (long long)(idx), (long long)(extent), (site))
+#define CSTR_OOB_RECORD() cstr_oob_record()
+#else
+#define CSTR_INB(rec, idx, extent, site) (true)
+#define CSTR_OOB_RECORD() ((unsigned long long *)nullptr)
+#endif
+
 // State ids inside the builder's tables are permuted within blocks of 256:
 // state 256 b + 8 l + j sits at slot 256 b + 32 j + l.  A warp whose lane l
 // owns the 8 consecutive states 8 l .. 8 l + 7 then reads 32 consecutive slots
@@ -126,8 +170,10 @@ struct cstr_workspace {
     unsigned long long *counters;  // DEVICE [2] bad-state rows, empty-mask rows
     // cstr_step_host only (created on its first use): a copy stream and one event
     // per slice of rows, so that uploads run ahead of the step kernels
-    cudaStream_t copy_stream;
+    cudaStream_t copy_stream;      // host -> device
+    cudaStream_t down_stream;      // device -> host (penalised logits, when asked for)
     cudaEvent_t slice_ready[CSTR_HOST_SLICES];
+    cudaEvent_t slice_done[CSTR_HOST_SLICES];
     cudaEvent_t inputs_free;
     int host_ready;
 };
@@ -204,7 +250,9 @@ struct cstr_pda_workspace {
 };
 
 // Kernel launchers (defined in cstr_build.cu / cstr_step.cu).
-int cstr_launch_build(cstr_table *table, const cstr_dfa *dfa, cudaStream_t stream);
+// dense_walk: every token walked from its first byte (no shared prefixes): the baseline
+int cstr_launch_build(cstr_table *table, const cstr_dfa *dfa, cudaStream_t stream,
+                      bool dense_walk = false);
 
 struct cstr_step_args {
     const cstr_table *tables[CSTR_MAX_TABLES];

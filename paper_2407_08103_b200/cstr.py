@@ -13,7 +13,7 @@ import os
 
 import numpy as np
 
-from .build import LIB_PATH
+from .build import CHECK_LIB_PATH, LIB_PATH
 
 CSTR_F32 = 0
 CSTR_BF16 = 1
@@ -23,7 +23,7 @@ CSTR_STATIC_MAX_BATCH = 4096
 EXPORTS = [
     "cstr_load_dfa", "cstr_load_dfa_terminals", "cstr_free_dfa", "cstr_load_vocab",
     "cstr_vocab_set_token_sets", "cstr_free_vocab",
-    "cstr_table_create", "cstr_table_build", "cstr_build_token_table", "cstr_table_info",
+    "cstr_table_create", "cstr_table_build", "cstr_table_build_dense", "cstr_build_token_table", "cstr_table_info",
     "cstr_table_download", "cstr_free_table", "cstr_workspace_create", "cstr_free_workspace",
     "cstr_step", "cstr_step_host", "cstr_step_history", "cstr_accept_draft", "cstr_step_status",
     "cstr_step_static", "cstr_last_error",
@@ -34,7 +34,12 @@ EXPORTS = [
     "cstr_pda_accept_draft", "cstr_pda_step_status",
 ]
 
+# entry points of the checking build only (include/cstr_debug.h)
+DEBUG_EXPORTS = ["cstr_debug_bounds_status", "cstr_test_set_group_hash_bits"]
+
 _lib = None
+_libs = {}            # path -> loaded library
+_active_path = None   # None: the release library at LIB_PATH
 
 
 class CstrError(RuntimeError):
@@ -43,25 +48,60 @@ class CstrError(RuntimeError):
         self.code = code
 
 
-def lib():
-    """Load libcstr.so (built in-tree by ``build.build_library``); fail loudly if absent."""
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
+def _load(path, debug):
+    if path not in _libs:
+        if not os.path.exists(path):
             raise RuntimeError(
-                "libcstr.so is missing at %s: build it with "
-                "`python -m paper_2407_08103_b200.build` (needs nvcc); there is no fallback path"
-                % LIB_PATH)
-        L = ctypes.CDLL(LIB_PATH)
-        for name in EXPORTS:
+                "%s is missing at %s: build it with `python -m paper_2407_08103_b200.build%s` "
+                "(needs nvcc); there is no fallback path"
+                % (os.path.basename(path), path, " --check" if debug else ""))
+        L = ctypes.CDLL(path)
+        for name in EXPORTS + (DEBUG_EXPORTS if debug else []):
             fn = getattr(L, name)
             fn.restype = ctypes.c_int
         L.cstr_last_error.restype = ctypes.c_char_p
         for name in ("cstr_free_dfa", "cstr_free_vocab", "cstr_free_table", "cstr_free_workspace",
                      "cstr_free_pda", "cstr_free_pda_table", "cstr_free_pda_workspace"):
             getattr(L, name).restype = None
-        _lib = L
+        L.is_check_build = debug
+        _libs[path] = L
+    return _libs[path]
+
+
+def lib():
+    """The active library: libcstr.so (built in-tree by ``build.build_library``) unless
+    ``use_check_library(True)`` selected the checking build.  Fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        _lib = _load(LIB_PATH, False) if _active_path is None else _load(_active_path, True)
     return _lib
+
+
+def use_check_library(on: bool) -> None:
+    """Route every later call through ``libcstr_check.so`` (bounds-checked kernels, test
+    setters) or back through the release library.  Handles stay bound to the library that
+    made them; do not mix handles of the two in one call."""
+    global _lib, _active_path
+    _active_path = CHECK_LIB_PATH if on else None
+    _lib = None
+
+
+def cstr_debug_bounds_status(reset: bool = True):
+    """Checking build only: (violations, site, index, extent) of the device's bounds record."""
+    L = lib()
+    if not getattr(L, "is_check_build", False):
+        raise RuntimeError("cstr_debug_bounds_status needs the checking build (use_check_library)")
+    out = (ctypes.c_uint64 * 4)()
+    _check(L.cstr_debug_bounds_status(out, ctypes.c_int32(1 if reset else 0)))
+    return tuple(int(x) for x in out)
+
+
+def cstr_test_set_group_hash_bits(bits: int) -> None:
+    """Checking build only: keep ``bits`` bits of the duplicate-column pass's hash (0 = all)."""
+    L = lib()
+    if not getattr(L, "is_check_build", False):
+        raise RuntimeError("cstr_test_set_group_hash_bits needs the checking build")
+    _check(L.cstr_test_set_group_hash_bits(ctypes.c_int32(bits)))
 
 
 def _check(rc):
@@ -89,10 +129,11 @@ class _Handle:
 
     def __init__(self, ptr):
         self.ptr = ptr
+        self._owner = lib() if ptr else None      # freed by the library that made it
 
     def close(self):
         if self.ptr:
-            getattr(lib(), self._free)(self.ptr)
+            getattr(self._owner, self._free)(self.ptr)
             self.ptr = None
 
     def __del__(self):
@@ -190,6 +231,12 @@ def cstr_table_create(vocab: Vocab, max_states: int) -> Table:
 
 def cstr_table_build(table: Table, dfa: Dfa, eos_id: int = -1, stream=None) -> None:
     _check(lib().cstr_table_build(table.ptr, dfa.ptr, ctypes.c_int32(eos_id), _stream_ptr(stream)))
+
+
+def cstr_table_build_dense(table: Table, dfa: Dfa, eos_id: int = -1, stream=None) -> None:
+    """The same table by the per-token walk without shared prefixes (measurement baseline)."""
+    _check(lib().cstr_table_build_dense(table.ptr, dfa.ptr, ctypes.c_int32(eos_id),
+                                        _stream_ptr(stream)))
 
 
 def cstr_build_token_table(dfa: Dfa, vocab_bytes, offsets, eos_id: int = -1, stream=None) -> Table:
@@ -302,11 +349,11 @@ def cstr_step(tables, logits, states, tokens_out, masked_out, ws: Workspace, noi
 
 def cstr_step_host(tables, logits_host, states, tokens_host, logits_dev, masked_out, tokens_dev,
                    ws: Workspace, states_host=None, noise_host=None, noise_dev=None, row_table=None,
-                   accept_out=None, stream=None) -> None:
+                   accept_out=None, masked_host=None, stream=None) -> None:
     """``cstr_step`` for logits in host memory (synchronous).  ``logits_host`` /
     ``noise_host`` / ``tokens_host`` / ``states_host`` are CPU tensors (pinned for speed),
-    ``logits_dev`` / ``noise_dev`` device staging tensors of the same shapes, the rest as
-    in ``cstr_step``."""
+    ``logits_dev`` / ``noise_dev`` device staging tensors of the same shapes, ``masked_host``
+    an optional CPU tensor that receives the penalised logits, the rest as in ``cstr_step``."""
     import torch
     if isinstance(tables, Table):
         tables = [tables]
@@ -323,6 +370,10 @@ def cstr_step_host(tables, logits_host, states, tokens_host, logits_dev, masked_
         if not t.is_cuda or t.dtype != logits_host.dtype or tuple(t.shape) != (batch, ld) \
                 or not t.is_contiguous():
             raise ValueError("%s must be a contiguous CUDA tensor shaped like logits_host" % name)
+    if masked_host is not None and (masked_host.is_cuda or masked_host.dtype != logits_host.dtype
+                                    or tuple(masked_host.shape) != (batch, ld)
+                                    or not masked_host.is_contiguous()):
+        raise ValueError("masked_host must be a contiguous CPU tensor shaped like logits_host")
     if (noise_host is None) != (noise_dev is None):
         raise ValueError("noise_host and noise_dev go together")
     if noise_host is not None:
@@ -341,8 +392,9 @@ def cstr_step_host(tables, logits_host, states, tokens_host, logits_dev, masked_
                                 _dev_ptr(logits_host), ctypes.c_int32(dtype), ctypes.c_int64(ld),
                                 _dev_ptr(noise_host), _dev_ptr(states), _dev_ptr(tokens_host),
                                 _dev_ptr(states_host), _dev_ptr(logits_dev), _dev_ptr(noise_dev),
-                                _dev_ptr(masked_out), _dev_ptr(tokens_dev), _dev_ptr(accept_out),
-                                ctypes.c_int32(batch), ws.ptr, _stream_ptr(stream)))
+                                _dev_ptr(masked_out), _dev_ptr(masked_host), _dev_ptr(tokens_dev),
+                                _dev_ptr(accept_out), ctypes.c_int32(batch), ws.ptr,
+                                _stream_ptr(stream)))
 
 
 def cstr_step_history(tables, logits, states_in, states_out, tokens_out, masked_out, ws: Workspace,

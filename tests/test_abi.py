@@ -33,9 +33,23 @@ def test_every_declared_symbol_is_exported(lib):
     assert set(names) == set(cstr.EXPORTS)
 
 
+def test_checking_build_exports_the_release_symbols_and_the_debug_ones(lib):
+    # libcstr_check.so: same entry points, plus those of include/cstr_debug.h, which the
+    # release library must not have
+    check = ctypes.CDLL(build.build_library(check=True))
+    text = open(os.path.join(ROOT, "include", "cstr_debug.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    debug = sorted(set(re.findall(r"\b(cstr_[a-z_0-9]+)\s*\(", text)))
+    assert debug == sorted(cstr.DEBUG_EXPORTS)
+    for name in declared_functions() + debug:
+        assert hasattr(check, name), name
+    for name in debug:
+        assert not hasattr(lib, name), name
+
+
 def test_header_compiles_as_plain_c(tmp_path):
     src = tmp_path / "t.c"
-    src.write_text('#include "cstr.h"\nint main(void) { return CSTR_OK; }\n')
+    src.write_text('#include "cstr.h"\n#include "cstr_debug.h"\nint main(void) { return CSTR_OK; }\n')
     import subprocess
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
                     "-c", str(src), "-o", str(tmp_path / "t.o")], check=True)
@@ -65,11 +79,12 @@ def test_null_and_range_errors(lib):
     assert lib.cstr_load_vocab(bp, None, 2, ctypes.byref(out)) == -1
     assert lib.cstr_table_create(None, 4, ctypes.byref(out)) == -1
     assert lib.cstr_table_build(None, None, -1, None) == -1
+    assert lib.cstr_table_build_dense(None, None, -1, None) == -1
     assert lib.cstr_workspace_create(0, ctypes.byref(out)) == -2
     assert lib.cstr_step(None, 1, None, None, 0, 0, None, None, None, None, None, 1, None, None) == -1
     assert lib.cstr_step_status(None, None, None, None) == -1
     assert lib.cstr_step_host(None, 1, None, None, 0, 0, None, None, None, None, None, None, None,
-                              None, None, 1, None, None) == -1
+                              None, None, None, 1, None, None) == -1
     assert lib.cstr_table_info(None, None, None, None, None) == -1
     # push-down entry points: validation that precedes every CUDA call
     z = np.zeros(2, dtype=np.int32)

@@ -327,13 +327,20 @@ def test_step_host_matches_the_oracle(dtype, gumbel, pinned):
         d_masked = torch.empty_like(d_logits)
         d_tok = torch.empty((B,), dtype=torch.int32, device=DEV)
         d_acc = torch.empty((B,), dtype=torch.uint8, device=DEV)
+        h_masked = torch.full(h_logits.shape, 7.0, dtype=h_logits.dtype) if t != 1 else None
+        if h_masked is not None and pinned:
+            h_masked = h_masked.pin_memory()
         cstr.cstr_step_host([table], h_logits, d_states, h_tok, d_logits, d_masked, d_tok, ws,
-                            states_host=h_st, noise_host=h_noise, noise_dev=d_noise, accept_out=d_acc)
+                            states_host=h_st, noise_host=h_noise, noise_dev=d_noise, accept_out=d_acc,
+                            masked_host=h_masked)
         ref = oracle.step([dfa], vb, vo, logits, states, noise=noise, threads=8)
         assert np.array_equal(h_tok.numpy(), ref["tokens"])          # no synchronisation needed
         assert np.array_equal(h_st.numpy(), ref["states"])
         assert np.array_equal(d_states.cpu().numpy(), ref["states"])
         assert np.array_equal(d_acc.cpu().numpy(), ref["accept"])
         assert bits_equal(from_dev_logits(d_masked), ref["masked"])
+        if h_masked is not None:                                     # the host copy, no synchronisation needed
+            got = h_masked.view(torch.int16).numpy().view(np.uint16) if dtype == "bf16" else h_masked.numpy()
+            assert bits_equal(got, ref["masked"])
         states = ref["states"]
     assert cstr.cstr_step_status(ws)[0] == 0

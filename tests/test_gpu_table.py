@@ -310,12 +310,28 @@ def test_load_dfa_reports_bad_targets_and_reuses_its_scratch():
         check_table(table, dfa, vb, vo, states=sorted(set([0, S // 2, S - 1])))
 
 
+@pytest.fixture
+def check_build():
+    """Route the test through the checking build (bounds-checked kernels, test setters); the
+    bounds record must be clean before and after."""
+    cstr.use_check_library(True)
+    try:
+        cstr.cstr_debug_bounds_status(reset=True)
+        yield
+        torch.cuda.synchronize()
+        record = cstr.cstr_debug_bounds_status(reset=True)
+        cstr.cstr_test_set_group_hash_bits(0)
+        assert record[0] == 0, "out-of-range index: site %d, index %d, extent %d" % record[1:]
+    finally:
+        cstr.use_check_library(False)
+
+
 @pytest.mark.parametrize("bits", [3, 12])
-def test_duplicate_column_pass_survives_hash_collisions(monkeypatch, bits):
+def test_duplicate_column_pass_survives_hash_collisions(check_build, bits):
     # with only a few hash bits kept, tokens of different class strings land in the same group;
     # the exact comparison must then leave them on their own, and the table stays the oracle's
     from synth import make_vocab_geometric
-    monkeypatch.setenv("CSTR_TEST_GROUP_HASH_BITS", str(bits))
+    cstr.cstr_test_set_group_hash_bits(bits)
     vb, vo = make_vocab_geometric(9000, seed=5)
     dfa = regex_to_dfa(r'"([^"\\]|\\.){0,1100}"')
     (table,) = gpu_tables([dfa], vb, vo, eos_id=17)
@@ -359,3 +375,30 @@ def test_small_automaton_kernels(S):
     check_table(table, dfa, vb, vo, eos_id=eos)
     (table,) = gpu_tables([dfa], vb, vo)
     check_table(table, dfa, vb, vo)
+
+
+@pytest.mark.parametrize("case", ["small", "eos_long_tokens", "json_32k", "wide"])
+def test_dense_walker_baseline_gives_the_same_table(case):
+    # cstr_table_build_dense (every token from its first byte, no trie) exists to measure
+    # what the trie walk saves; it must produce the oracle's table too
+    rng = np.random.default_rng(61)
+    eos, states = -1, None
+    if case == "small":
+        dfa = dense_random_dfa(rng, 70, live=0.7)
+        vb, vo = random_vocab(rng, 1500, max_len=20)
+    elif case == "eos_long_tokens":
+        dfa = dense_random_dfa(rng, 300, live=0.95)
+        vb, vo = random_vocab(rng, 700, max_len=40)
+        eos = 33
+    elif case == "json_32k":
+        dfa = config_dfas("json_32k")[0]
+        vb, vo = config_vocab("json_32k")
+    else:
+        dfa = random_range_dfa(33000, seed=9)
+        vb, vo = random_vocab(rng, 200, max_len=4)
+        states = [0, 1, 255, 256, 32766, 32767, 32768, 32999]
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    table = cstr.cstr_table_create(vocab, dfa[0].shape[0])
+    cstr.cstr_table_build_dense(table, cstr.cstr_load_dfa(*dfa), eos)
+    torch.cuda.synchronize()
+    check_table(table, dfa, vb, vo, eos_id=eos, states=states)
