@@ -40,7 +40,8 @@ unsigned long long g_test_hash_keep = ~0ull;
 struct BuildParams {
     const void *tt;            // [n_classes][row]
     const uint8_t *cls;        // [256]
-    const uint8_t *accept;     // [n_states]
+    const uint8_t *accept;     // [n_states], by the caller's state ids
+    const int32_t *unrank;     // internal id -> caller's id, or null (identity)
     const uint4 *desc;         // [V] sorted tokens
     const uint8_t *bytes;      // raw vocabulary bytes
     const uint32_t *off;       // [V + 1]
@@ -52,6 +53,7 @@ struct BuildParams {
     int tokens_per_cta;
     int warps_s;               // warps of a CTA that split its states ...
     int warps_t;               // ... times warps that split its token chunk
+    int slice_tokens;          // pruning walks: tokens per unit of work drawn by a warp
     // duplicate-column pass: desc lists one representative per class string and
     // its length is only known on the device
     const int32_t *count_dev;  // null: desc holds all V tokens
@@ -105,12 +107,13 @@ __device__ __forceinline__ void unpack_entries(typename Unit<ESZ * NS>::type u, 
 }
 
 // ST: entry type of the DFA table; NT: entry type of next; NS: states per lane;
-// SMEM: the class-major DFA table is staged in shared memory.
+// SMEM: the class-major DFA table is staged in shared memory; PRUNE: skip the
+// walks below a trie node at which all of the warp's states are dead.
 // Lane l of the warp that owns states [q0, q0 + 32 NS) holds the NS consecutive
 // states q0 + NS l + j.  Ballot j therefore carries state q0 + NS l + j in bit l;
 // it is stored as word (q0 / 32 + j) of the token's maskT row and un-permuted
 // by the transpose kernel.
-template <typename ST, typename NT, int NS, bool SMEM>
+template <typename ST, typename NT, int NS, bool SMEM, bool PRUNE>
 __global__ void __launch_bounds__(NS == 8 ? 1024 : 512)
 build_trie_kernel(const __grid_constant__ BuildParams p)
 {
@@ -130,6 +133,10 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     uint32_t *s_rowoff = (uint32_t *)smem;
     SPack *s_stack = (SPack *)(smem + 1024) + (size_t)warp * (kDepth + 1) * 32 + lane;
     const unsigned char *s_tt = smem + 1024 + (size_t)nwarps * (kDepth + 1) * 32 * sizeof(SPack);
+    __shared__ int s_unit_counter;
+    int *const s_unit = &s_unit_counter;
+    if (threadIdx.x == 0)
+        *s_unit = 0;
     for (int i = threadIdx.x; i < 256; i += blockDim.x)
         s_rowoff[i] = (uint32_t)p.cls[i] * (uint32_t)p.row * ESZ;
     if (SMEM) {
@@ -142,25 +149,6 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     __syncthreads();
     const unsigned char *g_tt = (const unsigned char *)p.tt;
 
-    const int warp_s = warp % p.warps_s, warp_t = warp / p.warps_s;
-    const int q0 = (blockIdx.x * p.warps_s + warp_s) * NS * 32;
-    if (q0 >= p.n_states)
-        return;                                          // whole warp out of range
-    const int qbase = q0 + NS * lane;
-    unsigned cur[NS], sinks[NS];
-    unsigned accbits = 0;
-#pragma unroll
-    for (int j = 0; j < NS; ++j) {
-        const bool in = qbase + j < p.n_states;
-        accbits |= (unsigned)(in && p.accept[qbase + j] != 0) << j;
-        cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) * ESZ : sink;
-        sinks[j] = sink;
-    }
-    SPack pk = pack_entries<ESZ, NS>(cur);               // cur[] in packed form, kept in step
-    const NPack dead_out = pack_entries<sizeof(NT), NS>(sinks);
-    s_stack[0] = pk;
-    __syncwarp();
-
     int n_tokens = p.V, tokens_per_cta = p.tokens_per_cta;
     if (p.count_dev) {                                   // representatives only: equal shares
         n_tokens = *p.count_dev;
@@ -168,78 +156,64 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     }
     const int c_begin = blockIdx.y * tokens_per_cta;
     const int c_end = min(n_tokens, c_begin + tokens_per_cta);
-    const int per_t = (c_end - c_begin + p.warps_t - 1) / p.warps_t;
-    const int t_begin = c_begin + warp_t * per_t;
-    const int t_end = min(c_end, t_begin + per_t);
-    if (t_begin >= t_end)
-        return;
-    int depth = 0;                                       // depth of the path held in cur[]
-    uint32_t words[NS > 4 ? NS : 4] = {0u, 0u, 0u, 0u};
-    NPack outp = dead_out;
-    bool prev_eos = true;                                // forces the first token's outputs
+
+    // One unit of work: the warp takes the 32 NS states of state block warp_s of
+    // this CTA through the sorted tokens [t_begin, t_end).
+    auto walk = [&](const int warp_s, const int t_begin, const int t_end) {
+    const int q0 = (blockIdx.x * p.warps_s + warp_s) * NS * 32;
+    if (q0 >= p.n_states || t_begin >= t_end)
+        return;                                          // whole warp out of range
+    const int qbase = q0 + NS * lane;
+    unsigned cur[NS], sinks[NS];
+    unsigned accbits = 0;
+#pragma unroll
+    for (int j = 0; j < NS; ++j) {
+        const bool in = qbase + j < p.n_states;       // the kernel's states are internal ids
+        accbits |= (unsigned)(in && p.accept[p.unrank ? p.unrank[qbase + j] : qbase + j] != 0) << j;
+        cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) * ESZ : sink;
+        sinks[j] = sink;
+    }
+    const NPack dead_out = pack_entries<sizeof(NT), NS>(sinks);
+    __syncwarp();                                        // the previous unit's stack reads are done
+    s_stack[0] = pack_entries<ESZ, NS>(cur);             // depth 0: the states themselves
+    __syncwarp();
     NT *const next_lane = (NT *)p.next + qbase;
     uint32_t *const maskT_warp = p.maskT + (q0 >> 5);
+    const unsigned char *const tbase = SMEM ? s_tt : g_tt;
 
-    uint4 d_next = __ldg(p.desc + t_begin);              // same address in every lane
-    for (int i = t_begin; i < t_end; ++i) {
-        const uint4 d = d_next;
-        if (i + 1 < t_end)
-            d_next = __ldg(p.desc + i + 1);
-        const unsigned tok = d.x;
-        const int n = (int)(d.y & 0xffffffu);
-        const bool first = (i == t_begin);
-        const int shared = first ? 0 : (int)(d.y >> 24);
-        if (shared < depth) {                            // climb back to the shared prefix
-            pk = s_stack[shared * 32];
-            unpack_entries<ESZ, NS>(pk, cur);
-        }
-#pragma unroll 1                         // 1.4 iterations on average: unrolling only adds dispatch code
-        for (int k = shared; k < n; ++k) {
-            unsigned b;
-            const unsigned r = (unsigned)(k - shared);
-            if (!first && r < 8u)
-                b = __byte_perm(d.z, d.w, r) & 0xffu;     // d.z / d.w hold bytes shared .. shared+7
+    // One byte of the walk for the lane's NS states: dst = delta(src, b).
+    auto step = [&](const unsigned (&src)[NS], unsigned (&dst)[NS], unsigned b) {
+        const unsigned char *rowp = tbase + s_rowoff[b];
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+            if (SMEM)
+                dst[j] = (unsigned)*(const SU *)(rowp + src[j]);
             else
-                b = __ldg(p.bytes + __ldg(p.off + tok) + k);
-            const uint32_t ro = s_rowoff[b];
-            if (SMEM) {
-                const unsigned char *rowp = s_tt + ro;
-#pragma unroll
-                for (int j = 0; j < NS; ++j)
-                    cur[j] = (unsigned)*(const SU *)(rowp + cur[j]);
-            } else {
-                const unsigned char *rowp = g_tt + ro;
-#pragma unroll
-                for (int j = 0; j < NS; ++j)
-                    cur[j] = (unsigned)__ldg((const SU *)(rowp + cur[j]));
-            }
-            pk = pack_entries<ESZ, NS>(cur);
-            if (k < kDepth)
-                s_stack[(k + 1) * 32] = pk;
+                dst[j] = (unsigned)__ldg((const SU *)(rowp + src[j]));
         }
-        depth = n;
-        const bool is_eos = (int)tok == p.eos_id;
-        // A token with no byte of its own equals its predecessor: same outputs.
-        // "No edge" goes out as the sink's own code (decoded to -1 by readers),
-        // so live walks are stored as they are; lanes past the last state sit
-        // in the sink from the start.
-        if (n != shared || first || is_eos || prev_eos) {
-            if (n == 0 || is_eos) {      // empty token: no edge.  EOS: allowed exactly in
-                outp = dead_out;         // accepting states, and it finishes the row.
+    };
+    // Every state of the warp sits in the sink (lanes past the last state always do).
+    auto all_dead = [&](const unsigned (&st)[NS]) -> bool {
+        unsigned x = 0u;
 #pragma unroll
-                for (int j = 0; j < NS; ++j)
-                    words[j] = __ballot_sync(kFull, is_eos && ((accbits >> j) & 1u));
-            } else {
-                if constexpr (sizeof(NT) == sizeof(ST))
-                    outp = pk;
-                else
-                    outp = pack_entries<sizeof(NT), NS>(cur);
+        for (int j = 0; j < NS; ++j)
+            x |= st[j] ^ sink;
+        return __all_sync(kFull, x == 0u);
+    };
+
+    // A token's outputs: the lane's entries of the token's row of next, and one
+    // ballot word per state slot of the lane.  "No edge" goes out as the sink's
+    // own code (decoded to -1 by readers), so live walks are stored as they
+    // are; lanes past the last state sit in the sink from the start.
+    NPack outp = dead_out;
+    uint32_t words[NS];
+    auto outputs_of = [&](const unsigned (&st)[NS]) {
+        outp = pack_entries<sizeof(NT), NS>(st);
 #pragma unroll
-                for (int j = 0; j < NS; ++j)
-                    words[j] = __ballot_sync(kFull, cur[j] != sink);
-            }
-        }
-        prev_eos = is_eos;
+        for (int j = 0; j < NS; ++j)
+            words[j] = __ballot_sync(kFull, st[j] != sink);
+    };
+    auto store_outputs = [&](unsigned tok) {
         // lds is a multiple of 256 states: the whole unit is inside the token's row
         *(NPack *)(next_lane + (unsigned long long)tok * p.lds) = outp;
         if (lane == 0) {                 // ballots are warp-uniform; (q0 >> 5) + NS <= lds / 32 < ldb
@@ -248,6 +222,160 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
             if constexpr (NS == 2) *(uint2 *)mrow = make_uint2(words[0], words[1]);
             if constexpr (NS >= 4) *(uint4 *)mrow = make_uint4(words[0], words[1], words[2], words[3]);
             if constexpr (NS == 8) *(uint4 *)(mrow + 4) = make_uint4(words[4], words[5], words[6], words[7]);
+        }
+    };
+
+    // par[] = the lane's states after the first pd bytes of the current trie
+    // path, kept in registers: consecutive tokens are mostly siblings (same
+    // shared prefix, one byte of their own), which then cost one lookup round
+    // and no stack traffic.  The shared-memory stack holds the states at depth
+    // j only while a later token can still resume there, i.e. for j up to the
+    // NEXT token's shared prefix (known from the prefetched descriptor): leaves,
+    // the bulk of the tokens, store nothing.
+    // PRUNE (sparse automata): once every state of the warp is dead at some
+    // depth of the path, every token below that trie node is dead in the whole
+    // warp; such tokens get their dead outputs without any lookup until a token
+    // resumes above that depth (the sparse composition touches live edges only).
+    unsigned par[NS];
+#pragma unroll
+    for (int j = 0; j < NS; ++j)
+        par[j] = cur[j];
+    int pd = 0;
+    int dead_from = 0x7fffffff;                          // depth at which the path died
+    bool first = true;      // the chunk's first token is walked from the root, all its bytes
+                            // from the vocabulary (its descriptor starts at a prefix shared
+                            // with a token of another chunk)
+    uint4 d = __ldg(p.desc + t_begin);                   // same address in every lane
+#pragma unroll 1
+    for (int i = t_begin; i < t_end; ++i) {
+        uint4 dn = make_uint4(0u, 0xffffffffu, 0u, 0u);
+        int nsh = 0;
+        if (i + 1 < t_end) {
+            dn = __ldg(p.desc + i + 1);
+            nsh = (int)(dn.y >> 24);                     // at most kDepth
+        }
+        const unsigned tok = d.x;
+        const int n = (int)(d.y & 0xffffffu);
+        const int sh = first ? 0 : (int)(d.y >> 24);
+        const bool is_eos = (int)tok == p.eos_id;
+        bool dead = PRUNE && sh >= dead_from;
+        if (!dead) {
+            if (PRUNE)
+                dead_from = 0x7fffffff;
+            if (sh != pd) {                              // resume at the shared prefix
+                unpack_entries<ESZ, NS>(s_stack[sh * 32], par);
+                pd = sh;
+            }
+            const int m = n - sh;                        // bytes of its own
+            if (m == 0) {                                // same string as its predecessor (or empty)
+                outputs_of(par);
+            } else {
+                // d.z / d.w hold bytes sh .. sh + 7; the rest (and all bytes of a chunk's
+                // first token) come from the vocabulary
+                const bool inline_bytes = !first;
+                uint32_t gb = 0u;
+                if (!inline_bytes || m > 8)
+                    gb = __ldg(p.off + tok) + (uint32_t)sh;
+                step(par, cur, inline_bytes ? (d.z & 0xffu) : (unsigned)__ldg(p.bytes + gb));
+                if (PRUNE && all_dead(cur)) {
+                    dead_from = sh + 1;
+                    dead = true;
+                }
+                if (m > 1 && !dead) {
+#pragma unroll 1
+                    for (int k = 1; k < m; ++k) {
+                        if (sh + k <= nsh)
+                            s_stack[(sh + k) * 32] = pack_entries<ESZ, NS>(cur);
+                        unsigned b;
+                        if (inline_bytes && k < 8)
+                            b = __byte_perm(d.z, d.w, (unsigned)k) & 0xffu;
+                        else
+                            b = __ldg(p.bytes + gb + k);
+                        step(cur, cur, b);
+                        if (PRUNE && all_dead(cur)) {
+                            dead_from = sh + k + 1;
+                            dead = true;
+                            break;
+                        }
+                    }
+                }
+                if (!dead) {
+                    outputs_of(cur);
+                    if (n <= nsh) {                      // the next token extends (or repeats) this one
+                        s_stack[n * 32] = pack_entries<ESZ, NS>(cur);
+#pragma unroll
+                        for (int j = 0; j < NS; ++j)
+                            par[j] = cur[j];
+                        pd = n;
+                    }
+                }
+            }
+        }
+        if (dead) {
+            outp = dead_out;
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+                words[j] = 0u;
+        }
+        if (n == 0 || is_eos) {          // empty token: no edge.  EOS: allowed exactly in
+            outp = dead_out;             // accepting states, and it finishes the row.
+#pragma unroll
+            for (int j = 0; j < NS; ++j)
+                words[j] = __ballot_sync(kFull, is_eos && ((accbits >> j) & 1u));
+        }
+        store_outputs(tok);
+        first = false;
+        // Tokens that repeat this one (same length, all of it shared: only strings of
+        // at most kDepth bytes can say so) have the same outputs.
+        if (!is_eos && n <= kDepth) {
+            const unsigned same = (unsigned)n | ((unsigned)n << 24);
+            while (dn.y == same && (int)dn.x != p.eos_id) {
+                ++i;
+                store_outputs(dn.x);
+                dn = make_uint4(0u, 0xffffffffu, 0u, 0u);
+                if (i + 1 < t_end)
+                    dn = __ldg(p.desc + i + 1);
+            }
+        }
+        // Tokens below a trie node at which the whole warp is dead: dead outputs, nothing else.
+        if (PRUNE && dead && !is_eos) {
+            while ((int)(dn.y >> 24) >= dead_from && dn.y != 0xffffffffu &&
+                   (int)dn.x != p.eos_id) {
+                ++i;
+                store_outputs(dn.x);
+                dn = make_uint4(0u, 0xffffffffu, 0u, 0u);
+                if (i + 1 < t_end)
+                    dn = __ldg(p.desc + i + 1);
+            }
+        }
+        d = dn;
+    }
+    };  // walk
+
+    if (!PRUNE) {
+        // static shares: state block = warp % warps_s, token slice = warp / warps_s
+        const int per_t = (c_end - c_begin + p.warps_t - 1) / p.warps_t;
+        const int t_begin = c_begin + (warp / p.warps_s) * per_t;
+        walk(warp % p.warps_s, t_begin, min(c_end, t_begin + per_t));
+    } else {
+        // Pruned walks differ widely in cost (a warp whose states all die early
+        // flies through its tokens), so the warps of the CTA draw (state block,
+        // token slice) units from a counter.  State blocks come in ascending
+        // order: the states that allow many bytes are numbered first, so the
+        // long units start first.
+        const int slice = p.slice_tokens;
+        const int n_slices = (c_end - c_begin + slice - 1) / slice;
+        const int n_units = p.warps_s * n_slices;
+        for (;;) {
+            int unit = 0;
+            if (lane == 0)
+                unit = atomicAdd(s_unit, 1);
+            unit = __shfl_sync(kFull, unit, 0);
+            if (unit >= n_units)
+                break;
+            const int ws = unit / n_slices;
+            const int t_begin = c_begin + (unit - ws * n_slices) * slice;
+            walk(ws, t_begin, min(c_end, t_begin + slice));
         }
     }
 }
@@ -259,11 +387,11 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
 // 32 x 32 bit block in registers (no shuffles), and for each of the 32 states
 // the warp stores 32 consecutive mask words of that state's row (128 bytes).
 // Ballot word k of a block of 32 NS states holds state NS l + k of the block
-// in bit l.
+// in bit l.  Ballot rows are in the builder's internal state numbering.
 __global__ void __launch_bounds__(256)
 mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
                       long long ldw, int n_states, int V, int ns,
-                      const uint32_t *__restrict__ reptok)
+                      const uint32_t *__restrict__ reptok, const int32_t *__restrict__ unrank)
 {
     // one padding word per 32 tokens: lane l then reads word 33 l + r, free of bank conflicts
     __shared__ uint32_t tile[8][1024 + 32];
@@ -337,12 +465,15 @@ mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_
         }
         m ^= m << (j >> 1);
     }
-    // now x[s]: state slot s, bit = token: mask word w0 + lane of state first_state + ns s
-    uint32_t *dst = mask + (long long)first_state * ldw + w0 + lane;         // ldw multiple of 32
+    // now x[s]: state slot s, bit = token: mask word w0 + lane of (internal) state
+    // first_state + ns s; the mask rows are indexed by the caller's state ids
+    uint32_t *dst = mask + w0 + lane;                                        // ldw multiple of 32
 #pragma unroll
-    for (int sl = 0; sl < 32; ++sl)
-        if (first_state + ns * sl < n_states)            // warp-uniform
-            dst[(long long)ns * sl * ldw] = x[sl];
+    for (int sl = 0; sl < 32; ++sl) {
+        const int qi = first_state + ns * sl;
+        if (qi < n_states)                               // warp-uniform
+            dst[(long long)(unrank ? unrank[qi] : qi) * ldw] = x[sl];
+    }
 }
 
 // Terminal-label edges (wildcards matched by pre-computed token sets): for
@@ -357,8 +488,9 @@ __global__ void __launch_bounds__(256)
 apply_terminals_kernel(const int32_t *__restrict__ tstate, const uint32_t *__restrict__ tset,
                        const uint32_t *__restrict__ ttarget, int n_term_states, int n_labels,
                        const uint32_t *__restrict__ tsets, const uint32_t *__restrict__ off, int V,
-                       int eos_id, unsigned sink, NT *__restrict__ next, long long lds,
-                       uint32_t *__restrict__ mask, long long ldw)
+                       int eos_id, unsigned sink, const int32_t *__restrict__ rank,
+                       NT *__restrict__ next, long long lds, uint32_t *__restrict__ mask,
+                       long long ldw)
 {
     const int v = blockIdx.x * 256 + threadIdx.x;
     const bool eligible = v < V && v != eos_id && off[min(v, V - 1) + 1] > off[min(v, V - 1)];
@@ -367,11 +499,12 @@ apply_terminals_kernel(const int32_t *__restrict__ tstate, const uint32_t *__res
         return;                                          // no token of this warp is in any set
     NT *row = next + (long long)min(v, V - 1) * lds;
     for (int i = 0; i < n_term_states; ++i) {
-        const int q = tstate[i];
+        const int q = tstate[i];                         // the caller's id: mask row
+        const int qi = rank ? rank[q] : q;               // internal id: entry of next
         const uint32_t labels = mine & tset[i];
         bool fresh = false;
-        if (labels != 0u && (unsigned)row[q] == sink) {
-            row[q] = (NT)ttarget[(long long)i * n_labels + (__ffs((int)labels) - 1)];
+        if (labels != 0u && (unsigned)row[qi] == sink) {
+            row[qi] = (NT)ttarget[(long long)i * n_labels + (__ffs((int)labels) - 1)];
             fresh = true;
         }
         const uint32_t word = __ballot_sync(kFull, fresh);
@@ -812,7 +945,7 @@ build_dense_kernel(const __grid_constant__ BuildParams p)
     const unsigned char *g_tt = (const unsigned char *)p.tt;
     bool ok;
     if (is_eos || n == 0) {
-        ok = is_eos && in && p.accept[q] != 0;
+        ok = is_eos && in && p.accept[p.unrank ? p.unrank[q] : q] != 0;
         cur = sink;
     } else {
         for (uint32_t k = 0; k < n; ++k) {
@@ -827,11 +960,11 @@ build_dense_kernel(const __grid_constant__ BuildParams p)
         p.maskT[(unsigned long long)v * p.ldb + (q >> 5)] = word;      // word k: states 32 k .. 32 k + 31
 }
 
-template <typename ST, typename NT, int NS, bool SMEM>
+template <typename ST, typename NT, int NS, bool SMEM, bool PRUNE>
 cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t smem_bytes,
                         cudaStream_t stream)
 {
-    auto kernel = build_trie_kernel<ST, NT, NS, SMEM>;
+    auto kernel = build_trie_kernel<ST, NT, NS, SMEM, PRUNE>;
     if (smem_bytes > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem_bytes);
@@ -843,12 +976,14 @@ cudaError_t launch_trie(const BuildParams &p, dim3 grid, int threads, size_t sme
 }
 
 template <typename ST, typename NT>
-cudaError_t launch_trie_ns(int ns, bool in_smem, const BuildParams &p, dim3 grid, int threads,
-                           size_t smem_bytes, cudaStream_t stream)
+cudaError_t launch_trie_ns(int ns, bool in_smem, bool prune, const BuildParams &p, dim3 grid,
+                           int threads, size_t smem_bytes, cudaStream_t stream)
 {
-#define CSTR_CASE(N)                                                                          \
-    return in_smem ? launch_trie<ST, NT, N, true>(p, grid, threads, smem_bytes, stream)       \
-                   : launch_trie<ST, NT, N, false>(p, grid, threads, smem_bytes, stream)
+#define CSTR_CASE(N)                                                                               \
+    return in_smem ? (prune ? launch_trie<ST, NT, N, true, true>(p, grid, threads, smem_bytes, stream)    \
+                            : launch_trie<ST, NT, N, true, false>(p, grid, threads, smem_bytes, stream))  \
+                   : (prune ? launch_trie<ST, NT, N, false, true>(p, grid, threads, smem_bytes, stream)   \
+                            : launch_trie<ST, NT, N, false, false>(p, grid, threads, smem_bytes, stream))
     switch (ns) {
     case 1: CSTR_CASE(1);
     case 2: CSTR_CASE(2);
@@ -886,12 +1021,13 @@ static int launch_terminals(cstr_table *t, const cstr_dfa *dfa, cudaStream_t str
         if (t->wide)
             apply_terminals_kernel<uint32_t><<<agrid, 256, 0, stream>>>(
                 dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
-                vc->off, t->V, t->eos_id, sink, (uint32_t *)t->next, t->lds, t->mask, t->ldw);
+                vc->off, t->V, t->eos_id, sink, dfa->rank, (uint32_t *)t->next, t->lds, t->mask,
+                t->ldw);
         else
             apply_terminals_kernel<uint16_t><<<agrid, 256, 0, stream>>>(
                 dfa->tstate, dfa->tset, dfa->ttarget, dfa->n_term_states, dfa->n_labels, vc->tsets,
-                vc->off, t->V, t->eos_id, sink & 0xffffu, (uint16_t *)t->next, t->lds, t->mask,
-                t->ldw);
+                vc->off, t->V, t->eos_id, sink & 0xffffu, dfa->rank, (uint16_t *)t->next, t->lds,
+                t->mask, t->ldw);
         CSTR_CUDA_TRY(cudaGetLastError());
     }
     return CSTR_OK;
@@ -904,6 +1040,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
     p.tt = dfa->tt;
     p.cls = dfa->cls;
     p.accept = dfa->accept;
+    p.unrank = dfa->unrank;
     p.desc = vc->desc;
     p.bytes = vc->bytes;
     p.off = vc->off;
@@ -935,7 +1072,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         const int words = (dfa->n_states + 31) / 32;
         dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
         mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
-                                                      dfa->n_states, t->V, 1, nullptr);
+                                                      dfa->n_states, t->V, 1, nullptr, dfa->unrank);
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }
@@ -966,7 +1103,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         const int words = (dfa->n_states + 31) / 32;
         dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
         mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
-                                                      dfa->n_states, t->V, 1, nullptr);
+                                                      dfa->n_states, t->V, 1, nullptr, nullptr);
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }
@@ -1095,15 +1232,22 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         chunks = (t->V + tokens_per_cta - 1) / tokens_per_cta;
     }
     p.tokens_per_cta = (int)tokens_per_cta;
+    // pruning walks: about four units per warp, so that the counter can even out
+    // state blocks that die early against those that do not
+    p.slice_tokens = (int)((tokens_per_cta + 4LL * warps_t - 1) / (4LL * warps_t));
+    if (p.slice_tokens < 16)
+        p.slice_tokens = 16;
     dim3 grid((unsigned)state_groups, (unsigned)chunks);
 
+    // Sparse automata (most states allow few bytes): prune dead subtrees per warp.
+    const bool prune = dfa->sparse != 0;
     cudaError_t e;
     if (!dfa->wide && !t->wide)
-        e = launch_trie_ns<int16_t, int16_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int16_t, int16_t>(ns, in_smem, prune, p, grid, threads, smem_bytes, stream);
     else if (!dfa->wide && t->wide)
-        e = launch_trie_ns<int16_t, int32_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int16_t, int32_t>(ns, in_smem, prune, p, grid, threads, smem_bytes, stream);
     else
-        e = launch_trie_ns<int32_t, int32_t>(ns, in_smem, p, grid, threads, smem_bytes, stream);
+        e = launch_trie_ns<int32_t, int32_t>(ns, in_smem, prune, p, grid, threads, smem_bytes, stream);
     if (e != cudaSuccess)
         return cstr_fail(CSTR_ERR_CUDA, "cstr_table_build: builder launch: %s",
                          cudaGetErrorString(e));
@@ -1123,7 +1267,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
     if (tgrid.y > 65535u)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: too many states for one launch");
     mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
-                                                     ns, p.reptok);
+                                                     ns, p.reptok, dfa->unrank);
     CSTR_CUDA_TRY(cudaGetLastError());
 
     return launch_terminals(t, dfa, stream);

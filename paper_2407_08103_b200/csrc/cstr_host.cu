@@ -83,10 +83,11 @@ namespace {
 
 // Two order-independent 64-bit hashes per byte column of the raw table
 // (thread = byte, a block sums a slab of rows, slabs combine with atomicAdd);
-// the same pass checks that every target is a state or -1.
+// the same pass checks that every target is a state or -1 and counts the
+// bytes that have an edge out of each state.
 __global__ void __launch_bounds__(256)
 dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_per_block,
-                       unsigned long long *__restrict__ hashes)
+                       unsigned long long *__restrict__ hashes, uint16_t *__restrict__ degree)
 {
     const int b = threadIdx.x;
     const int q0 = blockIdx.x * rows_per_block;
@@ -96,6 +97,9 @@ dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_p
     for (int q = q0; q < q1; ++q) {
         const int32_t target = raw[(long long)q * 256 + b];
         invalid |= target < -1 || target >= n_states;
+        const int edges = __syncthreads_count(target >= 0);      // bytes with an edge out of q
+        if (b == 0)
+            degree[q] = (uint16_t)edges;
         unsigned long long x = (unsigned long long)(unsigned)target +
                                ((unsigned long long)(unsigned)q << 32) + 0x9e3779b97f4a7c15ull;
         x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;        // splitmix64 finaliser: (q, value) -> 64 bits
@@ -111,12 +115,14 @@ dfa_column_hash_kernel(const int32_t *__restrict__ raw, int n_states, int rows_p
 }
 
 // Class-major code table from the raw table, proving the proposed classes on
-// the way: tt[c][PERM(q)] = code(raw[q][rep[c]] or sink); every raw[q][b] must
+// the way: tt[c][PERM(q)] = code(raw[q][rep[c]] or sink), q and the targets
+// taken through `rank` when the automaton is renumbered; every raw[q][b] must
 // equal raw[q][rep[cls[b]]], else *mismatch is set.  A block handles 8 states.
 __global__ void __launch_bounds__(256)
 dfa_build_table_kernel(const int32_t *__restrict__ raw, int n_states, int row, int n_classes,
                        const uint8_t *__restrict__ cls, const uint8_t *__restrict__ rep, int wide,
-                       void *__restrict__ tt, unsigned long long *__restrict__ mismatch)
+                       const int32_t *__restrict__ rank, void *__restrict__ tt,
+                       unsigned long long *__restrict__ mismatch)
 {
     __shared__ int32_t s_row[8][256];
     const int b = threadIdx.x;
@@ -137,9 +143,12 @@ dfa_build_table_kernel(const int32_t *__restrict__ raw, int n_states, int row, i
         const int q = q0 + i;
         if (q >= row)
             continue;
+        // slots and targets in internal ids (the sink and the padding slots map to themselves)
         const int32_t t = s_row[i][rep[c]];
-        const unsigned target = (unsigned)CSTR_PERM(t >= 0 ? t : n_states);
-        const long long at = (long long)c * row + CSTR_PERM(q);
+        const int ti = t >= 0 ? (rank ? rank[t] : t) : n_states;
+        const int qi = (rank && q < n_states) ? rank[q] : q;
+        const unsigned target = (unsigned)CSTR_PERM(ti);
+        const long long at = (long long)c * row + CSTR_PERM(qi);
         if (wide)
             ((uint32_t *)tt)[at] = target * 4u;
         else
@@ -175,6 +184,7 @@ static int first_bad_target(const int32_t *trans, int32_t n_states)
 // used on); larger requests are allocated and freed per call.
 namespace {
 constexpr int32_t kHostPathStates = 512;   // cstr_load_dfa: at or below, no device pre-processing
+constexpr int kManyBytes = 64;             // a state with edges on this many bytes "allows many"
 constexpr size_t kScratchKeep = 64u << 20;
 struct ScratchCache {
     int device = -1;
@@ -245,6 +255,8 @@ extern "C" void cstr_free_dfa(cstr_dfa_t *dfa)
     cudaFree(dfa->tstate);
     cudaFree(dfa->tset);
     cudaFree(dfa->ttarget);
+    cudaFree(dfa->rank);                 // one allocation: rank, then unrank
+    free(dfa->rank_host);
     delete dfa;
 }
 
@@ -358,7 +370,8 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     unsigned char *temp = nullptr;
     bool temp_cached = false;
     if (e == cudaSuccess)
-        e = scratch_acquire(d->device, raw_bytes + hash_bytes + 256, &temp, &temp_cached);
+        e = scratch_acquire(d->device, raw_bytes + hash_bytes + 256 + (size_t)n_states * 2, &temp,
+                            &temp_cached);
     if (e != cudaSuccess) {
         // No usable device: still tell the caller about a malformed table first.
         const int rc_dfa = first_bad_target(trans, n_states);
@@ -371,6 +384,7 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     int32_t *raw = (int32_t *)temp;
     unsigned long long *hashes = (unsigned long long *)(temp + raw_bytes);
     uint8_t *rep_dev = temp + raw_bytes + hash_bytes;
+    uint16_t *degree_dev = (uint16_t *)(temp + raw_bytes + hash_bytes + 256);
     e = cudaMalloc((void **)&d->cls, 256 + (size_t)n_states);
     d->accept = d->cls ? d->cls + 256 : nullptr;
     if (e == cudaSuccess)
@@ -383,17 +397,73 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
     if (e == cudaSuccess) {
         const int rows_per_block = 64;
         dfa_column_hash_kernel<<<(n_states + rows_per_block - 1) / rows_per_block, 256>>>(
-            raw, n_states, rows_per_block, hashes);
+            raw, n_states, rows_per_block, hashes, degree_dev);
         e = cudaGetLastError();
     }
-    if (e == cudaSuccess)
+    std::vector<uint16_t> degree;
+    if (e == cudaSuccess) {
+        try {
+            degree.resize((size_t)n_states);
+        } catch (const std::bad_alloc &) {
+            scratch_release(temp, temp_cached);
+            cstr_free_dfa(d);
+            return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+        }
         e = cudaMemcpy(host_hash, hashes, hash_bytes, cudaMemcpyDeviceToHost);
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpy(degree.data(), degree_dev, (size_t)n_states * 2, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && host_hash[513] != 0) {       // some target is out of range: say which
         scratch_release(temp, temp_cached);
         cstr_free_dfa(d);
         const int rc = first_bad_target(trans, n_states);
         return rc ? rc : cstr_fail(CSTR_ERR_DFA, "cstr_load_dfa: a target is outside [-1, %d)",
                                    n_states);
+    }
+
+    // Sparse automata: when at least one warp's worth of states (256) allows few
+    // bytes each, the builder prunes per warp, and the states that allow many
+    // bytes are numbered first so that they do not keep every warp alive.
+    if (e == cudaSuccess && host_hash[513] == 0) {
+        int32_t many = 0;
+        for (int32_t q = 0; q < n_states; ++q)
+            many += degree[q] >= kManyBytes;
+        d->sparse = n_states - many >= 256;
+        d->n_many = many;
+        bool in_order = true;                    // already "many first"?
+        for (int32_t q = 0; q + 1 < n_states && in_order; ++q)
+            in_order = !(degree[q] < kManyBytes && degree[q + 1] >= kManyBytes);
+        if (d->sparse && many > 0 && !in_order) {
+            d->rank_host = (int32_t *)malloc(((size_t)n_states + 1) * 4);
+            std::vector<int32_t> unrank;
+            try {
+                unrank.resize((size_t)n_states + 1);
+            } catch (const std::bad_alloc &) {
+                free(d->rank_host);
+                d->rank_host = nullptr;
+            }
+            if (!d->rank_host) {
+                scratch_release(temp, temp_cached);
+                cstr_free_dfa(d);
+                return cstr_fail(CSTR_ERR_NOMEM, "cstr_load_dfa: out of host memory");
+            }
+            int32_t at_many = 0, at_few = many;  // stable: each group keeps the caller's order
+            for (int32_t q = 0; q < n_states; ++q) {
+                const int32_t r = degree[q] >= kManyBytes ? at_many++ : at_few++;
+                d->rank_host[q] = r;
+                unrank[r] = q;
+            }
+            d->rank_host[n_states] = n_states;
+            unrank[n_states] = n_states;
+            e = cudaMalloc((void **)&d->rank, ((size_t)n_states + 1) * 8);   // rank, then unrank
+            d->unrank = d->rank ? d->rank + n_states + 1 : nullptr;
+            if (e == cudaSuccess)
+                e = cudaMemcpy(d->rank, d->rank_host, ((size_t)n_states + 1) * 4,
+                               cudaMemcpyHostToDevice);
+            if (e == cudaSuccess)
+                e = cudaMemcpy(d->unrank, unrank.data(), ((size_t)n_states + 1) * 4,
+                               cudaMemcpyHostToDevice);
+        }
     }
 
     uint8_t cls8[256], rep8[256];
@@ -433,7 +503,7 @@ extern "C" int cstr_load_dfa(const int32_t *trans, const uint8_t *accept, int32_
             e = cudaMemcpy(rep_dev, rep8, 256, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) {
             dfa_build_table_kernel<<<(unsigned)((d->row + 7) / 8), 256>>>(
-                raw, n_states, (int)d->row, n_classes, d->cls, rep_dev, d->wide, d->tt,
+                raw, n_states, (int)d->row, n_classes, d->cls, rep_dev, d->wide, d->rank, d->tt,
                 hashes + 512);
             e = cudaGetLastError();
         }
@@ -494,7 +564,9 @@ extern "C" int cstr_load_dfa_terminals(const int32_t *trans, const int32_t *term
             tstate.push_back(q);
             tset.push_back(labels);
             for (int32_t t = 0; t < n_labels; ++t) {
-                const int32_t target = term_trans[(int64_t)q * n_labels + t];
+                int32_t target = term_trans[(int64_t)q * n_labels + t];
+                if (target >= 0 && d->rank_host)         // table entries hold internal ids
+                    target = d->rank_host[target];
                 const uint32_t code = (uint32_t)CSTR_PERM(target < 0 ? n_states : target)
                                       << (d->wide ? 2 : 1);
                 ttarget.push_back(code);
@@ -767,6 +839,20 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
 
 namespace {
 
+// accept flags and (for a renumbered automaton) rank + unrank, which sit back to
+// back in both the DFA and the table, copied into the table in one launch.
+__global__ void __launch_bounds__(256)
+table_meta_kernel(const uint8_t *__restrict__ accept_src, uint8_t *__restrict__ accept_dst,
+                  int n_states, const int32_t *__restrict__ rank_src,
+                  int32_t *__restrict__ rank_dst, int rank_words)
+{
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i < n_states)
+        accept_dst[i] = accept_src[i];
+    else if (i - n_states < rank_words)
+        rank_dst[i - n_states] = rank_src[i - n_states];
+}
+
 // Logical view of a slab of states for cstr_table_download: out[q - q_lo][v] =
 // state reached from q on token v, -1 for "no edge".  The device table is
 // token-major (next[v][q]) and holds codes (CSTR_PERM(target) << shift, the sink
@@ -776,7 +862,8 @@ namespace {
 template <typename NT>
 __global__ void __launch_bounds__(256)
 table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo, int rows,
-                    int q_tile0, int n_states, int shift, int32_t *__restrict__ out)
+                    int q_tile0, int n_states, int shift, const int32_t *__restrict__ rank,
+                    const int32_t *__restrict__ unrank, int32_t *__restrict__ out)
 {
     __shared__ int32_t tile[32][33];
     const int v0 = blockIdx.x * 32;
@@ -787,10 +874,13 @@ table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo,
         const int v = v0 + ty + 8 * k, q = q0 + tx;
         int32_t u = -1;
         if (v < V && q < n_states) {                     // q < lds: inside the token's row
-            const int32_t code = (int32_t)next[(long long)v * lds + q];
+            const int qi = rank ? rank[q] : q;           // the table is indexed by internal ids
+            const int32_t code = (int32_t)next[(long long)v * lds + qi];
             u = CSTR_UNPERM(code >> shift);
             if (u == n_states)
                 u = -1;
+            else if (unrank)
+                u = unrank[u];
         }
         tile[ty + 8 * k][tx] = u;
     }
@@ -821,6 +911,7 @@ extern "C" void cstr_free_table(cstr_table_t *t)
     cudaFree(t->group_count);
     cudaFree(t->group_uniq);
     cudaFree(t->group_blk);
+    cudaFree(t->rank);                   // one allocation: rank, then unrank
     cstr_free_vocab(t->owned_vocab);
     delete t;
 }
@@ -880,6 +971,9 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->group_blk, ((size_t)t->V / 1024 + 1) * 4);
     if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->rank, ((size_t)max_states + 1) * 8);
+    t->unrank = t->rank ? t->rank + max_states + 1 : nullptr;
+    if (e == cudaSuccess)
         e = cudaMemset(t->mask, 0, mask_bytes);   // padding words stay zero for good
     if (e == cudaSuccess)
         e = cudaMemset(t->accept, 0, (size_t)max_states);
@@ -920,8 +1014,17 @@ static int table_build_common(cstr_table_t *table, const cstr_dfa_t *dfa, int32_
     table->start = dfa->start;
     table->eos_id = eos_id;
     table->code_shift = dfa->wide ? 2 : 1;
-    CSTR_CUDA_TRY(cudaMemcpyAsync(table->accept, dfa->accept, (size_t)dfa->n_states,
-                                  cudaMemcpyDeviceToDevice, stream));
+    // the table keeps its own copy of the accept flags and of the state numbering (one small
+    // kernel: separate device-to-device copies of a few KB cost several microseconds each)
+    table->renumbered = dfa->rank != nullptr;
+    table->unrank = table->rank + dfa->n_states + 1;     // as in the DFA: right behind rank
+    {
+        const int words = table->renumbered ? 2 * (dfa->n_states + 1) : 0;
+        const int total = dfa->n_states + words;
+        table_meta_kernel<<<(total + 255) / 256, 256, 0, stream>>>(
+            dfa->accept, table->accept, dfa->n_states, dfa->rank, table->rank, words);
+        CSTR_CUDA_TRY(cudaGetLastError());
+    }
     return cstr_launch_build(table, dfa, stream, dense_walk);
 }
 
@@ -1024,11 +1127,13 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
             if (t->wide)
                 table_decode_kernel<uint32_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
                     (const uint32_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
-                    t->code_shift, stage);
+                    t->code_shift, t->renumbered ? t->rank : nullptr,
+                    t->renumbered ? t->unrank : nullptr, stage);
             else
                 table_decode_kernel<uint16_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
                     (const uint16_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
-                    t->code_shift, stage);
+                    t->code_shift, t->renumbered ? t->rank : nullptr,
+                    t->renumbered ? t->unrank : nullptr, stage);
             e = cudaGetLastError();
             if (e == cudaSuccess)
                 e = cudaMemcpyAsync(next_host + r0 * t->V, stage, (size_t)nr * (size_t)t->V * 4,

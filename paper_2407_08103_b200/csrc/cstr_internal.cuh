@@ -90,6 +90,19 @@ struct cstr_dfa {
     int32_t start;
     int wide;            // 0: int16 entries (n_states + 1 <= 32767), 1: int32 entries
     int32_t n_classes;   // 1..256
+    int sparse;          // most states allow few bytes: the builder prunes dead subtrees
+    int32_t n_many;      // sparse automata: states that allow many bytes (numbered first)
+    // Internal state numbering (null = identity).  For sparse automata the few
+    // states that allow most bytes (free text inside a string, say) are numbered
+    // first, so that they share warps with each other and the many picky
+    // states fill warps that die quickly along the vocabulary trie.  Every
+    // table the builder reads or writes (tt, next, the ballot rows) is indexed
+    // by internal ids; the mask rows, the accept flags and the ABI use the
+    // caller's ids.  rank[q] = internal id of state q, unrank = its inverse,
+    // both with the sink n_states mapped to itself.
+    int32_t *rank;       // DEVICE [n_states + 1] or null
+    int32_t *unrank;     // DEVICE [n_states + 1] or null
+    int32_t *rank_host;  // HOST copy of rank (malloc) or null
     int64_t row;         // entries per class row (n_states + 1, rounded up to 256)
     void *tt;            // DEVICE [n_classes][row]
     uint8_t *cls;        // DEVICE [256] byte -> class
@@ -147,6 +160,10 @@ struct cstr_table {
     int32_t start;
     int32_t eos_id;
     int32_t code_shift; // next entries are CSTR_PERM(state) << code_shift (1: 16-bit DFA, 2: 32-bit)
+    // internal state numbering of the automaton currently held (see cstr_dfa)
+    int renumbered;     // 0: identity, rank / unrank unused
+    int32_t *rank;      // DEVICE [max_states + 1]
+    int32_t *unrank;    // DEVICE [max_states + 1]
     // Scratch of the builder's duplicate-column pass (tokens that read as the same
     // string of byte classes share one walk): an open-addressing table keyed by a
     // 64-bit hash of the class string, each sorted token's representative, the

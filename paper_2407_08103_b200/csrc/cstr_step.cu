@@ -26,6 +26,8 @@ struct TableDesc {
     const uint32_t *mask;
     const void *next;
     const uint8_t *accept;
+    const int32_t *rank;     // caller's state id -> index into a row of next, or null (identity)
+    const int32_t *unrank;   // and back
     long long lds;       // next is token-major: next[token * lds + state]
     long long ldw;
     int n_states;
@@ -165,11 +167,15 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     const TableDesc &tb = p.tab[c.t];
     if (c.active && key != 0ull) {
         tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
-        const long long at = (long long)tok * tb.lds + c.q;
+        // next is indexed by, and holds, the builder's internal state ids
+        const long long at = (long long)tok * tb.lds + (tb.rank ? tb.rank[c.q] : c.q);
         q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const uint16_t *)tb.next)[at];
         q2 = q2 >> tb.code_shift;                       // entries are codes of permuted ids ...
         q2 = CSTR_UNPERM(q2);
-        q2 = (q2 == tb.n_states) ? CSTR_DEAD : q2;      // ... and the sink n_states means "no edge"
+        if (q2 == tb.n_states)
+            q2 = CSTR_DEAD;                             // ... and the sink n_states means "no edge"
+        else if (tb.unrank)
+            q2 = tb.unrank[q2];
     } else if (c.active) {
         atomicAdd(p.counters + 1, 1ull);
     } else if (c.q != -1) {
@@ -455,6 +461,8 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
         p.tab[i].mask = t->mask;
         p.tab[i].next = t->next;
         p.tab[i].accept = t->accept;
+        p.tab[i].rank = t->renumbered ? t->rank : nullptr;
+        p.tab[i].unrank = t->renumbered ? t->unrank : nullptr;
         p.tab[i].lds = t->lds;
         p.tab[i].ldw = t->ldw;
         p.tab[i].n_states = t->n_states;

@@ -402,3 +402,61 @@ def test_dense_walker_baseline_gives_the_same_table(case):
     cstr.cstr_table_build_dense(table, cstr.cstr_load_dfa(*dfa), eos)
     torch.cuda.synchronize()
     check_table(table, dfa, vb, vo, eos_id=eos, states=states)
+
+
+def sparse_dfa(rng, S, many_every=37):
+    """Mostly picky states (1-3 edges each) with a state that allows nearly every byte now and
+    then: the shape of a schema constraint (fixed keys and punctuation around free text)."""
+    trans = np.full((S, 256), -1, dtype=np.int32)
+    for q in range(S):
+        if q % many_every == 3:
+            trans[q] = rng.integers(0, S, size=256)
+            trans[q, rng.random(256) < 0.1] = -1
+        else:
+            for b in rng.choice(np.arange(97, 123), size=int(rng.integers(1, 4)), replace=False):
+                trans[q, b] = int(rng.integers(0, S))
+    return trans, (rng.random(S) < 0.3).astype(np.uint8), int(rng.integers(S))
+
+
+@pytest.mark.parametrize("case", ["plain", "eos", "terminals", "wide", "dense_walker"])
+def test_sparse_automata_are_renumbered_and_pruned(case):
+    # More than 512 states, at least 256 of them picky, the states that allow many bytes
+    # scattered among them: the library numbers those first internally and prunes dead trie
+    # subtrees per warp.  Whole tables, then steps from random states (the step maps state
+    # ids into and out of the internal numbering).
+    from gpu_common import run_step_both
+    rng = np.random.default_rng(91)
+    S = 33100 if case == "wide" else 1300
+    dfa = sparse_dfa(rng, S)
+    V = 3000
+    vb, vo = random_vocab(rng, V, max_len=12, alphabet=b"abcdefghijklmnopqrstuvwxyz ", empty_prob=0.01)
+    eos = 77 if case in ("eos", "terminals") else -1
+    term, sets = None, None
+    if case == "terminals":
+        term = np.full((S, 2), -1, dtype=np.int32)
+        for q in range(0, S, 11):
+            term[q, int(rng.integers(2))] = int(rng.integers(S))
+        sets = rng.integers(0, 4, size=V).astype(np.uint32)
+    if case == "dense_walker":
+        vocab = cstr.cstr_load_vocab(vb, vo)
+        table = cstr.cstr_table_create(vocab, S)
+        cstr.cstr_table_build_dense(table, cstr.cstr_load_dfa(*dfa), eos)
+        torch.cuda.synchronize()
+        tables = [table]
+    else:
+        tables = gpu_tables([dfa], vb, vo, eos_id=eos, term_trans=None if term is None else [term],
+                            token_sets=sets)
+    states = None
+    if case == "wide":
+        states = sorted(set([0, 1, 2, 3, 40, 255, 256, 32767, 32768, S - 1] +
+                            rng.integers(0, S, 30).tolist()))
+    check_table(tables[0], dfa, vb, vo, eos_id=eos, states=states, term_trans=term, token_sets=sets)
+    B = 64
+    logits = rng.standard_normal((B, V)).astype(np.float32)
+    st = rng.integers(-1, S, size=B).astype(np.int32)
+    st[:8] = [3, 40, 77, 0, 1, S - 1, -1, S]            # many-byte states, picky ones, bad ones
+    for _ in range(3):
+        ref = run_step_both([dfa], tables, vb, vo, logits, st, eos_id=eos,
+                            term_trans=None if term is None else [term], token_sets=sets)
+        st = ref["states"]
+        logits = rng.standard_normal((B, V)).astype(np.float32)
