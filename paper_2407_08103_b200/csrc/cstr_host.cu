@@ -863,7 +863,8 @@ template <typename NT>
 __global__ void __launch_bounds__(256)
 table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo, int rows,
                     int q_tile0, int n_states, int shift, const int32_t *__restrict__ rank,
-                    const int32_t *__restrict__ unrank, int32_t *__restrict__ out)
+                    const int32_t *__restrict__ unrank, int32_t *__restrict__ out,
+                    unsigned long long *oob)
 {
     __shared__ int32_t tile[32][33];
     const int v0 = blockIdx.x * 32;
@@ -875,7 +876,8 @@ table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo,
         int32_t u = -1;
         if (v < V && q < n_states) {                     // q < lds: inside the token's row
             const int qi = rank ? rank[q] : q;           // the table is indexed by internal ids
-            const int32_t code = (int32_t)next[(long long)v * lds + qi];
+            const int32_t code = CSTR_INB(oob, qi, lds, CSTR_SITE_DOWNLOAD)
+                                     ? (int32_t)next[(long long)v * lds + qi] : (n_states << shift);
             u = CSTR_UNPERM(code >> shift);
             if (u == n_states)
                 u = -1;
@@ -888,7 +890,8 @@ table_decode_kernel(const NT *__restrict__ next, long long lds, int V, int q_lo,
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const int q = q0 + ty + 8 * k, v = v0 + tx;
-        if (q >= q_lo && q < q_lo + rows && v < V)
+        if (q >= q_lo && q < q_lo + rows && v < V &&
+            CSTR_INB(oob, (long long)(q - q_lo) * V + v, (long long)rows * V, CSTR_SITE_DOWNLOAD))
             out[(long long)(q - q_lo) * V + v] = tile[tx][ty + 8 * k];
     }
 }
@@ -912,6 +915,7 @@ extern "C" void cstr_free_table(cstr_table_t *t)
     cudaFree(t->group_uniq);
     cudaFree(t->group_blk);
     cudaFree(t->rank);                   // one allocation: rank, then unrank
+    cudaFree(t->build_status);
     cstr_free_vocab(t->owned_vocab);
     delete t;
 }
@@ -973,6 +977,10 @@ extern "C" int cstr_table_create(const cstr_vocab_t *vocab, int32_t max_states,
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&t->rank, ((size_t)max_states + 1) * 8);
     t->unrank = t->rank ? t->rank + max_states + 1 : nullptr;
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&t->build_status, 4);
+    if (e == cudaSuccess)
+        e = cudaMemset(t->build_status, 0, 4);
     if (e == cudaSuccess)
         e = cudaMemset(t->mask, 0, mask_bytes);   // padding words stay zero for good
     if (e == cudaSuccess)
@@ -1095,6 +1103,11 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
         return cstr_fail(CSTR_ERR_ARG, "cstr_table_download: states [%d, %d) outside [0, %d)",
                          state_lo, state_hi, t->n_states);
     CSTR_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    unsigned int build_status = 0;
+    CSTR_CUDA_TRY(cudaMemcpy(&build_status, t->build_status, 4, cudaMemcpyDeviceToHost));
+    if (build_status != 0)
+        return cstr_fail(CSTR_ERR_CUDA, "cstr_table_download: a build of this table gave up waiting "
+                         "for its staged rows (status %u); the table is incomplete", build_status);
     const int32_t rows = state_hi - state_lo;
     if (rows == 0)
         return CSTR_OK;
@@ -1128,12 +1141,12 @@ extern "C" int cstr_table_download(const cstr_table_t *t, int32_t state_lo, int3
                 table_decode_kernel<uint32_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
                     (const uint32_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
                     t->code_shift, t->renumbered ? t->rank : nullptr,
-                    t->renumbered ? t->unrank : nullptr, stage);
+                    t->renumbered ? t->unrank : nullptr, stage, CSTR_OOB_RECORD());
             else
                 table_decode_kernel<uint16_t><<<grid, block, 0, (cudaStream_t)cuda_stream>>>(
                     (const uint16_t *)t->next, t->lds, t->V, q_lo, nr, q_tile0, t->n_states,
                     t->code_shift, t->renumbered ? t->rank : nullptr,
-                    t->renumbered ? t->unrank : nullptr, stage);
+                    t->renumbered ? t->unrank : nullptr, stage, CSTR_OOB_RECORD());
             e = cudaGetLastError();
             if (e == cudaSuccess)
                 e = cudaMemcpyAsync(next_host + r0 * t->V, stage, (size_t)nr * (size_t)t->V * 4,

@@ -160,6 +160,9 @@ struct cstr_table {
     int32_t start;
     int32_t eos_id;
     int32_t code_shift; // next entries are CSTR_PERM(state) << code_shift (1: 16-bit DFA, 2: 32-bit)
+    // Status word of the builder's bulk-copy pipeline: non-zero once a bounded wait
+    // of a build gave up (never expected; reported by cstr_table_download).
+    unsigned int *build_status;    // DEVICE [1]
     // internal state numbering of the automaton currently held (see cstr_dfa)
     int renumbered;     // 0: identity, rank / unrank unused
     int32_t *rank;      // DEVICE [max_states + 1]
@@ -208,6 +211,10 @@ struct cstr_pda_view {
     const int2 *edge;
     int NT;
     int n_symbols;
+    // extents, for the checking build's range checks
+    long long act_len;             // entries of act
+    int n_edges;
+    unsigned long long *oob;       // bounds record, null in the release build
 };
 
 // What the step kernel needs to traverse an edge of the token-level PDA.

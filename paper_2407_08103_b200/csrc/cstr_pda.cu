@@ -382,7 +382,8 @@ static cudaError_t enqueue_pda_build(cstr_pda_table *t, cudaStream_t stream)
     cudaError_t e = cudaMemsetAsync(t->ndeep, 0, (size_t)t->n_cfg * 4, stream);
     if (e != cudaSuccess)
         return e;
-    cstr_pda_view P = {pda->act, pda->edge, pda->NT, pda->n_symbols};
+    cstr_pda_view P = {pda->act, pda->edge, pda->NT, pda->n_symbols,
+                       (long long)pda->n_states * pda->NT * 256, pda->n_edges, CSTR_OOB_RECORD()};
     const int warps = 8;
     const unsigned gx = (unsigned)((t->W + warps - 1) / warps);
     pda_state_pass_kernel<<<dim3(gx, (unsigned)pda->n_states), warps * 32, 0, stream>>>(
@@ -620,6 +621,9 @@ static int pda_step_common(const cstr_pda_table_t *table, const void *logits, in
     p.P.edge = pda->edge;
     p.P.NT = pda->NT;
     p.P.n_symbols = pda->n_symbols;
+    p.P.act_len = (long long)pda->n_states * pda->NT * 256;
+    p.P.n_edges = pda->n_edges;
+    p.P.oob = CSTR_OOB_RECORD();
     p.vbytes = table->vocab->bytes;
     p.voff = table->vocab->off;
     p.mask = table->mask;

@@ -34,11 +34,16 @@ __device__ __forceinline__ int pda_walk(const cstr_pda_view &P, int q, const int
         } else {
             t = unknown_below ? P.n_symbols + 1 : P.n_symbols;
         }
-        const uint32_t a = __ldg(P.act + ((long long)q * P.NT + t) * 256 + bytes[k]);
+        const long long at = ((long long)q * P.NT + t) * 256 + bytes[k];
+        if (!CSTR_INB(P.oob, at, P.act_len, CSTR_SITE_PDA))
+            return WALK_DEAD;
+        const uint32_t a = __ldg(P.act + at);
         if (a == CSTR_PDA_NONE)
             return WALK_DEAD;
         if (a == CSTR_PDA_NEEDCTX)
             return WALK_DEEP;
+        if (!CSTR_INB(P.oob, a, P.n_edges, CSTR_SITE_PDA))
+            return WALK_DEAD;
         const int2 e = __ldg(P.edge + a);
         const unsigned meta = (unsigned)e.y;
         if (meta >> 28) {                           // pops the symbol it looked at

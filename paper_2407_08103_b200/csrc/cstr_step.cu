@@ -53,6 +53,8 @@ struct StepParams {
     long long ld;
     int V;
     int n_tables;
+    int batch;           // rows; extent of the per-row arrays
+    unsigned long long *oob;   // checking build: bounds record (null in the release build)
     int nchunks;         // CTAs per row
     int tiles_per_cta;
     int tile_tokens;     // tokens per warp tile of the launched kernel
@@ -107,6 +109,14 @@ __device__ __forceinline__ RowCtx row_context(const StepParams &p)
     RowCtx c;
     c.r = blockIdx.x / p.nchunks;
     c.chunk = blockIdx.x - c.r * p.nchunks;
+    if (!CSTR_INB(p.oob, c.r, p.batch, CSTR_SITE_STEP_ROW)) {   // cannot happen: grid = batch x nchunks
+        c.r = 0;
+        c.t = 0;
+        c.q = -1;
+        c.active = false;
+        c.mrow = nullptr;
+        return c;
+    }
     if (PDA) {                                      // the rows' masks were resolved beforehand
         c.t = 0;
         c.q = 0;
@@ -169,6 +179,10 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
         tok = (int)(0xffffffffu - (unsigned)(key & 0xffffffffull));
         // next is indexed by, and holds, the builder's internal state ids
         const long long at = (long long)tok * tb.lds + (tb.rank ? tb.rank[c.q] : c.q);
+        if (!CSTR_INB(p.oob, at, (long long)p.V * tb.lds, CSTR_SITE_STEP_NEXT) ||
+            !CSTR_INB(p.oob, tok, p.V, CSTR_SITE_STEP_NEXT))
+            q2 = tb.n_states << tb.code_shift;          // decodes to "no edge"
+        else
         q2 = tb.wide ? ((const int32_t *)tb.next)[at] : (int)((const uint16_t *)tb.next)[at];
         q2 = q2 >> tb.code_shift;                       // entries are codes of permuted ids ...
         q2 = CSTR_UNPERM(q2);
@@ -184,7 +198,8 @@ __device__ __forceinline__ void finish_row(const StepParams &p, const RowCtx &c,
     p.tokens[c.r] = tok;
     p.states_out[c.r] = q2;
     if (p.accept_out)
-        p.accept_out[c.r] = (q2 >= 0) ? (uint8_t)(tb.accept[q2] != 0) : (uint8_t)0;
+        p.accept_out[c.r] = (q2 >= 0 && CSTR_INB(p.oob, q2, tb.n_states, CSTR_SITE_STEP_NEXT))
+                                ? (uint8_t)(tb.accept[q2] != 0) : (uint8_t)0;
 }
 
 // ---- per-vector processing ------------------------------------------------
@@ -262,7 +277,10 @@ __device__ __forceinline__ void apply_one(const StepParams &p, const RowCtx &c, 
                                           int i, Best &b)
 {
     bool ok = false;
-    if (c.active)
+    if (!CSTR_INB(p.oob, i, p.V, CSTR_SITE_STEP_LOGITS) ||
+        !CSTR_INB(p.oob, row_off + i, (long long)p.batch * p.ld, CSTR_SITE_STEP_LOGITS))
+        return;
+    if (c.active && CSTR_INB(p.oob, i >> 5, p.tab[c.t].ldw, CSTR_SITE_STEP_MASK))
         ok = (c.mrow[i >> 5] >> (i & 31)) & 1u;
     if (BF16) {
         const unsigned short *in = (const unsigned short *)p.logits + row_off;
@@ -319,7 +337,8 @@ step_vec_kernel(const __grid_constant__ StepParams p)
 #pragma unroll
             for (int j = 0; j < kUnroll; ++j) {
                 const int tok = tok0 + (j * 32 + lane) * VEC;
-                if (tok < Vv)
+                if (tok < Vv && CSTR_INB(p.oob, row_off + tok + VEC - 1, (long long)p.batch * p.ld,
+                                         CSTR_SITE_STEP_LOGITS))
                     __stcs(out + tok / VEC, fill);
             }
             continue;
@@ -328,6 +347,7 @@ step_vec_kernel(const __grid_constant__ StepParams p)
 #pragma unroll
         for (int i = 0; i < WPL; ++i) {
             const long long widx = (long long)tile * WORDS + i * 32 + lane;
+            // (the bound on widx is part of the kernel: the last tile of a row reaches past W)
             mw[i] = (i * 32 + lane < WORDS && widx < p.tab[c.t].ldw) ? __ldg(c.mrow + widx) : 0u;
         }
         uint4 x[kUnroll];
@@ -336,7 +356,8 @@ step_vec_kernel(const __grid_constant__ StepParams p)
         for (int j = 0; j < kUnroll; ++j) {
             const int tok = tok0 + (j * 32 + lane) * VEC;
             x[j] = make_uint4(0u, 0u, 0u, 0u);
-            if (tok < Vv)
+            if (tok < Vv && CSTR_INB(p.oob, row_off + tok + VEC - 1, (long long)p.batch * p.ld,
+                                     CSTR_SITE_STEP_LOGITS))
                 x[j] = __ldcs(in + tok / VEC);
         }
         if (NOISE) {
@@ -391,7 +412,7 @@ step_vec_kernel(const __grid_constant__ StepParams p)
     if (vb.vec >= 0) {                              // warp-uniform
         __syncwarp();
         bool match = false;
-        if (lane < VEC) {
+        if (lane < VEC && CSTR_INB(p.oob, vb.vec + lane, p.V, CSTR_SITE_STEP_LOGITS)) {
             const int i = vb.vec + lane;
             const bool ok = (c.mrow[i >> 5] >> (i & 31)) & 1u;
             float f;
@@ -488,6 +509,8 @@ int cstr_launch_step(const cstr_step_args &a, cudaStream_t stream)
     p.ld = a.ld;
     p.V = a.pda ? a.V : a.tables[0]->V;
     p.n_tables = a.n_tables;
+    p.batch = a.batch;
+    p.oob = CSTR_OOB_RECORD();
 
     const bool bf16 = a.dtype == CSTR_BF16;
     const int esz = bf16 ? 2 : 4;
