@@ -37,14 +37,16 @@ BYTES_PER_LOGIT_F32_GREEDY = 4 + 4 + 1.0 / 8.0    # read + masked write + mask b
 BYTES_PER_TRANSITION = 2 + 1.0 / 8.0              # int16 next entry + mask bit, stores only
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one step launch of the small profiling case
+# dram__bytes_read.sum and dram__bytes_write.sum of one step launch of the small profiling case
 # (`--case small`: 128 rows x 256,000 fp32 logits), from the ncu capture summarised in
 # profiles/step_vec_kernel_fp32_small_case.md, with the SHA-256 of the kernel source the
-# capture ran.  The bench scales it to its own launch by the logits processed (the traffic
-# is proportional to them) and reports null when the source has changed since.
-STEP_TRAFFIC_SMALL_CASE_BYTES = None
+# capture ran.  Reads grow in proportion to the logits per launch; writes are the algorithmic
+# bytes less what is still in L2 when the kernel ends (the same ~54 MB at any size).  The bench
+# reports null when the source has changed since the capture.
+STEP_TRAFFIC_SMALL_CASE_READ_BYTES = 133923840.0
+STEP_TRAFFIC_SMALL_CASE_WRITE_BYTES = 77379584.0
 STEP_TRAFFIC_SMALL_CASE_LOGITS = 128 * 256000
-STEP_TRAFFIC_SOURCE_SHA256 = None
+STEP_TRAFFIC_SOURCE_SHA256 = "b97172796b39aa93f7182c74308a3184f0e9afbb37beeff71bcb395fdce9b03e"
 STEP_KERNEL_SOURCE = os.path.join(ROOT, "paper_2407_08103_b200", "csrc", "cstr_step.cu")
 
 
@@ -55,16 +57,18 @@ def file_sha256(path: str) -> str:
 
 
 def step_traffic_bytes(logits_per_launch: int):
-    """DRAM traffic of one step launch, scaled from the recorded small-case capture; None
+    """DRAM traffic of one fp32 greedy step launch, from the recorded small-case capture; None
     when there is no capture or the step kernel's source is no longer the captured one."""
-    if STEP_TRAFFIC_SMALL_CASE_BYTES is None or STEP_TRAFFIC_SOURCE_SHA256 is None:
+    if STEP_TRAFFIC_SMALL_CASE_READ_BYTES is None or STEP_TRAFFIC_SOURCE_SHA256 is None:
         return None
     try:
         if file_sha256(STEP_KERNEL_SOURCE) != STEP_TRAFFIC_SOURCE_SHA256:
             return None
     except OSError:
         return None
-    return STEP_TRAFFIC_SMALL_CASE_BYTES * (logits_per_launch / STEP_TRAFFIC_SMALL_CASE_LOGITS)
+    scale = logits_per_launch / STEP_TRAFFIC_SMALL_CASE_LOGITS
+    in_l2_at_end = STEP_TRAFFIC_SMALL_CASE_LOGITS * 4 - STEP_TRAFFIC_SMALL_CASE_WRITE_BYTES
+    return STEP_TRAFFIC_SMALL_CASE_READ_BYTES * scale + max(logits_per_launch * 4 - in_l2_at_end, 0.0)
 
 
 def roofline_entry(achieved_gbs: float, peak: float, peak_kind: str, bound: str = "hbm",
@@ -76,6 +80,27 @@ def roofline_entry(achieved_gbs: float, peak: float, peak_kind: str, bound: str 
          "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS}
     d.update(extra)
     return d
+
+
+def time_copy_of(torch, n_bytes_moved: int, dev, stream, reps: int = 12) -> float:
+    """Milliseconds a plain device copy (torch ``copy_``, one read and one write stream) takes
+    to move `n_bytes_moved` bytes in total: what launch, ramp-up and tail cost ANY kernel of
+    that size on this GPU, the measured copy peak being quoted on a 4 GB copy.  Source and
+    destination alternate between two pairs, each pair larger than the L2 where possible."""
+    n = max(int(n_bytes_moved) // 8, 1)                # fp32 elements: 4 bytes read + 4 written
+    pairs = [(torch.empty(n, dtype=torch.float32, device=dev).normal_(),
+              torch.empty(n, dtype=torch.float32, device=dev)) for _ in range(2)]
+    ms = []
+    for i in range(reps + 3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        src, dst = pairs[i & 1]
+        a.record(stream)
+        dst.copy_(src)
+        b.record(stream)
+        b.synchronize()
+        if i >= 3:
+            ms.append(a.elapsed_time(b))
+    return float(np.mean(ms))
 
 
 def inputs_sha256(dfa, vb, vo, first_logits_row) -> str:
@@ -107,11 +132,20 @@ def parse_args():
     ap.add_argument("--build-only", default=None, metavar="WORKLOAD",
                     help="time only the token-table build of one workload (with --case small: the "
                          "4,099-state string DFA / a 4,096-state random DFA; small_constraints: the five "
-                         "small-constraint compiles over the 256,000-token vocabulary) and print its entry; "
+                         "small-constraint compiles over the 256,000-token vocabulary; wildcard: the "
+                         "terminal-label build; random9728_128k: a 9,728-state random DFA over the "
+                         "128,256-token vocabulary, which takes the staged-rows builder) and print its entry; "
                          "for profiler captures, not a bench line")
     ap.add_argument("--walker", default="trie", choices=["trie", "dense"],
                     help="with --build-only: trie = cstr_table_build, dense = cstr_table_build_dense "
                          "(every token from its first byte; the baseline the trie walk is compared with)")
+    ap.add_argument("--step-only", default=None, metavar="VARIANT",
+                    choices=["f32", "bf16", "f32_noise", "bf16_noise", "scalar", "speculative"],
+                    help="time only one instantiation of the step on the small profiling case (128 rows "
+                         "x 256,000 tokens, 4,099-state string DFA): the vector kernel for fp32 / bf16 "
+                         "logits without / with a noise stream, the scalar kernel (row stride not a "
+                         "multiple of 16 bytes), or the speculative-verification pair; for profiler "
+                         "captures, not a bench line")
     ap.add_argument("--pushdown-only", action="store_true",
                     help="time only the push-down step leg (batch 128 with --case small) and print "
                          "its entry; for profiler captures, not a bench line")
@@ -406,6 +440,7 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
     bms = float(np.mean(build_ms))
     bgbs = S0 * V * BYTES_PER_TRANSITION / (bms * 1e-3) / 1e9
     hbm_honest = pool_n * tensor_bytes >= 2 * l2
+    copy_ms = time_copy_of(torch, step_bytes, dev, stream) if hbm_honest else None
     return {
         "workload": name, "vocab": V, "batch": B, "dfa_states": [int(d[0].shape[0]) for d in dfas],
         "dtype": w.dtype, "sampler": "gumbel-max" if w.gumbel else "greedy",
@@ -416,7 +451,9 @@ def time_other_workload(name, torch, cstr, ConstrainedDecoder, dev, stream, peak
             gbs, peak, peak_kind,
             bound="hbm" if hbm_honest else "launch latency (working set sits in L2)",
             bytes_per_logit=bytes_per_logit,
-            logits_pool="%d tensors x %.1f MB" % (pool_n, tensor_bytes / 1e6)),
+            logits_pool="%d tensors x %.1f MB" % (pool_n, tensor_bytes / 1e6),
+            same_size_copy_ms=copy_ms,
+            frac_of_same_size_copy=None if copy_ms is None else copy_ms / kernel_ms),
         "table_build": {"dfa_states": S0, "ms": bms, "transitions_per_s": S0 * V / (bms * 1e-3),
                         "dense_walker_ms": dense_ms,
                         "roofline": roofline_entry(bgbs, peak, peak_kind,
@@ -523,12 +560,16 @@ def time_build_only(torch, cstr, name, case, stream, repeats=4, walker="trie"):
     from synth import random_range_dfa
     from synth.configs import CONFIGS, config_dfas, config_vocab
     from synth.regex_frontend import regex_to_dfa
-    w = CONFIGS[name]
-    vb, vo = config_vocab(name)
+    w = CONFIGS.get(name)
+    vb, vo = config_vocab(name) if name in CONFIGS else (None, None)
     if case == "small" and name == "string_256k":
         dfa = regex_to_dfa(w.regex.replace("{0,4096}", "{0,2048}"))
     elif case == "small" and name == "random10k_256k":
         dfa = random_range_dfa(4096, seed=2)
+    elif name == "random9728_128k":          # the staged-rows builder at a profiler-friendly size
+        w = CONFIGS["random10k_256k"]
+        vb, vo = config_vocab("schema40_128k")
+        dfa = random_range_dfa(9728, seed=2)
     else:
         dfa = config_dfas(name)[0]
     V, S = vo.size - 1, int(dfa[0].shape[0])
@@ -552,6 +593,65 @@ def time_build_only(torch, cstr, name, case, stream, repeats=4, walker="trie"):
     return {"workload": name + (" (small case)" if case == "small" else ""), "walker": walker,
             "dfa_states": S, "vocab": V, "ms": best, "transitions_per_s": S * V / (best * 1e-3),
             "roofline": roofline_entry(gbs, peak, kind, note="stores of next + mask only")}
+
+
+def time_step_variant(torch, cstr, variant, dev, stream, steps=12):
+    """One instantiation of the step kernel on the small profiling case."""
+    from synth.configs import config_vocab
+    from synth.regex_frontend import regex_to_dfa
+    from synth.constraints import STRING_LITERAL_REGEX
+    vb, vo = config_vocab(WORKLOAD)
+    V, B = vo.size - 1, 128
+    dfa = regex_to_dfa(STRING_LITERAL_REGEX.replace("{0,4096}", "{0,2048}"))
+    vocab = cstr.cstr_load_vocab(vb, vo)
+    table = cstr.cstr_table_create(vocab, dfa[0].shape[0])
+    cstr.cstr_table_build(table, cstr.cstr_load_dfa(*dfa), -1, stream)
+    bf16 = variant.startswith("bf16")
+    noise_on = variant.endswith("noise")
+    ld = V + 1 if variant == "scalar" else V          # an odd stride takes the scalar kernel
+    tdtype = torch.bfloat16 if bf16 else torch.float32
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(11)
+    pool = [torch.randn((B, ld), generator=gen, device=dev).to(tdtype) for _ in range(3)]
+    noise = None
+    if noise_on:
+        u = torch.rand((B, ld), generator=gen, device=dev).clamp_(1e-20, 1 - 1e-7)
+        noise = -torch.log(-torch.log(u))
+    out = torch.empty((B, ld), dtype=tdtype, device=dev)
+    ws = cstr.cstr_workspace_create(B)
+    start = torch.full((B,), int(dfa[2]), dtype=torch.int32, device=dev)
+    st = start.clone()
+    st_out = torch.empty_like(st)
+    tok = torch.empty(B, dtype=torch.int32, device=dev)
+    kk, seqs = 7, B // 8
+    draft = torch.zeros((seqs, kk), dtype=torch.int32, device=dev)
+    n_acc = torch.empty(seqs, dtype=torch.int32, device=dev)
+    out_tok = torch.empty((seqs, kk + 1), dtype=torch.int32, device=dev)
+    new_st = torch.empty(seqs, dtype=torch.int32, device=dev)
+    ms = []
+    for i in range(steps + 3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        if variant == "speculative":
+            cstr.cstr_step_history([table], pool[i % 3][:, :V], st, st_out, tok, out[:, :V], ws,
+                                   stream=stream)
+            cstr.cstr_accept_draft(draft, tok.view(seqs, kk + 1), st_out.view(seqs, kk + 1), n_acc,
+                                   out_tok, new_st, stream=stream)
+        else:
+            cstr.cstr_step([table], pool[i % 3][:, :V], st, tok, out[:, :V], ws, noise=None if noise
+                           is None else noise[:, :V], stream=stream)
+            torch.where(st < 0, start, st, out=st)
+        b.record(stream)
+        b.synchronize()
+        if i >= 3:
+            ms.append(a.elapsed_time(b))
+    best = float(np.mean(ms))
+    esz = 2 if bf16 else 4
+    bpl = 2 * esz + (4 if noise_on else 0) + 1.0 / 8.0
+    peak, kind = measured_hbm_peak()
+    return {"variant": variant, "batch": B, "vocab": V, "row_stride": ld, "ms": best,
+            "roofline": roofline_entry(B * V * bpl / (best * 1e-3) / 1e9, peak, kind,
+                                       bytes_per_logit=bpl)}
 
 
 def time_small_compiles(torch, cstr, vocab, stream):
@@ -693,6 +793,17 @@ def main():
     from synth import normal_logits
     libbuild.build_library()
 
+    if args.step_only:
+        print(json.dumps({"step_variant": time_step_variant(torch, cstr, args.step_only, dev,
+                                                            torch.cuda.current_stream())}))
+        return
+    if args.build_only == "wildcard":
+        from synth.configs import config_vocab
+        vb, vo = config_vocab("string_256k")
+        print(json.dumps({"wildcard_table_build": time_wildcard_build(
+            torch, cstr, cstr.cstr_load_vocab(vb, vo), vb, vo, torch.cuda.current_stream(),
+            *measured_hbm_peak())}))
+        return
     if args.build_only == "small_constraints":
         from synth.configs import config_vocab
         vb, vo = config_vocab("string_256k")
@@ -802,6 +913,8 @@ def main():
     kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
     kernel_ms_best = float(np.min([a.elapsed_time(b) for a, b in pairs]))
     active_frac = float((dec.states >= 0).float().mean().item())
+    # a plain copy moving as many bytes as one step launch, timed the same way
+    same_copy_ms = time_copy_of(torch, B * V * BYTES_PER_LOGIT_F32_GREEDY, dev, stream)
 
     # ---- speculative verification: 64 sequences x (7 drafted + 1) positions --------
     # one fused step over the state history (the 512 rows of the workload) + accept / rewind
@@ -1020,10 +1133,12 @@ def main():
         "clocks": clocks,
         "roofline": roofline_entry(
             achieved, peak, peak_kind, traffic=step_traffic_bytes(B * V),
-            traffic_source="ncu DRAM counters of the small profiling case (128 rows), scaled by "
-                           "the logits per launch; null when the kernel source changed since",
+            traffic_source="ncu DRAM counters of the small profiling case (128 rows): reads scaled by "
+                           "the logits per launch, writes = algorithmic less the output still in L2 at "
+                           "the end; null when the kernel source changed since",
             kernel="step_vec_kernel<fp32, greedy>", kernel_ms=kernel_ms,
             kernel_ms_best=kernel_ms_best, launches_timed=ks, bytes_per_launch=step_bytes,
+            same_size_copy_ms=same_copy_ms, frac_of_same_size_copy=same_copy_ms / kernel_ms,
             active_row_fraction_at_end=active_frac),
         "inputs_sha256": inputs_sha256(dfa, vb, vo, host_pool[0][0].numpy()),
         "cpu_baseline": cpu,

@@ -13,7 +13,7 @@
  *     P_{G o V} that reads token v from state q is a chain of byte edges that
  *     spells d(v); its pops are the symbols the chain takes from the stack it
  *     found (in stack order), its pushes what the chain leaves on top.  Edges
- *     may cross terminal boundaries and pop or push several symbols (Figure 5).
+ *     may cross terminal boundaries and pop or push several symbols (Figure 7).
  *   - Algorithm 3, loop body: A = inputs of the edges of P_{G o V} that leave q
  *     and whose pops the current stack s ends with; logits outside A become
  *     -infinity; a token is selected; the matching edge e is traversed:

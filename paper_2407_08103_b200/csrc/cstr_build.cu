@@ -3,7 +3,7 @@
 // with the DFA as in Algorithm 2; Theorem 2 fixes the meaning).
 //
 // The detokenizing transducer of Algorithm 1 has a compact, trie-like form in
-// which tokens share the chain of their common prefix (Section 2.3, Figure 3).
+// which tokens share the chain of their common prefix (Section 2.3, Figure 4).
 // The builder walks exactly that trie: tokens come in lexicographic order with
 // the length of the prefix each shares with its predecessor, and a warp that
 // owns a block of DFA states (one or more states per lane) keeps, per depth of

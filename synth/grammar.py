@@ -14,7 +14,7 @@ Expressions are regular expressions in the dialect of ``regex_frontend`` in
 which ``<name>`` refers to a rule.  Because every recursive call starts and
 ends with a byte of its own, the resulting PDA is real-time: the opening byte
 pushes the call's return address (one stack symbol per call site, like the
-dotted rules of the paper's Figure 4) and jumps to the callee's body, the
+dotted rules of the paper's Figure 6) and jumps to the callee's body, the
 closing byte pops it and resumes after the call.  Every edge reads one byte,
 pops at most one symbol and pushes at most one.  Grammars that are not
 deterministic in this form are rejected.

@@ -91,7 +91,7 @@ class PdaBuilder:
 
 
 def anbn_pda() -> Pda:
-    """The language a^n b^n, n >= 1 (the grammar S -> ab | a S b of Figure 4).
+    """The language a^n b^n, n >= 1 (the grammar S -> ab | a S b of Figure 6).
 
     The first ``a`` pushes a bottom marker, every later ``a`` a counter symbol;
     a ``b`` pops one symbol, and the one that pops the marker reaches the final

@@ -402,7 +402,7 @@ def test_random_pdas_allowed_set_and_traversal_against_direct_walk(seed):
 
 def test_bracketed_grammar_front_end():
     # The PDAs it builds are inputs of both sides; here they are checked as languages:
-    # Figure 4's grammar against the closed form, nested JSON against the json module and
+    # Figure 6's grammar against the closed form, nested JSON against the json module and
     # against the hand-built PDA, and ambiguous grammars are refused.
     from synth import GrammarError, anbn_grammar_pda, grammar_to_pda, json_grammar_pda
     P = anbn_grammar_pda()
