@@ -265,10 +265,13 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
         return (idx < t_end && CSTR_INB(p.oob, idx, n_tokens, CSTR_SITE_BUILD_VOCAB))
                    ? __ldg(p.desc + idx) : no_desc;
     };
-    uint4 d = fetch(t_begin);
+    // Descriptors are loaded two tokens ahead: the NEXT token's shared prefix is
+    // needed while the current token is walked, so one token ahead would put the
+    // load latency back on the critical path.
+    uint4 d = fetch(t_begin), dn = fetch(t_begin + 1);
 #pragma unroll 1
     for (int i = t_begin; i < t_end; ++i) {
-        uint4 dn = fetch(i + 1);
+        uint4 dnn = fetch(i + 2);
         const int nsh = dn.y == 0xffffffffu ? 0 : (int)(dn.y >> 24);    // at most kDepth
         const unsigned tok = d.x;
         const int n = (int)(d.y & 0xffffffu);
@@ -344,26 +347,41 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
         }
         store_outputs(tok);
         first = false;
-        // Tokens that repeat this one (same length, all of it shared: only strings of
-        // at most kDepth bytes can say so) have the same outputs.
-        if (!is_eos && n <= kDepth) {
+        // Runs of tokens with these same outputs: tokens that repeat this one (same
+        // length, all of it shared: only strings of at most kDepth bytes can say so),
+        // and, below a trie node at which the whole warp is dead, every token of the
+        // subtree.  The run's descriptors come 32 at a time, one per lane (a single
+        // load latency per block instead of one per token); a ballot finds where the
+        // run ends and the token ids are handed round by shuffles.
+        if (!is_eos) {
             const unsigned same = (unsigned)n | ((unsigned)n << 24);
-            while (dn.y == same && (int)dn.x != p.eos_id) {
-                ++i;
-                store_outputs(dn.x);
-                dn = fetch(i + 1);
-            }
-        }
-        // Tokens below a trie node at which the whole warp is dead: dead outputs, nothing else.
-        if (PRUNE && dead && !is_eos) {
-            while ((int)(dn.y >> 24) >= dead_from && dn.y != 0xffffffffu &&
-                   (int)dn.x != p.eos_id) {
-                ++i;
-                store_outputs(dn.x);
-                dn = fetch(i + 1);
+            const bool by_death = PRUNE && dead;
+            auto in_run = [&](const uint4 &x) -> bool {
+                if (x.y == 0xffffffffu || (int)x.x == p.eos_id)
+                    return false;
+                return by_death ? (int)(x.y >> 24) >= dead_from : (n <= kDepth && x.y == same);
+            };
+            if (in_run(dn)) {
+                int j = i + 1;                               // first token of the run
+                for (;;) {
+                    const uint4 mine = fetch(j + lane);
+                    const unsigned not_in = ~__ballot_sync(kFull, in_run(mine));
+                    const int len = not_in == 0u ? 32 : __ffs((int)not_in) - 1;
+                    for (int t = 0; t < len; ++t)
+                        store_outputs(__shfl_sync(kFull, mine.x, t));
+                    j += len;
+                    if (len < 32) {                          // lane `len` holds the token after the run
+                        dn = make_uint4(__shfl_sync(kFull, mine.x, len), __shfl_sync(kFull, mine.y, len),
+                                        __shfl_sync(kFull, mine.z, len), __shfl_sync(kFull, mine.w, len));
+                        break;
+                    }
+                }
+                i = j - 1;
+                dnn = fetch(i + 2);
             }
         }
         d = dn;
+        dn = dnn;
     }
     };  // walk
 
@@ -378,8 +396,14 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
         // token slice) units from a counter.  State blocks come in ascending
         // order: the states that allow many bytes are numbered first, so the
         // long units start first.
+        // The slices of a CTA are spread over the whole sorted token list (slice
+        // y, y + gridDim.y, ...): the cost of a stretch of tokens varies along the
+        // list (runs of repeated one-byte tokens are nearly free, long tokens are
+        // not), and a contiguous chunk per CTA would leave some SMs idle early.
         const int slice = p.slice_tokens;
-        const int n_slices = (c_end - c_begin + slice - 1) / slice;
+        const int total_slices = (n_tokens + slice - 1) / slice;
+        const int n_slices = total_slices > (int)blockIdx.y
+                                 ? (total_slices - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y : 0;
         const int n_units = p.warps_s * n_slices;
         for (;;) {
             int unit = 0;
@@ -389,8 +413,8 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
             if (unit >= n_units)
                 break;
             const int ws = unit / n_slices;
-            const int t_begin = c_begin + (unit - ws * n_slices) * slice;
-            walk(ws, t_begin, min(c_end, t_begin + slice));
+            const int t_begin = ((int)blockIdx.y + (unit - ws * n_slices) * (int)gridDim.y) * slice;
+            walk(ws, t_begin, min(n_tokens, t_begin + slice));
         }
     }
 }
