@@ -43,6 +43,7 @@ struct BuildParams {
     const uint8_t *accept;     // [n_states], by the caller's state ids
     const int32_t *unrank;     // internal id -> caller's id, or null (identity)
     const uint4 *desc;         // [V] sorted tokens
+    const uint32_t *pre4;      // [V] first 4 bytes of each sorted token (little endian), or null
     const uint8_t *bytes;      // raw vocabulary bytes
     const uint32_t *off;       // [V + 1]
     void *next;                // [V][lds]
@@ -174,7 +175,8 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
 #pragma unroll
     for (int j = 0; j < NS; ++j) {
         const bool in = qbase + j < p.n_states;       // the kernel's states are internal ids
-        accbits |= (unsigned)(in && p.accept[p.unrank ? p.unrank[qbase + j] : qbase + j] != 0) << j;
+        if (p.eos_id >= 0)                            // accept flags only matter for an EOS token
+            accbits |= (unsigned)(in && p.accept[p.unrank ? p.unrank[qbase + j] : qbase + j] != 0) << j;
         cur[j] = in ? (unsigned)CSTR_PERM(qbase + j) * ESZ : sink;
         sinks[j] = sink;
     }
@@ -269,6 +271,12 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     // needed while the current token is walked, so one token ahead would put the
     // load latency back on the critical path.
     uint4 d = fetch(t_begin), dn = fetch(t_begin + 1);
+    // The walk's first token starts at the root, but its descriptor carries its bytes
+    // only from its shared prefix on; the (at most kDepth) bytes before that come from
+    // pre4, loaded here beside the descriptors, so that no dependent load sits in the
+    // first token's walk.
+    const uint32_t first_pre = (PRUNE && p.pre4) ? __ldg(p.pre4 + t_begin) : 0u;
+    const int first_tsh = (PRUNE && p.pre4) ? (int)(d.y >> 24) : 0;
 #pragma unroll 1
     for (int i = t_begin; i < t_end; ++i) {
         uint4 dnn = fetch(i + 2);
@@ -289,16 +297,43 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
             if (m == 0) {                                // same string as its predecessor (or empty)
                 outputs_of(par);
             } else {
-                // d.z / d.w hold bytes sh .. sh + 7; the rest (and all bytes of a chunk's
-                // first token) come from the vocabulary
-                const bool inline_bytes = !first;
+                // (bz, bw, bx) hold the token's next `inl` bytes from position sh on: d.z / d.w
+                // carry 8 bytes from the shared prefix on; for a walk's first token (sh = 0)
+                // the up to kDepth bytes before that come from pre4.  Whatever lies beyond
+                // comes from the vocabulary.
+                unsigned bz = d.z, bw = d.w, bx = 0u;
+                int inl = 8;
+                if (first) {
+                    if (PRUNE && p.pre4) {       // (only the pruning walks, whose units are short,
+                                                 // gain from it; elsewhere it only costs instructions)
+                        const int tsh = first_tsh;           // 0 .. kDepth
+                        const unsigned long long tail = ((unsigned long long)d.w << 32) | d.z;
+                        const unsigned long long lo = tsh ? ((tail << (8 * tsh)) | first_pre) : tail;
+                        bz = (unsigned)lo;
+                        bw = (unsigned)(lo >> 32);
+                        bx = tsh ? (unsigned)(tail >> (64 - 8 * tsh)) : 0u;
+                        inl = 8 + tsh;
+                    } else {
+                        inl = 0;
+                    }
+                }
                 uint32_t gb = 0u;
-                if ((!inline_bytes || m > 8) && CSTR_INB(p.oob, tok, p.V, CSTR_SITE_BUILD_VOCAB))
+                if (m > inl && CSTR_INB(p.oob, tok, p.V, CSTR_SITE_BUILD_VOCAB))
                     gb = __ldg(p.off + tok) + (uint32_t)sh;
                 // (a token's bytes end inside the vocabulary: gb + m <= bytes_len)
                 const bool bytes_ok = CSTR_INB(p.oob, (long long)gb + m - 1, p.bytes_len, CSTR_SITE_BUILD_VOCAB);
-                step(par, cur, inline_bytes ? (d.z & 0xffu)
-                                            : (bytes_ok ? (unsigned)__ldg(p.bytes + gb) : 0u));
+                auto byte_at = [&](int k) -> unsigned {  // own byte k of the token (position sh + k)
+                    if (PRUNE) {
+                        if (k < 8 && k < inl)
+                            return __byte_perm(bz, bw, (unsigned)k) & 0xffu;
+                        if (k < inl)
+                            return __byte_perm(bx, 0u, (unsigned)(k - 8)) & 0xffu;
+                    } else if (k < inl) {                // inl is 0 or 8 here
+                        return __byte_perm(bz, bw, (unsigned)k) & 0xffu;
+                    }
+                    return bytes_ok ? (unsigned)__ldg(p.bytes + gb + k) : 0u;
+                };
+                step(par, cur, byte_at(0));
                 if (PRUNE && all_dead(cur)) {
                     dead_from = sh + 1;
                     dead = true;
@@ -308,12 +343,7 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
                     for (int k = 1; k < m; ++k) {
                         if (sh + k <= nsh && CSTR_INB(p.oob, sh + k, kDepth + 1, CSTR_SITE_BUILD_STACK))
                             s_stack[(sh + k) * 32] = pack_entries<ESZ, NS>(cur);
-                        unsigned b;
-                        if (inline_bytes && k < 8)
-                            b = __byte_perm(d.z, d.w, (unsigned)k) & 0xffu;
-                        else
-                            b = bytes_ok ? __ldg(p.bytes + gb + k) : 0u;
-                        step(cur, cur, b);
+                        step(cur, cur, byte_at(k));
                         if (PRUNE && all_dead(cur)) {
                             dead_from = sh + k + 1;
                             dead = true;
@@ -1436,6 +1466,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
     p.accept = dfa->accept;
     p.unrank = dfa->unrank;
     p.desc = vc->desc;
+    p.pre4 = vc->pre4;
     p.bytes = vc->bytes;
     p.off = vc->off;
     p.next = t->next;
@@ -1546,6 +1577,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
                                                  vc->off, t->group_desc);
         CSTR_CUDA_TRY(cudaGetLastError());
         p.desc = t->group_desc;
+        p.pre4 = nullptr;            // the representatives' own list has no such array
         p.count_dev = t->group_count;
         p.reptok = t->group_reptok;
     }

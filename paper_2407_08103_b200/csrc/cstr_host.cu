@@ -633,6 +633,7 @@ extern "C" void cstr_free_vocab(cstr_vocab_t *v)
     cudaFree(v->bytes);
     cudaFree(v->off);
     cudaFree(v->desc);
+    cudaFree(v->pre4);
     cudaFree(v->by_len);
     cudaFree(v->tsets);
     delete v;
@@ -673,11 +674,13 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
     std::vector<uint32_t> off32;
     std::vector<int32_t> order;
     std::vector<uint4> desc;
+    std::vector<uint32_t> pre4;
     uint32_t max_len = 0;
     try {
         off32.resize((size_t)vocab_size + 1);
         order.resize((size_t)vocab_size);
         desc.resize((size_t)vocab_size);
+        pre4.resize((size_t)vocab_size);
         for (int32_t v = 0; v <= vocab_size; ++v)
             off32[v] = (uint32_t)offsets[v];
         // lexicographic order of the byte strings (a prefix sorts before its
@@ -777,6 +780,10 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
             memcpy(&r.z, sfx, 4);
             memcpy(&r.w, sfx + 4, 4);
             desc[i] = r;
+            uint32_t head = 0;                   // bytes 0..3: a walk that starts at this token
+            for (uint32_t k = 0; k < 4 && k < n; ++k)    // needs them (its descriptor starts at p)
+                head |= (uint32_t)cur[k] << (8 * k);
+            pre4[i] = head;
         }
     } catch (const std::bad_alloc &) {
         delete vh;
@@ -811,6 +818,10 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
         e = cudaMalloc((void **)&vh->off, ((size_t)vocab_size + 1) * sizeof(uint32_t));
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&vh->desc, (size_t)vocab_size * sizeof(uint4));
+    if (e == cudaSuccess)
+        e = cudaMalloc((void **)&vh->pre4, (size_t)vocab_size * sizeof(uint32_t));
+    if (e == cudaSuccess)
+        e = cudaMemcpy(vh->pre4, pre4.data(), pre4.size() * sizeof(uint32_t), cudaMemcpyHostToDevice);
     if (e == cudaSuccess)
         e = cudaMalloc((void **)&vh->by_len, (size_t)vocab_size * sizeof(uint32_t));
     if (e == cudaSuccess)

@@ -130,6 +130,7 @@ struct cstr_vocab {
     uint8_t *bytes;    // DEVICE [total_bytes + 16]
     uint32_t *off;     // DEVICE [V + 1]
     uint4 *desc;       // DEVICE [V], sorted order
+    uint32_t *pre4;    // DEVICE [V], sorted order: the token's first 4 bytes (little endian, 0-padded)
     uint32_t max_len;
     int32_t n_labels;  // terminal labels with a token set (0 = none attached)
     uint32_t *by_len;  // DEVICE [V] token ids ordered by length (then id): warps of equal-length tokens
