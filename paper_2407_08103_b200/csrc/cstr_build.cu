@@ -449,6 +449,35 @@ build_trie_kernel(const __grid_constant__ BuildParams p)
     }
 }
 
+// The table's own copy of the automaton's accept flags and (for a renumbered
+// automaton) of rank + unrank, which sit back to back in both the DFA and the
+// table.  A few KB: separate device-to-device copies or a kernel of their own
+// would cost several microseconds of every build, so the first CTA of the
+// mask transpose does it on the side; builds without a transpose pass launch
+// table_meta_kernel.
+struct MetaCopy {
+    const uint8_t *accept_src;
+    uint8_t *accept_dst;
+    int n_states;
+    const int32_t *rank_src;
+    int32_t *rank_dst;
+    int rank_words;            // 2 (n_states + 1), or 0 for the identity numbering
+};
+
+__device__ __forceinline__ void meta_copy(const MetaCopy &m, int first, int stride)
+{
+    for (int i = first; i < m.n_states; i += stride)
+        m.accept_dst[i] = m.accept_src[i];
+    for (int i = first; i < m.rank_words; i += stride)
+        m.rank_dst[i] = m.rank_src[i];
+}
+
+__global__ void __launch_bounds__(256)
+table_meta_kernel(const MetaCopy m)
+{
+    meta_copy(m, blockIdx.x * 256 + threadIdx.x, gridDim.x * 256);
+}
+
 // mask[q][w] bit t = validity of token 32 w + t in state q, gathered from the
 // per-token ballot words: 32 x 32 bit-matrix transposes.  A CTA takes 1,024
 // tokens (32 mask words) x 8 ballot words.  Warp j handles ballot word sb0 + j;
@@ -461,11 +490,13 @@ __global__ void __launch_bounds__(256)
 mask_transpose_kernel(const uint32_t *__restrict__ maskT, long long ldb, uint32_t *__restrict__ mask,
                       long long ldw, int n_states, int V, int ns,
                       const uint32_t *__restrict__ reptok, const int32_t *__restrict__ unrank,
-                      long long mask_words, unsigned long long *oob)
+                      long long mask_words, unsigned long long *oob, const MetaCopy meta)
 {
     // one padding word per 32 tokens: lane l then reads word 33 l + r, free of bank conflicts
     __shared__ uint32_t tile[8][1024 + 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        meta_copy(meta, threadIdx.x, 256);
     // x = group of 32 mask words, y = group of 8 ballot words: CTAs launched
     // together write neighbouring 128-byte pieces of the same mask rows (the four
     // CTAs that read the 32-byte quarters of one maskT line meet again in L2)
@@ -1482,6 +1513,13 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
     p.tt_bytes = (long long)dfa->n_classes * dfa->row * (dfa->wide ? 4 : 2);
     p.bytes_len = vc->total_bytes + 16;
     p.mask_words = (long long)t->max_states * t->ldw;
+    MetaCopy meta;
+    meta.accept_src = dfa->accept;
+    meta.accept_dst = t->accept;
+    meta.n_states = dfa->n_states;
+    meta.rank_src = dfa->rank;
+    meta.rank_dst = t->rank;
+    meta.rank_words = dfa->rank ? 2 * (dfa->n_states + 1) : 0;
 
     if (dfa->wide && !t->wide)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: DFA wider than the table");
@@ -1502,7 +1540,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
         mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
                                                       dfa->n_states, t->V, 1, nullptr, dfa->unrank,
-                                                      p.mask_words, p.oob);
+                                                      p.mask_words, p.oob, meta);
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }
@@ -1517,6 +1555,8 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
             (const unsigned short *)dfa->tt, dfa->cls, dfa->accept, vc->bytes, vc->off,
             (unsigned short *)t->next, t->mask, (unsigned)t->lds, t->ldw, (int)dfa->row,
             dfa->n_states, dfa->n_classes, t->V, t->W, t->eos_id, p.bytes_len, p.oob);
+        CSTR_CUDA_TRY(cudaGetLastError());
+        table_meta_kernel<<<1, 256, 0, stream>>>(meta);          // no transpose pass on this path
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }
@@ -1534,7 +1574,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
         mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
                                                       dfa->n_states, t->V, 1, nullptr, nullptr,
-                                                      p.mask_words, p.oob);
+                                                      p.mask_words, p.oob, meta);
         CSTR_CUDA_TRY(cudaGetLastError());
         return launch_terminals(t, dfa, stream);
     }
@@ -1624,7 +1664,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
             dim3 tg((unsigned)(t->ldw / 32), (unsigned)((words + 7) / 8));
             mask_transpose_kernel<<<tg, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw,
                                                           dfa->n_states, t->V, kRowsNS, nullptr,
-                                                          dfa->unrank, p.mask_words, p.oob);
+                                                          dfa->unrank, p.mask_words, p.oob, meta);
             CSTR_CUDA_TRY(cudaGetLastError());
             return launch_terminals(t, dfa, stream);
         }
@@ -1747,7 +1787,7 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
     if (tgrid.y > 65535u)
         return cstr_fail(CSTR_ERR_SHAPE, "cstr_table_build: too many states for one launch");
     mask_transpose_kernel<<<tgrid, 256, 0, stream>>>(t->maskT, t->ldb, t->mask, t->ldw, S, t->V,
-                                                     ns, p.reptok, dfa->unrank, p.mask_words, p.oob);
+                                                     ns, p.reptok, dfa->unrank, p.mask_words, p.oob, meta);
     CSTR_CUDA_TRY(cudaGetLastError());
 
     return launch_terminals(t, dfa, stream);

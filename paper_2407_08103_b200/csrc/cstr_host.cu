@@ -850,20 +850,6 @@ extern "C" int cstr_load_vocab(const uint8_t *vocab_bytes, const int64_t *offset
 
 namespace {
 
-// accept flags and (for a renumbered automaton) rank + unrank, which sit back to
-// back in both the DFA and the table, copied into the table in one launch.
-__global__ void __launch_bounds__(256)
-table_meta_kernel(const uint8_t *__restrict__ accept_src, uint8_t *__restrict__ accept_dst,
-                  int n_states, const int32_t *__restrict__ rank_src,
-                  int32_t *__restrict__ rank_dst, int rank_words)
-{
-    const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i < n_states)
-        accept_dst[i] = accept_src[i];
-    else if (i - n_states < rank_words)
-        rank_dst[i - n_states] = rank_src[i - n_states];
-}
-
 // Logical view of a slab of states for cstr_table_download: out[q - q_lo][v] =
 // state reached from q on token v, -1 for "no edge".  The device table is
 // token-major (next[v][q]) and holds codes (CSTR_PERM(target) << shift, the sink
@@ -1033,17 +1019,10 @@ static int table_build_common(cstr_table_t *table, const cstr_dfa_t *dfa, int32_
     table->start = dfa->start;
     table->eos_id = eos_id;
     table->code_shift = dfa->wide ? 2 : 1;
-    // the table keeps its own copy of the accept flags and of the state numbering (one small
-    // kernel: separate device-to-device copies of a few KB cost several microseconds each)
+    // the table keeps its own copy of the accept flags and of the state numbering; the builder
+    // copies them on the device (cstr_launch_build)
     table->renumbered = dfa->rank != nullptr;
     table->unrank = table->rank + dfa->n_states + 1;     // as in the DFA: right behind rank
-    {
-        const int words = table->renumbered ? 2 * (dfa->n_states + 1) : 0;
-        const int total = dfa->n_states + words;
-        table_meta_kernel<<<(total + 255) / 256, 256, 0, stream>>>(
-            dfa->accept, table->accept, dfa->n_states, dfa->rank, table->rank, words);
-        CSTR_CUDA_TRY(cudaGetLastError());
-    }
     return cstr_launch_build(table, dfa, stream, dense_walk);
 }
 
