@@ -41,10 +41,10 @@ NOMINAL_HBM_GBS = 8000.0
 # (`--case small`: 128 rows x 256,000 fp32 logits), from the ncu capture summarised in
 # profiles/step_vec_kernel_fp32_small_case.md, with the SHA-256 of the kernel source the
 # capture ran.  Reads grow in proportion to the logits per launch; writes are the algorithmic
-# bytes less what is still in L2 when the kernel ends (the same ~54 MB at any size).  The bench
+# bytes less what is still in L2 when the kernel ends (the same ~53 MB at any size).  The bench
 # reports null when the source has changed since the capture.
-STEP_TRAFFIC_SMALL_CASE_READ_BYTES = 133923840.0
-STEP_TRAFFIC_SMALL_CASE_WRITE_BYTES = 77379584.0
+STEP_TRAFFIC_SMALL_CASE_READ_BYTES = 133925376.0
+STEP_TRAFFIC_SMALL_CASE_WRITE_BYTES = 78181632.0
 STEP_TRAFFIC_SMALL_CASE_LOGITS = 128 * 256000
 STEP_TRAFFIC_SOURCE_SHA256 = "b97172796b39aa93f7182c74308a3184f0e9afbb37beeff71bcb395fdce9b03e"
 STEP_KERNEL_SOURCE = os.path.join(ROOT, "paper_2407_08103_b200", "csrc", "cstr_step.cu")
