@@ -146,6 +146,9 @@ def parse_args():
                          "logits without / with a noise stream, the scalar kernel (row stride not a "
                          "multiple of 16 bytes), or the speculative-verification pair; for profiler "
                          "captures, not a bench line")
+    ap.add_argument("--download-only", action="store_true",
+                    help="time only cstr_table_download of a 256-state slab of the small string table "
+                         "(device-side decode + transpose, one copy to the host); for profiler captures")
     ap.add_argument("--pushdown-only", action="store_true",
                     help="time only the push-down step leg (batch 128 with --case small) and print "
                          "its entry; for profiler captures, not a bench line")
@@ -793,6 +796,24 @@ def main():
     from synth import normal_logits
     libbuild.build_library()
 
+    if args.download_only:
+        from synth.configs import config_vocab
+        from synth.constraints import STRING_LITERAL_REGEX
+        from synth.regex_frontend import regex_to_dfa
+        vb, vo = config_vocab(WORKLOAD)
+        dfa = regex_to_dfa(STRING_LITERAL_REGEX.replace("{0,4096}", "{0,2048}"))
+        table = cstr.cstr_table_create(cstr.cstr_load_vocab(vb, vo), dfa[0].shape[0])
+        cstr.cstr_table_build(table, cstr.cstr_load_dfa(*dfa))
+        torch.cuda.synchronize()
+        ms = []
+        for lo in (0, 1000, 2000, 3000):
+            t0 = time.perf_counter()
+            nxt, _ = cstr.cstr_table_download(table, lo, lo + 256)
+            ms.append((time.perf_counter() - t0) * 1e3)
+        print(json.dumps({"table_download": {"states_per_slab": 256, "vocab": vo.size - 1,
+                                             "host_ms_per_slab": float(np.mean(ms[1:])),
+                                             "logical_bytes_per_slab": int(nxt.nbytes)}}))
+        return
     if args.step_only:
         print(json.dumps({"step_variant": time_step_variant(torch, cstr, args.step_only, dev,
                                                             torch.cuda.current_stream())}))
