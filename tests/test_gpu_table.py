@@ -460,3 +460,48 @@ def test_sparse_automata_are_renumbered_and_pruned(case):
                             term_trans=None if term is None else [term], token_sets=sets)
         st = ref["states"]
         logits = rng.standard_normal((B, V)).astype(np.float32)
+
+
+@pytest.mark.parametrize("block", range(6))
+def test_randomised_automaton_and_vocabulary_shapes(block):
+    # Many shapes in one go: automata that are dense, byte-range, sparse (with and without
+    # scattered many-byte states) or of a few byte classes, of 1 to 9,300 states (every builder
+    # kernel and both sides of each threshold), against vocabularies over 256 / 27 / 2 symbols
+    # with many repeated strings, in sorted, reverse-sorted or random order, with and without EOS.
+    for case in range(25):
+        rng = np.random.default_rng(7000 + 25 * block + case)
+        kind = str(rng.choice(["dense", "range", "sparse", "fewclass"]))
+        S = int(rng.choice([1, 2, 15, 16, 17, 63, 64, 65, 200, 255, 256, 257, 511, 512, 513, 700, 1300,
+                            2049, 2500, 9000, 9300]))
+        if kind == "fewclass" and rng.random() < 0.5:
+            S = int(rng.choice([2048, 2300, 4100]))
+        V = int(rng.choice([1, 31, 33, 700, 2049, 8200, 9000]))
+        alphabet = [None, b"abcdefghijklmnopqrstuvwxyz ", b"ab"][int(rng.integers(3))]
+        vb, vo = random_vocab(rng, V, max_len=int(rng.choice([3, 12, 40])), alphabet=alphabet,
+                              empty_prob=0.01)
+        toks = [bytes(vb[vo[v]:vo[v + 1]]) for v in range(V)]
+        dup = float(rng.choice([0.0, 0.3, 0.7]))
+        for v in range(1, V):                            # repeated strings
+            if rng.random() < dup:
+                toks[v] = toks[int(rng.integers(v))]
+        if rng.random() < 0.5:
+            toks.sort(reverse=bool(rng.random() < 0.5))
+        vb, vo = vocab_from_strings(toks)
+        if kind == "dense":
+            dfa = dense_random_dfa(rng, S, live=float(rng.choice([0.3, 0.7, 1.0])))
+        elif kind == "range":
+            dfa = random_range_dfa(S, seed=int(rng.integers(1 << 30)))
+        elif kind == "sparse":
+            dfa = sparse_dfa(rng, S, many_every=int(rng.choice([7, 37, 101, 10 ** 9])))
+        else:
+            k = int(rng.integers(1, 5))
+            cls = rng.integers(0, k, size=256)
+            base = rng.integers(-1, S, size=(S, k)).astype(np.int32)
+            dfa = (np.ascontiguousarray(base[:, cls]), (rng.random(S) < 0.3).astype(np.uint8),
+                   int(rng.integers(S)))
+        eos = int(rng.integers(-1, V)) if rng.random() < 0.4 else -1
+        (table,) = gpu_tables([dfa], vb, vo, eos_id=eos)
+        states = None
+        if S * V > 6_000_000:
+            states = sorted(set([0, 1, S - 1] + rng.integers(0, S, 40).tolist()))
+        check_table(table, dfa, vb, vo, eos_id=eos, states=states, slab=max(S, 1))
