@@ -344,3 +344,31 @@ def test_step_host_matches_the_oracle(dtype, gumbel, pinned):
             assert bits_equal(got, ref["masked"])
         states = ref["states"]
     assert cstr.cstr_step_status(ws)[0] == 0
+
+
+def test_mixed_batch_with_a_renumbered_table():
+    # one sparse automaton (numbered internally: its many-byte states first) beside a dense one
+    # and a small one in the same call: every row's state goes into and out of its own table's
+    # numbering; fp32 and bf16, with and without noise, a few steps each
+    from test_gpu_table import sparse_dfa
+    rng = np.random.default_rng(44)
+    V = 6000
+    vb, vo = random_vocab(rng, V, max_len=8, alphabet=b"abcdefghijklmnopqrstuvwxyz ", empty_prob=0.0)
+    dfas = [sparse_dfa(rng, 1500, many_every=29), dense_random_dfa(rng, 700, live=0.6),
+            dense_random_dfa(rng, 9, live=0.9)]
+    tables = gpu_tables(dfas, vb, vo)
+    B = 96
+    row_table = rng.integers(0, 3, size=B).astype(np.int32)
+    states = np.array([rng.integers(0, dfas[t][0].shape[0]) for t in row_table], dtype=np.int32)
+    states[:4] = [3, 32, 61, 1499]                   # many-byte and picky states of the sparse one
+    row_table[:4] = 0
+    for dtype in ("f32", "bf16"):
+        st = states.copy()
+        for t in range(4):
+            logits = rand_logits(rng, B, V, V, dtype)
+            noise = None
+            if t % 2:
+                noise = -np.log(-np.log(rng.random((B, V)))).astype(np.float32)
+            ref = run_step_both(dfas, tables, vb, vo, logits, st, noise=noise, row_table=row_table)
+            st = ref["states"]
+            st[st < 0] = 0                           # keep rows going
