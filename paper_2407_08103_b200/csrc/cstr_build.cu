@@ -676,20 +676,21 @@ group_insert_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ 
     }
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 group_resolve_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__ bytes,
                      const uint32_t *__restrict__ off, const uint8_t *__restrict__ cls, int V,
                      int eos_id, const unsigned long long *__restrict__ key,
                      const uint32_t *__restrict__ minv, uint32_t slots, unsigned long long keep,
-                     uint32_t *__restrict__ rep, uint32_t *__restrict__ reptok)
+                     uint32_t *__restrict__ rep, uint32_t *__restrict__ reptok,
+                     int32_t *__restrict__ blk)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= V)
-        return;
-    const unsigned tok = desc[i].x;
+    // blocks of 1,024 sorted tokens; the block also counts its representatives (blk)
+    const int i = blockIdx.x * 1024 + threadIdx.x;
+    const bool in = i < V;
+    const unsigned tok = in ? desc[i].x : 0u;
     uint32_t r = (uint32_t)i;
     unsigned rtok = tok;
-    if ((int)tok != eos_id) {
+    if (in && (int)tok != eos_id) {
         const uint32_t b0 = off[tok], n = off[tok + 1] - b0;
         const unsigned long long h = class_string_hash(cls, bytes + b0, n, keep);
         uint32_t slot = (uint32_t)(h >> 20) & (slots - 1);
@@ -715,21 +716,17 @@ group_resolve_kernel(const uint4 *__restrict__ desc, const uint8_t *__restrict__
             }
         }
     }
-    rep[i] = r;
-    reptok[tok] = rtok;
-}
-
-// Representatives in sorted order: a count per block of 1,024 sorted tokens, an
-// exclusive scan of the counts, and a scatter by rank.
-__global__ void __launch_bounds__(1024)
-group_count_kernel(const uint32_t *__restrict__ rep, int V, int32_t *__restrict__ blk)
-{
-    const int i = blockIdx.x * 1024 + threadIdx.x;
-    const int n = __syncthreads_count(i < V && rep[i] == (uint32_t)i);
+    if (in) {
+        rep[i] = r;
+        reptok[tok] = rtok;
+    }
+    const int n = __syncthreads_count(in && r == (uint32_t)i);
     if (threadIdx.x == 0)
         blk[blockIdx.x] = n;
 }
 
+// Representatives in sorted order: the resolve pass leaves a count per block of
+// 1,024 sorted tokens; an exclusive scan of the counts, then a scatter by rank.
 __global__ void __launch_bounds__(1024)
 group_scan_kernel(int32_t *__restrict__ blk, int n_blocks, int32_t *__restrict__ count)
 {
@@ -1604,12 +1601,11 @@ int cstr_launch_build(cstr_table *t, const cstr_dfa *dfa, cudaStream_t stream, b
         group_insert_kernel<<<(unsigned)((t->V - seed + 255) / 256), 256, 0, stream>>>(
             vc->desc, vc->bytes, vc->off, dfa->cls, seed, t->V, t->eos_id, t->group_key,
             t->group_min, t->group_slots, keep);
-        group_resolve_kernel<<<g, 256, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
-                                                    t->eos_id, t->group_key, t->group_min,
-                                                    t->group_slots, keep, t->group_rep,
-                                                    t->group_reptok);
         const int n_blk = (t->V + 1023) / 1024;
-        group_count_kernel<<<n_blk, 1024, 0, stream>>>(t->group_rep, t->V, t->group_blk);
+        group_resolve_kernel<<<n_blk, 1024, 0, stream>>>(vc->desc, vc->bytes, vc->off, dfa->cls, t->V,
+                                                         t->eos_id, t->group_key, t->group_min,
+                                                         t->group_slots, keep, t->group_rep,
+                                                         t->group_reptok, t->group_blk);
         group_scan_kernel<<<1, 1024, 0, stream>>>(t->group_blk, n_blk, t->group_count);
         group_scatter_kernel<<<n_blk, 1024, 0, stream>>>(t->group_rep, t->V, t->group_blk,
                                                          t->group_uniq);
